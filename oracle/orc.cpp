@@ -1,0 +1,659 @@
+// CPU oracle for adaptive self-speculative decoding (arXiv 2410.01028).
+//
+// THIS IS TEST INFRASTRUCTURE, NOT A PRODUCT PATH.  It is a plain, slow,
+// obviously-correct restatement of what the CUDA library computes, used only
+// by the tests, by the smoke check and by the benchmark's CPU-baseline leg.
+// It shares no code, header, table or constant generator with the CUDA
+// library and neither includes the other.
+//
+// What it computes, and the passage each part follows:
+//   * cosine similarity of a hidden-state row before and after a sublayer and
+//     its average over the prompt (ACS, C_l)            -- Section 3.1, Section 3.2 (definition of C_l)
+//   * the Adaptive Draft Model Generator                 -- Algorithm 1, rules 1 and 2 of Section 3.2,
+//                                                           rule subsets of Table 5
+//   * greedy self-speculative decoding: draft with the sub-network D, verify
+//     k+1 tokens with M, accept the matching prefix, replace the first
+//     rejected token with M's                           -- Section 1 (paragraphs 2 and 3)
+//   * the Llama-style dense decoder those run on.  The paper treats the model
+//     as given; the architecture (RMSNorm, rotary embedding with half-split
+//     pairing, SwiGLU, untied LM head, bf16 weights) and the points where
+//     activations are rounded are a reading fixed by this build and listed
+//     in the design notes (roundings R1..R8 below).
+//
+// Arithmetic: every sum is accumulated in double; values are rounded to float
+// or bfloat16 only at the stated points:
+//   R1 residual stream is float                R5 attention output -> bf16
+//   R2 RMSNorm output -> bf16                  R6 o, y = x + o are float
+//   R3 q,k (after RoPE), v -> bf16; cache bf16 R7 silu(g)*u -> bf16; z = y + dn float
+//   R4 scores, softmax: no rounding            R8 logits float; argmax = lowest index of the maximum
+// With ORC_FLAG_NO_ROUNDING the bf16 roundings (R2,R3,R5,R7) are skipped,
+// which gives the "exact arithmetic" variant used to bound the rounding error.
+//
+// Pins (tests/test_oracle_*.py): closed forms of the cosine; hand-derived ADMG
+// sets; brute force over all masks on L=2; prefill == sequential decode;
+// zeroed output projections => identity sublayer, cosine exactly 1; S=1 =>
+// attention output equals the value row; rotation at position 0 is the
+// identity; a numpy restatement of single sublayers; speculative == greedy
+// autoregressive output for every mask and draft length.
+// Parity unpinned: absolute token ids / logits of the random synthetic models
+// (the paper prints no worked example).
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+// ---------------------------------------------------------------- number formats
+inline float bf16_bits_to_float(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+// round a float to the nearest bfloat16 (ties to even); result returned as float
+inline float round_bf16(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u) return f;  // inf / nan unchanged
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+// ---------------------------------------------------------------- dot product
+// sum_k w[k]*x[k], bf16 weights, float activations, double accumulation.
+// The product of two floats is exact in double, so the only rounding is in the
+// eight running sums (element k goes to sum k mod 8) and their final addition.
+__attribute__((target_clones("default", "arch=haswell", "arch=skylake-avx512")))
+double dot_bf16_f32(const uint16_t* w, const float* x, int64_t n) {
+    double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int64_t k = 0;
+    for (; k + 8 <= n; k += 8)
+        for (int j = 0; j < 8; ++j) acc[j] += (double)bf16_bits_to_float(w[k + j]) * (double)x[k + j];
+    for (int j = 0; k < n; ++k, ++j) acc[j] += (double)bf16_bits_to_float(w[k]) * (double)x[k];
+    return ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+}
+
+// out[m][r] = sum_k W[r][k] * x[m][k]     W: [n_out, n_in] bf16 row-major, x: [M, n_in]
+void matvec_rows(const uint16_t* W, int64_t n_out, int64_t n_in, const float* x, int M, double* out) {
+    const int MB = 32;  // rows of x handled per sweep over W (cache blocking only; each dot is independent)
+    for (int m0 = 0; m0 < M; m0 += MB) {
+        const int m1 = std::min(M, m0 + MB);
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < n_out; ++r)
+            for (int m = m0; m < m1; ++m) out[(int64_t)m * n_out + r] = dot_bf16_f32(W + r * n_in, x + (int64_t)m * n_in, n_in);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---------------------------------------------------------------- public structs
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_seq;
+    float rms_eps, rope_theta;
+    uint32_t flags;
+} orc_config;
+
+typedef struct {  // bf16 bit patterns, row-major [out,in], stacked over layers; borrowed, never copied
+    const uint16_t *embed, *lm_head, *final_norm;
+    const uint16_t *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *wg, *wu, *wd;
+} orc_weights;
+
+typedef struct { float alpha; int32_t m, n; uint32_t flags; } orc_admg_params;
+typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; } orc_gen_params;
+typedef struct {
+    int64_t full_passes, draft_passes, verify_passes, rounds, drafted, accepted, prefill_rows;
+    double ms_prefill, ms_full, ms_draft, ms_verify, ms_total;
+} orc_stats;
+
+enum { ORC_FLAG_NO_ROUNDING = 1u };
+enum { ORC_USE_CS = 1u, ORC_USE_RULE1 = 2u, ORC_USE_RULE2 = 4u };
+enum { ORC_MODE_AR = 0, ORC_MODE_SPEC = 1, ORC_MODE_SPEC_MANUAL_MASK = 2 };
+enum { ORC_OK = 0, ORC_ERR_ARG = -1, ORC_ERR_STATE = -2, ORC_ERR_OVERFLOW = -4 };
+
+// ---------------------------------------------------------------- cosine (Section 3.2, summand of C_l)
+// <x,y> / (||x||_2 ||y||_2); the denominator is clamped at 1e-30 so that two
+// zero rows do not divide by zero (the paper is silent on that case).
+double orc_cosine(const float* x, const float* y, int64_t n) {
+    double sxy = 0, sxx = 0, syy = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        sxy += (double)x[i] * (double)y[i];
+        sxx += (double)x[i] * (double)x[i];
+        syy += (double)y[i] * (double)y[i];
+    }
+    return sxy / std::max(std::sqrt(sxx) * std::sqrt(syy), 1e-30);
+}
+
+// ---------------------------------------------------------------- ADMG (Algorithm 1)
+// Layers are numbered l = 1..L as in the paper; array index is l-1.
+//   remove_MLP  = { l : l is a positive multiple of m, l <= L-n }          (rule 1, guarded by rule 2)
+//   remove_ATTN = { l : C_l >= alpha, l <= L-n }  union  remove_MLP         (CS thresholding, rule 2)
+// flags choose the rule subsets of Table 5: without ORC_USE_RULE2 n is taken
+// as 0; without ORC_USE_RULE1 remove_MLP is empty; without ORC_USE_CS the
+// threshold test is dropped.  The comparison is done in float, inclusive.
+int orc_admg(const float* C, int32_t L, float alpha, int32_t m, int32_t n, uint32_t flags, uint8_t* remove_attn,
+             uint8_t* remove_mlp) {
+    if (!C || L < 0 || n < 0 || m < 0 || !remove_attn || !remove_mlp) return ORC_ERR_ARG;
+    const int32_t n_eff = (flags & ORC_USE_RULE2) ? n : 0;
+    for (int32_t l = 1; l <= L; ++l) {
+        const bool removable = l <= L - n_eff;
+        const bool by_rule1 = (flags & ORC_USE_RULE1) && m >= 1 && (l % m == 0) && removable;
+        const bool by_cs = (flags & ORC_USE_CS) && (C[l - 1] >= alpha) && removable;
+        remove_mlp[l - 1] = by_rule1 ? 1 : 0;
+        remove_attn[l - 1] = (by_cs || by_rule1) ? 1 : 0;
+    }
+    return ORC_OK;
+}
+
+// ---------------------------------------------------------------- decoder state
+struct orc_ctx {
+    orc_config c;
+    orc_weights w;
+    bool round;                      // apply the bf16 roundings R2,R3,R5,R7
+    int32_t kv_dim;
+    std::vector<float> rope_cos, rope_sin;  // [max_seq][head_dim/2]
+    std::vector<float> kcache, vcache;      // [L][max_seq][kv_dim]
+    int32_t n_committed = 0;         // positions whose K/V belong to the accepted sequence
+    int32_t draft_cursor = 0;        // next position a draft step writes
+    std::vector<uint8_t> skip_attn, skip_mlp;
+    std::vector<double> sumcos_attn, sumcos_mlp;  // running sums over prompt rows
+    int64_t n_sim_rows = 0;
+    // results of the last pass
+    int32_t last_M = 0;
+    std::vector<float> last_logits;              // [M][V]
+    std::vector<float> last_cos_attn, last_cos_mlp;  // [L][M]; NaN where the sublayer was skipped
+    std::vector<int32_t> last_argmax;            // [M]
+    std::vector<float> last_margin;              // [M] top1 - top2
+    orc_stats stats{};
+    std::string err;
+};
+
+static double now_ms() {
+    return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+int orc_create(const orc_config* cfg, const orc_weights* w, orc_ctx** out) {
+    if (!cfg || !w || !out) return ORC_ERR_ARG;
+    const orc_config& c = *cfg;
+    if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.head_dim % 2 ||
+        c.n_heads * c.head_dim != c.d_model || c.n_heads % c.n_kv_heads || c.d_ffn <= 0 || c.vocab <= 0 || c.max_seq <= 0)
+        return ORC_ERR_ARG;
+    orc_ctx* x = new orc_ctx();
+    x->c = c;
+    x->w = *w;
+    x->round = !(c.flags & ORC_FLAG_NO_ROUNDING);
+    x->kv_dim = c.n_kv_heads * c.head_dim;
+    const int half = c.head_dim / 2;
+    x->rope_cos.resize((size_t)c.max_seq * half);
+    x->rope_sin.resize((size_t)c.max_seq * half);
+    // rotary embedding: pair (j, j+hd/2) of a head is rotated by angle p * theta^(-2j/hd)
+    for (int p = 0; p < c.max_seq; ++p)
+        for (int j = 0; j < half; ++j) {
+            const double ang = (double)p * std::pow((double)c.rope_theta, -2.0 * j / (double)c.head_dim);
+            x->rope_cos[(size_t)p * half + j] = (float)std::cos(ang);
+            x->rope_sin[(size_t)p * half + j] = (float)std::sin(ang);
+        }
+    x->kcache.assign((size_t)c.n_layers * c.max_seq * x->kv_dim, 0.f);
+    x->vcache.assign((size_t)c.n_layers * c.max_seq * x->kv_dim, 0.f);
+    x->skip_attn.assign(c.n_layers, 0);
+    x->skip_mlp.assign(c.n_layers, 0);
+    x->sumcos_attn.assign(c.n_layers, 0.0);
+    x->sumcos_mlp.assign(c.n_layers, 0.0);
+    *out = x;
+    return ORC_OK;
+}
+
+int orc_destroy(orc_ctx* x) {
+    delete x;
+    return ORC_OK;
+}
+
+const char* orc_last_error(orc_ctx* x) { return x ? x->err.c_str() : "null context"; }
+
+// new context: nothing cached, no similarities, empty skip mask
+int orc_reset(orc_ctx* x) {
+    if (!x) return ORC_ERR_ARG;
+    x->n_committed = x->draft_cursor = 0;
+    std::fill(x->skip_attn.begin(), x->skip_attn.end(), 0);
+    std::fill(x->skip_mlp.begin(), x->skip_mlp.end(), 0);
+    std::fill(x->sumcos_attn.begin(), x->sumcos_attn.end(), 0.0);
+    std::fill(x->sumcos_mlp.begin(), x->sumcos_mlp.end(), 0.0);
+    x->n_sim_rows = 0;
+    x->last_M = 0;
+    x->stats = orc_stats{};
+    return ORC_OK;
+}
+
+// RMSNorm of each row, R2:  xn_i = x_i * (mean(x^2)+eps)^(-1/2) * gain_i   (rounded to bf16)
+static void rmsnorm_rows(const orc_ctx* x, const float* in, int M, const uint16_t* gain, float* out) {
+    const int d = x->c.d_model;
+    for (int m = 0; m < M; ++m) {
+        double ss = 0;
+        for (int i = 0; i < d; ++i) ss += (double)in[(size_t)m * d + i] * (double)in[(size_t)m * d + i];
+        const double inv = 1.0 / std::sqrt(ss / d + (double)x->c.rms_eps);
+        for (int i = 0; i < d; ++i) {
+            const float v = (float)((double)in[(size_t)m * d + i] * inv * (double)bf16_bits_to_float(gain[i]));
+            out[(size_t)m * d + i] = x->round ? round_bf16(v) : v;
+        }
+    }
+}
+
+// One pass of M rows (tokens at positions pos0..pos0+M-1) through the decoder.
+//   use_mask : sublayers in the context's skip sets are the identity (the draft model D, Section 1 / 3.2);
+//              a skipped attention sublayer neither reads nor writes its K/V.
+//   acc_sim  : add each row's cosines to the running sums that define C_l (prefill only).
+// Rows are causal among themselves: the row at position p attends to keys 0..p.
+static int forward_rows(orc_ctx* x, const int32_t* tokens, int M, int pos0, bool use_mask, bool acc_sim) {
+    const orc_config& c = x->c;
+    const int d = c.d_model, hd = c.head_dim, half = hd / 2, f = c.d_ffn, V = c.vocab, kvd = x->kv_dim, L = c.n_layers;
+    const int group = c.n_heads / c.n_kv_heads;
+    if (M <= 0 || pos0 < 0) return ORC_ERR_ARG;
+    if ((int64_t)pos0 + M > c.max_seq) return ORC_ERR_OVERFLOW;
+    for (int m = 0; m < M; ++m)
+        if (tokens[m] < 0 || tokens[m] >= V) return ORC_ERR_ARG;
+
+    std::vector<float> h((size_t)M * d), hn((size_t)M * d), y((size_t)M * d), att((size_t)M * d), t((size_t)M * f);
+    std::vector<double> q((size_t)M * d), kk((size_t)M * kvd), vv((size_t)M * kvd), o((size_t)M * d), g((size_t)M * f),
+        u((size_t)M * f);
+    std::vector<float> qf((size_t)M * d);
+    const float nanv = std::nanf("");
+    x->last_M = M;
+    x->last_cos_attn.assign((size_t)L * M, nanv);
+    x->last_cos_mlp.assign((size_t)L * M, nanv);
+
+    // R1: the residual stream starts as the embedding row, widened exactly
+    for (int m = 0; m < M; ++m)
+        for (int i = 0; i < d; ++i) h[(size_t)m * d + i] = bf16_bits_to_float(x->w.embed[(size_t)tokens[m] * d + i]);
+
+    for (int l = 0; l < L; ++l) {
+        // ------------------------------------------------ attention sublayer
+        if (!(use_mask && x->skip_attn[l])) {
+            rmsnorm_rows(x, h.data(), M, x->w.attn_norm + (size_t)l * d, hn.data());
+            matvec_rows(x->w.wq + (size_t)l * d * d, d, d, hn.data(), M, q.data());
+            matvec_rows(x->w.wk + (size_t)l * kvd * d, kvd, d, hn.data(), M, kk.data());
+            matvec_rows(x->w.wv + (size_t)l * kvd * d, kvd, d, hn.data(), M, vv.data());
+            float* kc = x->kcache.data() + (size_t)l * c.max_seq * kvd;
+            float* vc = x->vcache.data() + (size_t)l * c.max_seq * kvd;
+            for (int m = 0; m < M; ++m) {
+                const int p = pos0 + m;
+                const float* rc = x->rope_cos.data() + (size_t)p * half;
+                const float* rs = x->rope_sin.data() + (size_t)p * half;
+                // R3: rotate q and k pairwise, then round; v is only rounded
+                for (int hh = 0; hh < c.n_heads; ++hh)
+                    for (int j = 0; j < half; ++j) {
+                        const float a = (float)q[(size_t)m * d + hh * hd + j], b = (float)q[(size_t)m * d + hh * hd + j + half];
+                        const float ra = (float)((double)a * rc[j] - (double)b * rs[j]);
+                        const float rb = (float)((double)b * rc[j] + (double)a * rs[j]);
+                        qf[(size_t)m * d + hh * hd + j] = x->round ? round_bf16(ra) : ra;
+                        qf[(size_t)m * d + hh * hd + j + half] = x->round ? round_bf16(rb) : rb;
+                    }
+                for (int hh = 0; hh < c.n_kv_heads; ++hh)
+                    for (int j = 0; j < half; ++j) {
+                        const float a = (float)kk[(size_t)m * kvd + hh * hd + j], b = (float)kk[(size_t)m * kvd + hh * hd + j + half];
+                        const float ra = (float)((double)a * rc[j] - (double)b * rs[j]);
+                        const float rb = (float)((double)b * rc[j] + (double)a * rs[j]);
+                        kc[(size_t)p * kvd + hh * hd + j] = x->round ? round_bf16(ra) : ra;
+                        kc[(size_t)p * kvd + hh * hd + j + half] = x->round ? round_bf16(rb) : rb;
+                    }
+                for (int i = 0; i < kvd; ++i) {
+                    const float v = (float)vv[(size_t)m * kvd + i];
+                    vc[(size_t)p * kvd + i] = x->round ? round_bf16(v) : v;
+                }
+            }
+            // R4: softmax(q.k / sqrt(hd)) over keys 0..p, times V
+            const double inv_sqrt_hd = 1.0 / std::sqrt((double)hd);
+#pragma omp parallel for collapse(2) schedule(static)
+            for (int m = 0; m < M; ++m)
+                for (int hh = 0; hh < c.n_heads; ++hh) {
+                    const int p = pos0 + m, kvh = hh / group;
+                    std::vector<double> s(p + 1);
+                    double smax = -INFINITY;
+                    for (int j = 0; j <= p; ++j) {
+                        double acc = 0;
+                        for (int e = 0; e < hd; ++e)
+                            acc += (double)qf[(size_t)m * d + hh * hd + e] * (double)kc[(size_t)j * kvd + kvh * hd + e];
+                        s[j] = acc * inv_sqrt_hd;
+                        smax = std::max(smax, s[j]);
+                    }
+                    double denom = 0;
+                    for (int j = 0; j <= p; ++j) {
+                        s[j] = std::exp(s[j] - smax);
+                        denom += s[j];
+                    }
+                    for (int e = 0; e < hd; ++e) {
+                        double acc = 0;
+                        for (int j = 0; j <= p; ++j) acc += s[j] * (double)vc[(size_t)j * kvd + kvh * hd + e];
+                        const float a = (float)(acc / denom);
+                        att[(size_t)m * d + hh * hd + e] = x->round ? round_bf16(a) : a;  // R5
+                    }
+                }
+            matvec_rows(x->w.wo + (size_t)l * d * d, d, d, att.data(), M, o.data());
+            for (int m = 0; m < M; ++m) {
+                for (int i = 0; i < d; ++i) y[(size_t)m * d + i] = (float)((double)h[(size_t)m * d + i] + o[(size_t)m * d + i]);  // R6
+                const double cs = orc_cosine(h.data() + (size_t)m * d, y.data() + (size_t)m * d, d);
+                x->last_cos_attn[(size_t)l * M + m] = (float)cs;
+                if (acc_sim) x->sumcos_attn[l] += cs;
+            }
+            h.swap(y);
+        }
+        // ------------------------------------------------ MLP sublayer
+        if (!(use_mask && x->skip_mlp[l])) {
+            rmsnorm_rows(x, h.data(), M, x->w.mlp_norm + (size_t)l * d, hn.data());
+            matvec_rows(x->w.wg + (size_t)l * f * d, f, d, hn.data(), M, g.data());
+            matvec_rows(x->w.wu + (size_t)l * f * d, f, d, hn.data(), M, u.data());
+            for (size_t i = 0; i < (size_t)M * f; ++i) {  // R7: silu(g) * u
+                const double gv = (double)(float)g[i], uv = (double)(float)u[i];
+                const float tv = (float)(gv / (1.0 + std::exp(-gv)) * uv);
+                t[i] = x->round ? round_bf16(tv) : tv;
+            }
+            matvec_rows(x->w.wd + (size_t)l * d * f, d, f, t.data(), M, o.data());
+            for (int m = 0; m < M; ++m) {
+                for (int i = 0; i < d; ++i) y[(size_t)m * d + i] = (float)((double)h[(size_t)m * d + i] + o[(size_t)m * d + i]);
+                const double cs = orc_cosine(h.data() + (size_t)m * d, y.data() + (size_t)m * d, d);
+                x->last_cos_mlp[(size_t)l * M + m] = (float)cs;
+                if (acc_sim) x->sumcos_mlp[l] += cs;
+            }
+            h.swap(y);
+        }
+    }
+    if (acc_sim) x->n_sim_rows += M;
+
+    // R8: final norm, LM head, argmax (lowest index among equal maxima)
+    rmsnorm_rows(x, h.data(), M, x->w.final_norm, hn.data());
+    std::vector<double> lg((size_t)M * V);
+    matvec_rows(x->w.lm_head, V, d, hn.data(), M, lg.data());
+    x->last_logits.resize((size_t)M * V);
+    x->last_argmax.resize(M);
+    x->last_margin.resize(M);
+    for (int m = 0; m < M; ++m) {
+        int best = 0;
+        float bestv = -INFINITY, second = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+            const float z = (float)lg[(size_t)m * V + v];
+            x->last_logits[(size_t)m * V + v] = z;
+            if (z > bestv) {
+                second = bestv;
+                bestv = z;
+                best = v;
+            } else if (z > second) {
+                second = z;
+            }
+        }
+        x->last_argmax[m] = best;
+        x->last_margin[m] = bestv - second;
+    }
+    return ORC_OK;
+}
+
+// Section 3.2: the whole input context goes through M, fills the KV cache, yields t_1 and the
+// per-layer similarity sums.  May be called repeatedly to feed the prompt in pieces.
+int orc_prefill(orc_ctx* x, const int32_t* tokens, int32_t n, int32_t* first_token) {
+    if (!x || !tokens || n <= 0) return ORC_ERR_ARG;
+    const double t0 = now_ms();
+    const int rc = forward_rows(x, tokens, n, x->n_committed, false, true);
+    if (rc) return rc;
+    x->n_committed += n;
+    x->draft_cursor = x->n_committed;
+    x->stats.prefill_rows += n;
+    x->stats.ms_prefill += now_ms() - t0;
+    if (first_token) *first_token = x->last_argmax[n - 1];
+    return ORC_OK;
+}
+
+// C_l = (1/S) sum_s cos(X_s^l, Y_s^l), for the attention and the MLP sublayers
+int orc_get_similarity(orc_ctx* x, float* c_attn, float* c_mlp, int32_t* n_rows) {
+    if (!x) return ORC_ERR_ARG;
+    if (n_rows) *n_rows = (int32_t)x->n_sim_rows;
+    if (x->n_sim_rows == 0) return ORC_ERR_STATE;
+    for (int l = 0; l < x->c.n_layers; ++l) {
+        if (c_attn) c_attn[l] = (float)(x->sumcos_attn[l] / (double)x->n_sim_rows);
+        if (c_mlp) c_mlp[l] = (float)(x->sumcos_mlp[l] / (double)x->n_sim_rows);
+    }
+    return ORC_OK;
+}
+
+int orc_set_skip_mask(orc_ctx* x, const uint8_t* skip_attn, const uint8_t* skip_mlp) {
+    if (!x || !skip_attn || !skip_mlp) return ORC_ERR_ARG;
+    for (int l = 0; l < x->c.n_layers; ++l) {
+        x->skip_attn[l] = skip_attn[l] ? 1 : 0;
+        x->skip_mlp[l] = skip_mlp[l] ? 1 : 0;
+    }
+    x->draft_cursor = x->n_committed;
+    return ORC_OK;
+}
+
+// Algorithm 1 on the attention similarities of the prompt; installs the result as the draft model's mask
+int orc_admg_update(orc_ctx* x, const orc_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp) {
+    if (!x || !p) return ORC_ERR_ARG;
+    std::vector<float> C(x->c.n_layers);
+    int rc = orc_get_similarity(x, C.data(), nullptr, nullptr);
+    if (rc) return rc;
+    std::vector<uint8_t> a(x->c.n_layers), b(x->c.n_layers);
+    rc = orc_admg(C.data(), x->c.n_layers, p->alpha, p->m, p->n, p->flags, a.data(), b.data());
+    if (rc) return rc;
+    orc_set_skip_mask(x, a.data(), b.data());
+    if (skip_attn) std::memcpy(skip_attn, a.data(), a.size());
+    if (skip_mlp) std::memcpy(skip_mlp, b.data(), b.size());
+    return ORC_OK;
+}
+
+// one autoregressive step of M: consumes token_in at the next position, commits it, returns the argmax
+int orc_decode_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
+    if (!x) return ORC_ERR_ARG;
+    const double t0 = now_ms();
+    const int rc = forward_rows(x, &token_in, 1, x->n_committed, false, false);
+    if (rc) return rc;
+    x->n_committed += 1;
+    x->draft_cursor = x->n_committed;
+    x->stats.full_passes += 1;
+    x->stats.ms_full += now_ms() - t0;
+    if (token_out) *token_out = x->last_argmax[0];
+    return ORC_OK;
+}
+
+// one step of the draft model D (M without the masked sublayers) at the draft cursor; commits nothing
+int orc_draft_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
+    if (!x) return ORC_ERR_ARG;
+    const double t0 = now_ms();
+    const int rc = forward_rows(x, &token_in, 1, x->draft_cursor, true, false);
+    if (rc) return rc;
+    x->draft_cursor += 1;
+    x->stats.draft_passes += 1;
+    x->stats.ms_draft += now_ms() - t0;
+    if (token_out) *token_out = x->last_argmax[0];
+    return ORC_OK;
+}
+
+// Section 1: M processes [t_last, d_1..d_k] in parallel at positions n..n+k; d_{j+1} is accepted while it
+// equals M's prediction g_j; the first rejected draft is replaced by M's token.  out_tokens receives the
+// accepted drafts followed by g_a (a+1 tokens); a+1 positions are committed.
+int orc_verify(orc_ctx* x, const int32_t* tokens, int32_t k, int32_t* n_accepted, int32_t* out_tokens) {
+    if (!x || !tokens || k < 0) return ORC_ERR_ARG;
+    const double t0 = now_ms();
+    const int rc = forward_rows(x, tokens, k + 1, x->n_committed, false, false);
+    if (rc) return rc;
+    int a = 0;
+    while (a < k && tokens[a + 1] == x->last_argmax[a]) ++a;
+    if (out_tokens) {
+        for (int j = 0; j < a; ++j) out_tokens[j] = tokens[j + 1];
+        out_tokens[a] = x->last_argmax[a];
+    }
+    if (n_accepted) *n_accepted = a;
+    x->n_committed += a + 1;
+    x->draft_cursor = x->n_committed;
+    x->stats.verify_passes += 1;
+    x->stats.drafted += k;
+    x->stats.accepted += a;
+    x->stats.ms_verify += now_ms() - t0;
+    return ORC_OK;
+}
+
+// Whole method: prefill -> t_1 -> (ADMG) -> repeat { k draft steps, verify } until max_new tokens.
+// out receives max_new tokens, out[0] = t_1.  margins (optional) receives, for each emitted token, the
+// top1-top2 logit gap of the full-model row that produced it.
+int orc_generate(orc_ctx* x, const int32_t* prompt, int32_t n_prompt, const orc_gen_params* gp, int32_t* out,
+                 int32_t* n_out, orc_stats* stats, float* margins) {
+    if (!x || !prompt || n_prompt <= 0 || !gp || !out || !n_out || gp->max_new <= 0 || gp->draft_len < 0)
+        return ORC_ERR_ARG;
+    std::vector<uint8_t> ka = x->skip_attn, km = x->skip_mlp;
+    orc_reset(x);
+    if (gp->mode == ORC_MODE_SPEC_MANUAL_MASK) orc_set_skip_mask(x, ka.data(), km.data());
+    const double t0 = now_ms();
+    int32_t last;
+    int rc = orc_prefill(x, prompt, n_prompt, &last);
+    if (rc) return rc;
+    int32_t produced = 0;
+    auto emit = [&](int32_t tok, float margin) {
+        if (produced < gp->max_new) {
+            if (margins) margins[produced] = margin;
+            out[produced++] = tok;
+        }
+    };
+    emit(last, x->last_margin[n_prompt - 1]);
+    bool stop = (gp->eos_id >= 0 && last == gp->eos_id);
+    if (gp->mode == ORC_MODE_SPEC) {
+        rc = orc_admg_update(x, &gp->admg, nullptr, nullptr);
+        if (rc) return rc;
+    }
+    std::vector<int32_t> row(gp->draft_len + 1), acc(gp->draft_len + 1);
+    while (produced < gp->max_new && !stop) {
+        if (gp->mode == ORC_MODE_AR) {
+            int32_t nxt;
+            rc = orc_decode_step(x, last, &nxt);
+            if (rc) return rc;
+            emit(nxt, x->last_margin[0]);
+            last = nxt;
+            stop = (gp->eos_id >= 0 && nxt == gp->eos_id);
+            continue;
+        }
+        int32_t k = std::min<int32_t>(gp->draft_len, gp->max_new - produced - 1);
+        k = std::min<int32_t>(k, x->c.max_seq - x->n_committed - 1);
+        if (k < 0) return ORC_ERR_OVERFLOW;
+        row[0] = last;
+        for (int j = 0; j < k; ++j) {
+            rc = orc_draft_step(x, row[j], &row[j + 1]);
+            if (rc) return rc;
+        }
+        int32_t a = 0;
+        rc = orc_verify(x, row.data(), k, &a, acc.data());
+        if (rc) return rc;
+        x->stats.rounds += 1;
+        for (int j = 0; j <= a && !stop; ++j) {
+            emit(acc[j], x->last_margin[j]);
+            stop = (gp->eos_id >= 0 && acc[j] == gp->eos_id);
+        }
+        last = acc[a];
+    }
+    *n_out = produced;
+    x->stats.ms_total = now_ms() - t0;
+    if (stats) *stats = x->stats;
+    return ORC_OK;
+}
+
+int orc_get_stats(orc_ctx* x, orc_stats* s) {
+    if (!x || !s) return ORC_ERR_ARG;
+    *s = x->stats;
+    return ORC_OK;
+}
+
+int orc_get_positions(orc_ctx* x, int32_t* n_committed, int32_t* draft_cursor) {
+    if (!x) return ORC_ERR_ARG;
+    if (n_committed) *n_committed = x->n_committed;
+    if (draft_cursor) *draft_cursor = x->draft_cursor;
+    return ORC_OK;
+}
+
+// per-row results of the last pass.  cos arrays are [L][M], NaN where the sublayer was skipped.
+int orc_get_last(orc_ctx* x, int32_t* M, float* logits, float* cos_attn, float* cos_mlp, int32_t* argmax, float* margin) {
+    if (!x || x->last_M == 0) return ORC_ERR_STATE;
+    const int m = x->last_M;
+    if (M) *M = m;
+    if (logits) std::memcpy(logits, x->last_logits.data(), sizeof(float) * (size_t)m * x->c.vocab);
+    if (cos_attn) std::memcpy(cos_attn, x->last_cos_attn.data(), sizeof(float) * (size_t)m * x->c.n_layers);
+    if (cos_mlp) std::memcpy(cos_mlp, x->last_cos_mlp.data(), sizeof(float) * (size_t)m * x->c.n_layers);
+    if (argmax) std::memcpy(argmax, x->last_argmax.data(), sizeof(int32_t) * m);
+    if (margin) std::memcpy(margin, x->last_margin.data(), sizeof(float) * m);
+    return ORC_OK;
+}
+
+// K and V rows of one layer at one position, as floats (tests of the cache logic)
+int orc_get_kv(orc_ctx* x, int32_t layer, int32_t pos, float* k, float* v) {
+    if (!x || layer < 0 || layer >= x->c.n_layers || pos < 0 || pos >= x->c.max_seq) return ORC_ERR_ARG;
+    const size_t off = ((size_t)layer * x->c.max_seq + pos) * x->kv_dim;
+    if (k) std::memcpy(k, x->kcache.data() + off, sizeof(float) * x->kv_dim);
+    if (v) std::memcpy(v, x->vcache.data() + off, sizeof(float) * x->kv_dim);
+    return ORC_OK;
+}
+
+// ---------------------------------------------------------------- single fused sublayer product
+// The building block of every sublayer, for kernel-level comparisons:
+//   xin = has_norm ? bf16(RMSNorm(x; gain, eps)) : x          x: [M, n_in] float
+//   a   = W  xin                                              W: [n_out, n_in] bf16
+//   epilogue 0 (plain)    : out[M, n_out] = float(a)
+//   epilogue 1 (SwiGLU)   : b = W2 xin;  out = bf16(silu(float(a)) * float(b))
+//   epilogue 2 (residual) : out = float(res + a);  cos[m] = cosine(res[m], out[m])
+int orc_fused_matvec(const float* x, int32_t M, int32_t n_in, const uint16_t* gain, float eps, const uint16_t* W,
+                     const uint16_t* W2, int32_t n_out, int32_t epilogue, const float* res, float* out, float* cosv) {
+    if (!x || !W || !out || M <= 0 || n_in <= 0 || n_out <= 0) return ORC_ERR_ARG;
+    std::vector<float> xin((size_t)M * n_in);
+    if (gain) {
+        for (int m = 0; m < M; ++m) {
+            double ss = 0;
+            for (int i = 0; i < n_in; ++i) ss += (double)x[(size_t)m * n_in + i] * (double)x[(size_t)m * n_in + i];
+            const double inv = 1.0 / std::sqrt(ss / n_in + (double)eps);
+            for (int i = 0; i < n_in; ++i)
+                xin[(size_t)m * n_in + i] =
+                    round_bf16((float)((double)x[(size_t)m * n_in + i] * inv * (double)bf16_bits_to_float(gain[i])));
+        }
+    } else {
+        std::memcpy(xin.data(), x, sizeof(float) * xin.size());
+    }
+    std::vector<double> a((size_t)M * n_out), b;
+    matvec_rows(W, n_out, n_in, xin.data(), M, a.data());
+    if (epilogue == 0) {
+        for (size_t i = 0; i < a.size(); ++i) out[i] = (float)a[i];
+    } else if (epilogue == 1) {
+        if (!W2) return ORC_ERR_ARG;
+        b.resize(a.size());
+        matvec_rows(W2, n_out, n_in, xin.data(), M, b.data());
+        for (size_t i = 0; i < a.size(); ++i) {
+            const double gv = (double)(float)a[i], uv = (double)(float)b[i];
+            out[i] = round_bf16((float)(gv / (1.0 + std::exp(-gv)) * uv));
+        }
+    } else if (epilogue == 2) {
+        if (!res) return ORC_ERR_ARG;
+        for (int m = 0; m < M; ++m) {
+            for (int i = 0; i < n_out; ++i) out[(size_t)m * n_out + i] = (float)((double)res[(size_t)m * n_out + i] + a[(size_t)m * n_out + i]);
+            if (cosv) cosv[m] = (float)orc_cosine(res + (size_t)m * n_out, out + (size_t)m * n_out, n_out);
+        }
+    } else {
+        return ORC_ERR_ARG;
+    }
+    return ORC_OK;
+}
+
+int orc_num_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}
+
+}  // extern "C"

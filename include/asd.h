@@ -1,0 +1,198 @@
+/*
+ * libasd -- adaptive self-speculative decoding (arXiv 2410.01028) on one NVIDIA B200 (sm_100a).
+ *
+ * The library runs single-sequence, memory-bound decoding of a Llama-style dense decoder M in which
+ *   - every attention and MLP sublayer of a full-model pass also yields the cosine similarity between the
+ *     hidden state entering and leaving it (Section 3.1; the summand of C_l in Section 3.2), computed in the
+ *     epilogue of the residual add;
+ *   - the Adaptive Draft Model Generator (Algorithm 1; rules 1 and 2 of Section 3.2) turns the similarities
+ *     averaged over the prompt into a per-context skip mask that defines the draft model D, a sub-network of M;
+ *   - k drafted tokens are verified by one (k+1)-row pass of M, the matching prefix is accepted and the first
+ *     rejected token is replaced by M's (Section 1), so the output equals greedy autoregressive decoding.
+ *
+ * Conventions
+ *   - C ABI. Every call returns an int: ASD_OK (0) or a negative asd_status. No call throws or aborts;
+ *     asd_last_error() returns a description of the last failure of that context (static storage duration
+ *     per context; valid until the next failing call).
+ *   - Pointers are HOST pointers unless the parameter is documented as DEVICE. Host arrays are borrowed for
+ *     the duration of the call only. Calls are synchronous with respect to their host outputs.
+ *   - The context owns no device memory: all of it is carved out of one caller-provided DEVICE workspace of
+ *     asd_workspace_bytes() bytes (256-byte aligned), which must outlive the context. Work is enqueued on
+ *     the caller-provided CUDA stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - One context holds one sequence (batch size 1, as in Section 3.2). Contexts are not thread safe.
+ *   - Layers are numbered l = 1..L in the paper; arrays indexed by layer use index l-1.
+ *   - Matrices are bf16, row-major [out, in] (y = W x); accumulation is fp32; the residual stream is fp32.
+ */
+#ifndef ASD_H_
+#define ASD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ASD_OK = 0,
+    ASD_ERR_ARG = -1,            /* null pointer, out-of-range value, unsupported shape */
+    ASD_ERR_STATE = -2,          /* call not valid in the current state (no weights, nothing prefetched, ...) */
+    ASD_ERR_NOMEM = -3,          /* workspace too small or misaligned */
+    ASD_ERR_OVERFLOW = -4,       /* the call would write past max_seq positions */
+    ASD_ERR_CUDA = -5,           /* a CUDA runtime call failed; see asd_last_error() */
+    ASD_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired */
+    ASD_ERR_IO = -7              /* weight file missing, short or malformed */
+} asd_status;
+
+/* Shape of the decoder. Requirements: n_heads * head_dim == d_model; n_heads % n_kv_heads == 0;
+ * head_dim % 8 == 0 and head_dim <= 256; d_model % 8 == 0; d_ffn % 8 == 0; 0 <= max_draft <= 8. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t max_seq;   /* capacity of the KV cache in positions */
+    int32_t max_draft; /* largest draft length k accepted by asd_verify / asd_generate */
+    float rms_eps;     /* epsilon under the root of RMSNorm */
+    float rope_theta;  /* base of the rotary embedding */
+} asd_config;
+
+/* bf16 weights on the HOST, as raw 16-bit patterns, row-major [out, in], stacked over layers. */
+typedef struct {
+    const uint16_t* embed;      /* [vocab, d_model]                 */
+    const uint16_t* lm_head;    /* [vocab, d_model] (untied)        */
+    const uint16_t* final_norm; /* [d_model]                        */
+    const uint16_t* attn_norm;  /* [L, d_model]                     */
+    const uint16_t* wq;         /* [L, d_model, d_model]            */
+    const uint16_t* wk;         /* [L, n_kv_heads*head_dim, d_model]*/
+    const uint16_t* wv;         /* [L, n_kv_heads*head_dim, d_model]*/
+    const uint16_t* wo;         /* [L, d_model, d_model]            */
+    const uint16_t* mlp_norm;   /* [L, d_model]                     */
+    const uint16_t* wg;         /* [L, d_ffn, d_model]  gate        */
+    const uint16_t* wu;         /* [L, d_ffn, d_model]  up          */
+    const uint16_t* wd;         /* [L, d_model, d_ffn]  down        */
+} asd_host_weights;
+
+/* Hyper-parameters of Algorithm 1. flags select the rule subsets of Table 5. */
+#define ASD_USE_CS 1u    /* cosine-similarity thresholding: remove attention layer l if C_l >= alpha */
+#define ASD_USE_RULE1 2u /* remove every m-th attention and MLP layer */
+#define ASD_USE_RULE2 4u /* never remove the last n layers */
+#define ASD_ADMG_ALL 7u
+typedef struct {
+    float alpha;
+    int32_t m, n;
+    uint32_t flags;
+} asd_admg_params;
+
+#define ASD_MODE_AR 0               /* plain greedy decoding with M */
+#define ASD_MODE_SPEC 1             /* self-speculative; mask from Algorithm 1 on the prompt's similarities */
+#define ASD_MODE_SPEC_MANUAL_MASK 2 /* self-speculative with the mask installed by asd_set_skip_mask */
+typedef struct {
+    int32_t mode, draft_len, max_new;
+    int32_t eos_id; /* -1 = none */
+    asd_admg_params admg;
+} asd_gen_params;
+
+/* Counters and device times (CUDA events) accumulated since the last asd_reset / asd_generate start.
+ * bytes_* are the algorithmic bytes of the passes: weights actually streamed plus K/V read. */
+typedef struct {
+    int64_t full_passes, draft_passes, verify_passes, rounds, drafted, accepted, prefill_rows;
+    double ms_prefill, ms_full, ms_draft, ms_verify, ms_total;
+    double bytes_full, bytes_draft, bytes_verify;
+    int64_t kernel_launches;
+} asd_stats;
+
+typedef struct asd_ctx asd_ctx;
+
+/* Size of the device workspace a context of this shape needs (weights + KV cache + scratch); 0 on a bad config. */
+size_t asd_workspace_bytes(const asd_config* cfg);
+
+/* Create a context inside dev_workspace (DEVICE, 256-byte aligned, >= asd_workspace_bytes(cfg)).
+ * The workspace's KV region is zeroed. cuda_stream is a cudaStream_t. Errors: ARG, NOMEM, CUDA. */
+int asd_create(const asd_config* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, asd_ctx** out);
+int asd_destroy(asd_ctx* ctx);
+const char* asd_last_error(asd_ctx* ctx);
+
+/* Copy the weights into the workspace (gate and up rows are interleaved on the way). Blocking. */
+int asd_load_weights_host(asd_ctx* ctx, const asd_host_weights* w);
+/* Same tensors from a flat little-endian file: the twelve arrays of asd_host_weights in declaration order,
+ * without header or padding. Errors: IO when the file is missing or short. */
+int asd_load_weights_file(asd_ctx* ctx, const char* path);
+
+/* New context: nothing cached, similarity sums cleared, empty skip mask, statistics cleared. */
+int asd_reset(asd_ctx* ctx);
+
+/* Section 3.2, first step of inference: pass n prompt tokens through M, fill the KV cache, add each row's
+ * per-sublayer cosine to the running sums behind C_l, return M's first token. May be called again to append
+ * more prompt. Errors: ARG (n <= 0, token out of range), OVERFLOW, STATE (no weights). */
+int asd_prefill(asd_ctx* ctx, const int32_t* tokens, int32_t n, int32_t* first_token);
+/* As asd_prefill with the tokens in DEVICE memory (inputs already resident). */
+int asd_prefill_device(asd_ctx* ctx, const int32_t* dev_tokens, int32_t n, int32_t* first_token);
+
+/* C_l of Section 3.2 for the attention sublayers (c_attn[L]) and, as in Table 1, the MLP sublayers
+ * (c_mlp[L]); n_rows = number of prompt rows averaged. Any output may be NULL. STATE if no row yet. */
+int asd_get_similarity(asd_ctx* ctx, float* c_attn, float* c_mlp, int32_t* n_rows);
+
+/* Algorithm 1 on the current C: computes remove_ATTN / remove_MLP, installs them as the draft model's skip
+ * mask and optionally returns them (uint8[L], 1 = removed). Resets the draft cursor. */
+int asd_admg_update(asd_ctx* ctx, const asd_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp);
+/* Install a mask by hand (uint8[L] each, non-zero = skip). Resets the draft cursor. */
+int asd_set_skip_mask(asd_ctx* ctx, const uint8_t* skip_attn, const uint8_t* skip_mlp);
+
+/* One autoregressive step of M: consumes token_in at the next position, commits it, returns the argmax. */
+int asd_decode_step(asd_ctx* ctx, int32_t token_in, int32_t* token_out);
+/* One step of the draft model D at the draft cursor: sublayers in the mask are the identity, stream no
+ * weights and touch no K/V. Commits nothing; advances the draft cursor. */
+int asd_draft_step(asd_ctx* ctx, int32_t token_in, int32_t* token_out);
+/* Section 1: M processes tokens[0..k] = [t_last, d_1..d_k] at the next k+1 positions in one pass, rewriting
+ * K/V there in every layer. d_{j+1} is accepted while it equals M's argmax g_j; out_tokens receives the
+ * accepted drafts followed by g_a (a+1 tokens, a = *n_accepted); a+1 positions are committed and the draft
+ * cursor returns to the committed length. 0 <= k <= max_draft. */
+int asd_verify(asd_ctx* ctx, const int32_t* tokens, int32_t k, int32_t* n_accepted, int32_t* out_tokens);
+
+/* The whole method: reset, prefill, t_1, (Algorithm 1), then rounds of draft_len draft steps and one verify
+ * until max_new tokens (out[0] = t_1) or eos. out has room for max_new tokens. stats may be NULL. */
+int asd_generate(asd_ctx* ctx, const int32_t* prompt, int32_t n_prompt, const asd_gen_params* p, int32_t* out,
+                 int32_t* n_out, asd_stats* stats);
+/* As asd_generate with the prompt and the output array in DEVICE memory; n_out stays a host pointer. */
+int asd_generate_device(asd_ctx* ctx, const int32_t* dev_prompt, int32_t n_prompt, const asd_gen_params* p,
+                        int32_t* dev_out, int32_t* n_out, asd_stats* stats);
+
+/* Per-row results of the last pass of M rows: cosines [L][M] (NaN where the sublayer was skipped),
+ * argmax [M]. *M receives the row count. Any output may be NULL. */
+int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_mlp);
+/* Logits [M][vocab] of the last pass; only recorded while asd_set_debug(ctx, 1) is in effect. */
+int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
+int asd_set_debug(asd_ctx* ctx, int32_t record_logits);
+/* K and V rows (bf16 patterns, n_kv_heads*head_dim each) of one layer (0-based) at one position. */
+int asd_get_kv(asd_ctx* ctx, int32_t layer, int32_t pos, uint16_t* k, uint16_t* v);
+int asd_get_positions(asd_ctx* ctx, int32_t* n_committed, int32_t* draft_cursor);
+int asd_get_stats(asd_ctx* ctx, asd_stats* stats);
+
+/* ------------------------------------------------------------------------------------------------------
+ * The sublayer building block on its own (kernel-level tests and micro-benchmarks): one fused
+ *   xin = gain ? bf16(RMSNorm(x; gain, eps)) : x ;  a = W xin ;  epilogue
+ * for M <= 9 rows. All pointers are DEVICE pointers.
+ *   x        : gain != NULL -> float [M, n_in] ; gain == NULL -> bf16 [M, n_in]
+ *   W        : bf16 [n_rows, n_in]; n_in % 8 == 0
+ *   epilogue : ASD_EPI_PLAIN    out = float [M, n_rows]
+ *              ASD_EPI_SWIGLU   rows of W alternate gate_i, up_i (n_rows even);
+ *                               out = bf16 [M, n_rows/2] = silu(gate) * up
+ *              ASD_EPI_RESIDUAL out = float [M, n_rows], updated IN PLACE: out += a (the residual add), and
+ *                               cos[m] = cosine(out before, out after)  -- the summand of C_l, Section 3.2
+ *   scratch  : >= asd_fused_gemv_scratch_bytes() bytes, 256-byte aligned; its first 256 bytes must be zero
+ *              before the first use and are left zero by every call.
+ * Errors: ARG, NOMEM (scratch too small), CUDA. Asynchronous on the stream.
+ */
+#define ASD_EPI_PLAIN 0
+#define ASD_EPI_SWIGLU 1
+#define ASD_EPI_RESIDUAL 2
+size_t asd_fused_gemv_scratch_bytes(void);
+int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, const void* x, const uint16_t* gain,
+                   float eps, const uint16_t* W, int32_t epilogue, void* out, float* cos, void* scratch,
+                   size_t scratch_bytes);
+
+/* Algorithm 1 as a pure host function (no context): C[L] -> remove_attn[L], remove_mlp[L]. */
+int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASD_H_ */

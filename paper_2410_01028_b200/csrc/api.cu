@@ -1,0 +1,929 @@
+// Host side of libasd: workspace layout, pass scheduling under the skip mask, Algorithm 1, the decode loops
+// and the C ABI declared in include/asd.h.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <string>
+#include <vector>
+
+#include "../../include/asd.h"
+#include "common.cuh"
+
+namespace asd {
+
+constexpr int kPrefillRows = 8;  // prompt rows per pass of the chunked prefill
+constexpr size_t kAlign = 256;
+constexpr int kMaxGemvGrid = 1024;
+
+static size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+// ---------------------------------------------------------------- shared-memory budgets
+size_t gemv_smem_bytes(int M, int n_rows, int n_in, int grid, bool x_in_smem) {
+    const size_t n_pairs = ((size_t)n_rows + 1) / 2;
+    const size_t max_np = (n_pairs + grid - 1) / grid;
+    const size_t n_seg = ((size_t)n_in + kSeg - 1) / kSeg;
+    size_t psum = (max_np * n_seg * 2 * M + 3) & ~(size_t)3;
+    size_t b = (size_t)kGemvWarps * kMaxRows * 4 * 4 + 16 + psum * 4;
+    if (x_in_smem) b += (size_t)M * n_in * 2;
+    return b;
+}
+size_t attn_smem_bytes(int M, int head_dim) {
+    return (size_t)kAttnChunk * (head_dim + 8) * 2 + (size_t)kAttnChunk * head_dim * 2 + (size_t)M * head_dim * 4 +
+           (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16;
+}
+
+static cudaError_t launch_gemv(int M, int epi, bool norm, const GemvParams& p, int grid, size_t smem, cudaStream_t s) {
+    switch (M) {
+        case 1: return launch_gemv_m1(epi, norm, p, grid, smem, s);
+        case 2: return launch_gemv_m2(epi, norm, p, grid, smem, s);
+        case 3: return launch_gemv_m3(epi, norm, p, grid, smem, s);
+        case 4: return launch_gemv_m4(epi, norm, p, grid, smem, s);
+        case 5: return launch_gemv_m5(epi, norm, p, grid, smem, s);
+        case 6: return launch_gemv_m6(epi, norm, p, grid, smem, s);
+        case 7: return launch_gemv_m7(epi, norm, p, grid, smem, s);
+        case 8: return launch_gemv_m8(epi, norm, p, grid, smem, s);
+        case 9: return launch_gemv_m9(epi, norm, p, grid, smem, s);
+    }
+    return cudaErrorInvalidValue;
+}
+static cudaError_t launch_attn(int M, const AttnParams& p, size_t smem, cudaStream_t s) {
+    switch (M) {
+        case 1: return launch_attn_m1(p, smem, s);
+        case 2: return launch_attn_m2(p, smem, s);
+        case 3: return launch_attn_m3(p, smem, s);
+        case 4: return launch_attn_m4(p, smem, s);
+        case 5: return launch_attn_m5(p, smem, s);
+        case 6: return launch_attn_m6(p, smem, s);
+        case 7: return launch_attn_m7(p, smem, s);
+        case 8: return launch_attn_m8(p, smem, s);
+        case 9: return launch_attn_m9(p, smem, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// per-device facts and one-time kernel configuration
+struct DeviceInfo {
+    bool ready = false;
+    int num_sms = 0, max_smem = 0;
+};
+static DeviceInfo g_dev[64];
+
+static cudaError_t device_info(DeviceInfo** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    DeviceInfo& d = g_dev[dev];
+    if (!d.ready) {
+        if ((e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&d.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+        if ((e = configure_m1(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m2(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m3(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m4(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m5(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m6(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m7(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m8(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m9(d.max_smem)) != cudaSuccess) return e;
+        d.ready = true;
+    }
+    *out = &d;
+    return cudaSuccess;
+}
+
+// Choose the launch shape of one fused GEMV: one CTA per SM; more CTAs only when the per-CTA partial-sum
+// buffer would not fit in shared memory; activations fall back to L1 reads when they do not fit.
+static bool plan_gemv(const DeviceInfo& dv, int M, int n_rows, int n_in, bool norm, int* grid, int* x_in_smem, size_t* smem) {
+    for (int g = dv.num_sms; g <= kMaxGemvGrid; g += dv.num_sms) {
+        size_t b = gemv_smem_bytes(M, n_rows, n_in, g, true);
+        if (b <= (size_t)dv.max_smem) {
+            *grid = g, *x_in_smem = 1, *smem = b;
+            return true;
+        }
+        if (!norm) {
+            b = gemv_smem_bytes(M, n_rows, n_in, g, false);
+            if (b <= (size_t)dv.max_smem) {
+                *grid = g, *x_in_smem = 0, *smem = b;
+                return true;
+            }
+        }
+    }
+    return false;
+}
+
+__global__ void embed_kernel(const int* tokens, const __nv_bfloat16* E, float* x, int d, int vocab) {
+    const int m = blockIdx.x;
+    int t = tokens[m];
+    t = min(max(t, 0), vocab - 1);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)m * d + i] = __bfloat162float(E[(size_t)t * d + i]);
+}
+
+// ---------------------------------------------------------------- workspace layout
+struct Layout {
+    size_t embed, lm_head, final_norm, layers, layer_stride;
+    size_t l_attn_norm, l_wqkv, l_wo, l_mlp_norm, l_wgu, l_wd;  // offsets inside one layer block
+    size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
+    size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
+    size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits;
+    size_t total;
+    int chunk_stride;
+};
+
+static bool check_config(const asd_config& c) {
+    if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.d_ffn <= 0 ||
+        c.vocab <= 0 || c.max_seq <= 0)
+        return false;
+    if ((long long)c.n_heads * c.head_dim != c.d_model || c.n_heads % c.n_kv_heads) return false;
+    if (c.head_dim % 8 || c.head_dim > 256 || c.d_model % 8 || c.d_ffn % 8) return false;
+    if (c.max_draft < 0 || c.max_draft > kMaxRows - 1) return false;
+    if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return false;
+    return true;
+}
+
+static Layout make_layout(const asd_config& c) {
+    Layout L{};
+    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = (size_t)c.n_kv_heads * c.head_dim, S = c.max_seq;
+    size_t o = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = o;
+        o = align_up(o + bytes);
+        return at;
+    };
+    L.embed = take(V * d * 2);
+    L.lm_head = take(V * d * 2);
+    L.final_norm = take(d * 2);
+    {
+        size_t lo = 0;
+        auto ltake = [&](size_t bytes) {
+            size_t at = lo;
+            lo = align_up(lo + bytes);
+            return at;
+        };
+        L.l_attn_norm = ltake(d * 2);
+        L.l_wqkv = ltake((d + 2 * kvd) * d * 2);
+        L.l_wo = ltake(d * d * 2);
+        L.l_mlp_norm = ltake(d * 2);
+        L.l_wgu = ltake(2 * f * d * 2);
+        L.l_wd = ltake(d * f * 2);
+        L.layer_stride = lo;
+    }
+    L.layers = take(L.layer_stride * c.n_layers);
+    L.rope_cos = take(S * (c.head_dim / 2) * 4);
+    L.rope_sin = take(S * (c.head_dim / 2) * 4);
+    L.kv_layer_stride = align_up(S * kvd * 2);
+    L.kcache = take(L.kv_layer_stride * c.n_layers);
+    L.vcache = take(L.kv_layer_stride * c.n_layers);
+    L.x = take(kMaxRows * d * 4);
+    L.q = take(kMaxRows * d * 2);
+    L.a = take(kMaxRows * d * 2);
+    L.t = take(kMaxRows * f * 2);
+    L.chunk_stride = (int)((S + kAttnChunk - 1) / kAttnChunk);
+    L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * c.head_dim * 4);
+    L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * 2 * 4);
+    L.partials = take((size_t)kMaxGemvGrid * kMaxRows * 4 * 4);
+    L.counters = take((size_t)(c.n_kv_heads + 64) * 4);
+    L.cosv = take((size_t)2 * std::max(c.n_layers, 1) * kMaxRows * 4);
+    L.sumcos = take((size_t)2 * std::max(c.n_layers, 1) * 8);
+    L.tok_in = take(64 * 4);
+    L.draft_toks = take(64 * 4);
+    L.gen_toks = take((S + 16) * 4);
+    L.prompt_toks = take((S + 16) * 4);
+    L.argmax = take(64 * 4);
+    L.accept = take(64 * 4);
+    L.logits = take((size_t)kMaxRows * V * 4);
+    L.total = o;
+    return L;
+}
+
+}  // namespace asd
+
+using namespace asd;
+
+// ---------------------------------------------------------------- context
+struct asd_ctx {
+    asd_config c;
+    Layout lay;
+    unsigned char* ws = nullptr;
+    cudaStream_t stream = nullptr;
+    DeviceInfo* dev = nullptr;
+    int kv_dim = 0;
+    bool have_weights = false;
+    int n_committed = 0, draft_cursor = 0;
+    std::vector<uint8_t> skip_attn, skip_mlp;
+    int64_t n_sim_rows = 0;
+    int last_M = 0;
+    bool debug_logits = false, last_has_logits = false;
+    asd_stats stats{};
+    int32_t* pinned = nullptr;  // small host staging buffer
+    std::vector<cudaEvent_t> events;
+    size_t events_used = 0;
+    struct Span { int kind; size_t e0, e1; };
+    std::vector<Span> spans;
+    std::string err;
+
+    template <class T>
+    T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+    unsigned char* layer(int l) const { return ws + lay.layers + (size_t)l * lay.layer_stride; }
+};
+
+enum { SPAN_PREFILL, SPAN_FULL, SPAN_DRAFT, SPAN_VERIFY };
+
+static int fail(asd_ctx* x, int code, const std::string& what) {
+    if (x) x->err = what;
+    return code;
+}
+#define ASD_CUDA(x, expr)                                                                             \
+    do {                                                                                              \
+        cudaError_t e__ = (expr);                                                                     \
+        if (e__ != cudaSuccess)                                                                       \
+            return fail((x), ASD_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__));      \
+    } while (0)
+
+static int new_event(asd_ctx* x, size_t* idx) {
+    if (x->events_used == x->events.size()) {
+        cudaEvent_t e;
+        ASD_CUDA(x, cudaEventCreate(&e));
+        x->events.push_back(e);
+    }
+    *idx = x->events_used++;
+    ASD_CUDA(x, cudaEventRecord(x->events[*idx], x->stream));
+    return ASD_OK;
+}
+
+// turn the recorded spans into statistics; requires the stream to be idle
+static int resolve_spans(asd_ctx* x) {
+    for (const auto& s : x->spans) {
+        float ms = 0.f;
+        ASD_CUDA(x, cudaEventElapsedTime(&ms, x->events[s.e0], x->events[s.e1]));
+        switch (s.kind) {
+            case SPAN_PREFILL: x->stats.ms_prefill += ms; break;
+            case SPAN_FULL: x->stats.ms_full += ms; break;
+            case SPAN_DRAFT: x->stats.ms_draft += ms; break;
+            case SPAN_VERIFY: x->stats.ms_verify += ms; break;
+        }
+    }
+    x->spans.clear();
+    x->events_used = 0;
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- one pass of M rows through the decoder
+// tokens (DEVICE) feed rows at positions pos0..pos0+M-1. use_mask selects the draft model D: sublayers in the
+// skip sets are the identity and launch nothing. acc_sim adds the rows' cosines to the prompt sums behind C_l.
+static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use_mask, bool acc_sim, bool lm_head,
+                    int* dev_argmax_out, bool accept, double* bytes_out) {
+    const asd_config& c = x->c;
+    const Layout& ly = x->lay;
+    const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
+    cudaStream_t s = x->stream;
+    if (M < 1 || M > kMaxRows) return fail(x, ASD_ERR_ARG, "row count out of range");
+    if ((long long)pos0 + M > c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "pass would exceed max_seq positions");
+    double bytes = 0;
+
+    float* cosv = x->at<float>(ly.cosv);
+    ASD_CUDA(x, cudaMemsetAsync(cosv, 0xFF, (size_t)2 * std::max(L, 1) * kMaxRows * 4, s));  // NaN = skipped
+    embed_kernel<<<M, 256, 0, s>>>(dev_tokens, x->at<__nv_bfloat16>(ly.embed), x->at<float>(ly.x), d, c.vocab);
+    ASD_CUDA(x, cudaGetLastError());
+    x->stats.kernel_launches += 1;
+
+    GemvParams base{};
+    base.eps = c.rms_eps;
+    base.partials = x->at<float>(ly.partials);
+    base.counter = x->at<unsigned>(ly.counters);  // slot 0; attention uses slots 64..
+    base.pos0 = pos0;
+    base.d_model = d;
+    base.kv_dim = kvd;
+    base.head_dim = c.head_dim;
+    base.rope_cos = x->at<float>(ly.rope_cos);
+    base.rope_sin = x->at<float>(ly.rope_sin);
+
+    auto gemv = [&](int epi, bool norm, GemvParams& p) -> int {
+        int grid, xin;
+        size_t smem;
+        if (!plan_gemv(*x->dev, M, p.n_rows, p.n_in, norm, &grid, &xin, &smem))
+            return fail(x, ASD_ERR_ARG, "matrix shape does not fit the kernel's shared-memory plan");
+        p.x_in_smem = xin;
+        ASD_CUDA(x, launch_gemv(M, epi, norm, p, grid, smem, s));
+        x->stats.kernel_launches += 1;
+        return ASD_OK;
+    };
+
+    for (int l = 0; l < L; ++l) {
+        unsigned char* lw = x->layer(l);
+        if (!(use_mask && x->skip_attn[l])) {
+            GemvParams p = base;
+            p.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wqkv);
+            p.n_rows = d + 2 * kvd;
+            p.n_in = d;
+            p.x = x->at<float>(ly.x);
+            p.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_attn_norm);
+            p.q_out = x->at<__nv_bfloat16>(ly.q);
+            p.k_cache = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.kcache + (size_t)l * ly.kv_layer_stride);
+            p.v_cache = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.vcache + (size_t)l * ly.kv_layer_stride);
+            int rc = gemv(kEpiQkv, true, p);
+            if (rc) return rc;
+
+            AttnParams ap{};
+            ap.q = p.q_out;
+            ap.k_cache = p.k_cache;
+            ap.v_cache = p.v_cache;
+            ap.pos0 = pos0;
+            ap.n_heads = c.n_heads;
+            ap.n_kv_heads = c.n_kv_heads;
+            ap.head_dim = c.head_dim;
+            ap.kv_dim = kvd;
+            ap.d_model = d;
+            ap.scale = 1.0f / sqrtf((float)c.head_dim);
+            ap.part_acc = x->at<float>(ly.part_acc);
+            ap.part_ml = x->at<float>(ly.part_ml);
+            ap.counters = x->at<unsigned>(ly.counters) + 64;
+            ap.a_out = x->at<__nv_bfloat16>(ly.a);
+            ap.n_chunks = (pos0 + M - 1) / kAttnChunk + 1;
+            ap.chunk_stride = ly.chunk_stride;
+            ASD_CUDA(x, launch_attn(M, ap, attn_smem_bytes(M, c.head_dim), s));
+            x->stats.kernel_launches += 1;
+
+            GemvParams o = base;
+            o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wo);
+            o.n_rows = d;
+            o.n_in = d;
+            o.x = x->at<__nv_bfloat16>(ly.a);
+            o.out = x->at<float>(ly.x);
+            o.cos_out = cosv + (size_t)(0 * L + l) * kMaxRows;
+            o.sumcos = acc_sim ? x->at<double>(ly.sumcos) + l : nullptr;
+            rc = gemv(kEpiResidual, false, o);
+            if (rc) return rc;
+            bytes += 2.0 * ((double)(d + 2 * kvd) * d + (double)d * d) + 2.0 * 2.0 * kvd * (double)(pos0 + M);
+        }
+        if (!(use_mask && x->skip_mlp[l])) {
+            GemvParams p = base;
+            p.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wgu);
+            p.n_rows = 2 * f;
+            p.n_in = d;
+            p.x = x->at<float>(ly.x);
+            p.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_mlp_norm);
+            p.out = x->at<__nv_bfloat16>(ly.t);
+            int rc = gemv(kEpiSwiglu, true, p);
+            if (rc) return rc;
+            GemvParams o = base;
+            o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wd);
+            o.n_rows = d;
+            o.n_in = f;
+            o.x = x->at<__nv_bfloat16>(ly.t);
+            o.out = x->at<float>(ly.x);
+            o.cos_out = cosv + (size_t)(1 * L + l) * kMaxRows;
+            o.sumcos = acc_sim ? x->at<double>(ly.sumcos) + L + l : nullptr;
+            rc = gemv(kEpiResidual, false, o);
+            if (rc) return rc;
+            bytes += 2.0 * 3.0 * (double)d * f;
+        }
+    }
+    x->last_has_logits = false;
+    if (lm_head) {
+        GemvParams p = base;
+        p.W = x->at<__nv_bfloat16>(ly.lm_head);
+        p.n_rows = c.vocab;
+        p.n_in = d;
+        p.x = x->at<float>(ly.x);
+        p.gain = x->at<__nv_bfloat16>(ly.final_norm);
+        p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
+        p.row_tokens = accept ? dev_tokens : nullptr;
+        p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
+        p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
+        int rc = gemv(kEpiArgmax, true, p);
+        if (rc) return rc;
+        x->last_has_logits = x->debug_logits;
+        bytes += 2.0 * (double)c.vocab * d;
+    }
+    x->last_M = M;
+    if (bytes_out) *bytes_out = bytes;
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- Algorithm 1
+// remove_MLP = { l : l = j*m, j >= 1, l <= L-n };  remove_ATTN = { l : C_l >= alpha, l <= L-n } U remove_MLP,
+// layers numbered from 1. flags drop individual rules (Table 5).
+extern "C" int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp) {
+    if (!C || !p || !remove_attn || !remove_mlp || L < 0 || p->m < 0 || p->n < 0) return ASD_ERR_ARG;
+    const bool cs = p->flags & ASD_USE_CS, r1 = (p->flags & ASD_USE_RULE1) && p->m >= 1, r2 = p->flags & ASD_USE_RULE2;
+    const int32_t last_removable = L - (r2 ? p->n : 0);
+    for (int32_t i = 0; i < L; ++i) {
+        const int32_t l = i + 1;
+        const bool free_to_go = l <= last_removable;
+        remove_mlp[i] = (r1 && free_to_go && l % p->m == 0) ? 1 : 0;
+        remove_attn[i] = (remove_mlp[i] || (cs && free_to_go && C[i] >= p->alpha)) ? 1 : 0;
+    }
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- life cycle
+extern "C" size_t asd_workspace_bytes(const asd_config* cfg) {
+    if (!cfg || !check_config(*cfg)) return 0;
+    return make_layout(*cfg).total;
+}
+
+extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, asd_ctx** out) {
+    if (!cfg || !out || !dev_workspace || !check_config(*cfg)) return ASD_ERR_ARG;
+    Layout lay = make_layout(*cfg);
+    if (bytes < lay.total || ((uintptr_t)dev_workspace % kAlign)) return ASD_ERR_NOMEM;
+    asd_ctx* x = new asd_ctx();
+    x->c = *cfg;
+    x->lay = lay;
+    x->ws = static_cast<unsigned char*>(dev_workspace);
+    x->stream = static_cast<cudaStream_t>(cuda_stream);
+    x->kv_dim = cfg->n_kv_heads * cfg->head_dim;
+    x->skip_attn.assign(cfg->n_layers, 0);
+    x->skip_mlp.assign(cfg->n_layers, 0);
+    auto bail = [&](cudaError_t e) {
+        fprintf(stderr, "asd_create: %s\n", cudaGetErrorString(e));
+        if (x->pinned) cudaFreeHost(x->pinned);
+        delete x;
+        return ASD_ERR_CUDA;
+    };
+    cudaError_t e = device_info(&x->dev);
+    if (e != cudaSuccess) return bail(e);
+    const size_t worst_attn = attn_smem_bytes(kMaxRows, cfg->head_dim);
+    if (worst_attn > (size_t)x->dev->max_smem) {
+        delete x;
+        return ASD_ERR_ARG;
+    }
+    if ((e = cudaHostAlloc((void**)&x->pinned, 4096, cudaHostAllocDefault)) != cudaSuccess) return bail(e);
+    // rotary table: angle(p, j) = p * theta^(-2j/head_dim), evaluated in double, stored as float
+    {
+        const int half = cfg->head_dim / 2;
+        std::vector<float> hc((size_t)cfg->max_seq * half), hs((size_t)cfg->max_seq * half);
+        std::vector<double> inv_freq(half);
+        for (int j = 0; j < half; ++j) inv_freq[j] = exp(-log((double)cfg->rope_theta) * (2.0 * j / cfg->head_dim));
+        for (int p = 0; p < cfg->max_seq; ++p)
+            for (int j = 0; j < half; ++j) {
+                const double a = (double)p * inv_freq[j];
+                hc[(size_t)p * half + j] = (float)cos(a);
+                hs[(size_t)p * half + j] = (float)sin(a);
+            }
+        if ((e = cudaMemcpyAsync(x->ws + lay.rope_cos, hc.data(), hc.size() * 4, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess) return bail(e);
+        if ((e = cudaMemcpyAsync(x->ws + lay.rope_sin, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess) return bail(e);
+        if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e);
+    }
+    // zero everything behind the weights: KV cache, scratch, counters
+    if ((e = cudaMemsetAsync(x->ws + lay.kcache, 0, lay.total - lay.kcache, x->stream)) != cudaSuccess) return bail(e);
+    if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e);
+    *out = x;
+    return ASD_OK;
+}
+
+extern "C" int asd_destroy(asd_ctx* x) {
+    if (!x) return ASD_ERR_ARG;
+    cudaStreamSynchronize(x->stream);
+    for (auto e : x->events) cudaEventDestroy(e);
+    if (x->pinned) cudaFreeHost(x->pinned);
+    delete x;
+    return ASD_OK;
+}
+
+extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : "null context"; }
+
+static int upload_weights(asd_ctx* x, const asd_host_weights& w) {
+    const asd_config& c = x->c;
+    const Layout& ly = x->lay;
+    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = x->kv_dim;
+    cudaStream_t s = x->stream;
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.embed, w.embed, V * d * 2, cudaMemcpyHostToDevice, s));
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.lm_head, w.lm_head, V * d * 2, cudaMemcpyHostToDevice, s));
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.final_norm, w.final_norm, d * 2, cudaMemcpyHostToDevice, s));
+    for (int l = 0; l < c.n_layers; ++l) {
+        unsigned char* lw = x->layer(l);
+        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_attn_norm, w.attn_norm + (size_t)l * d, d * 2, cudaMemcpyHostToDevice, s));
+        unsigned char* qkv = lw + ly.l_wqkv;
+        ASD_CUDA(x, cudaMemcpyAsync(qkv, w.wq + (size_t)l * d * d, d * d * 2, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpyAsync(qkv + d * d * 2, w.wk + (size_t)l * kvd * d, kvd * d * 2, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpyAsync(qkv + (d + kvd) * d * 2, w.wv + (size_t)l * kvd * d, kvd * d * 2, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_wo, w.wo + (size_t)l * d * d, d * d * 2, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_mlp_norm, w.mlp_norm + (size_t)l * d, d * 2, cudaMemcpyHostToDevice, s));
+        // gate row i -> row 2i, up row i -> row 2i+1, so that one warp holds both operands of SwiGLU
+        ASD_CUDA(x, cudaMemcpy2DAsync(lw + ly.l_wgu, 2 * d * 2, w.wg + (size_t)l * f * d, d * 2, d * 2, f, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpy2DAsync(lw + ly.l_wgu + d * 2, 2 * d * 2, w.wu + (size_t)l * f * d, d * 2, d * 2, f, cudaMemcpyHostToDevice, s));
+        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_wd, w.wd + (size_t)l * d * f, d * f * 2, cudaMemcpyHostToDevice, s));
+    }
+    ASD_CUDA(x, cudaStreamSynchronize(s));
+    x->have_weights = true;
+    return ASD_OK;
+}
+
+extern "C" int asd_load_weights_host(asd_ctx* x, const asd_host_weights* w) {
+    if (!x || !w) return ASD_ERR_ARG;
+    const void* ptrs[] = {w->embed, w->lm_head, w->final_norm, w->attn_norm, w->wq, w->wk, w->wv, w->wo, w->mlp_norm, w->wg, w->wu, w->wd};
+    for (const void* p : ptrs)
+        if (!p && x->c.n_layers > 0) return fail(x, ASD_ERR_ARG, "null weight pointer");
+    return upload_weights(x, *w);
+}
+
+extern "C" int asd_load_weights_file(asd_ctx* x, const char* path) {
+    if (!x || !path) return ASD_ERR_ARG;
+    const asd_config& c = x->c;
+    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = x->kv_dim, L = c.n_layers;
+    const size_t counts[12] = {V * d, V * d, d, L * d, L * d * d, L * kvd * d, L * kvd * d, L * d * d, L * d, L * f * d, L * f * d, L * d * f};
+    FILE* fh = fopen(path, "rb");
+    if (!fh) return fail(x, ASD_ERR_IO, std::string("cannot open ") + path);
+    std::vector<std::vector<uint16_t>> bufs(12);
+    for (int i = 0; i < 12; ++i) {
+        bufs[i].resize(counts[i]);
+        if (counts[i] && fread(bufs[i].data(), 2, counts[i], fh) != counts[i]) {
+            fclose(fh);
+            return fail(x, ASD_ERR_IO, "weight file is shorter than the configured shape");
+        }
+    }
+    fclose(fh);
+    asd_host_weights w{bufs[0].data(), bufs[1].data(), bufs[2].data(), bufs[3].data(), bufs[4].data(), bufs[5].data(),
+                       bufs[6].data(), bufs[7].data(), bufs[8].data(), bufs[9].data(), bufs[10].data(), bufs[11].data()};
+    return upload_weights(x, w);
+}
+
+extern "C" int asd_reset(asd_ctx* x) {
+    if (!x) return ASD_ERR_ARG;
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    x->n_committed = x->draft_cursor = 0;
+    std::fill(x->skip_attn.begin(), x->skip_attn.end(), 0);
+    std::fill(x->skip_mlp.begin(), x->skip_mlp.end(), 0);
+    x->n_sim_rows = 0;
+    x->last_M = 0;
+    x->stats = asd_stats{};
+    x->spans.clear();
+    x->events_used = 0;
+    ASD_CUDA(x, cudaMemsetAsync(x->ws + x->lay.sumcos, 0, (size_t)2 * std::max(x->c.n_layers, 1) * 8, x->stream));
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- prefill (Section 3.2)
+static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int32_t* first_token, bool resolve) {
+    if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (n <= 0) return fail(x, ASD_ERR_ARG, "empty prompt");
+    if ((long long)x->n_committed + n > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "prompt exceeds max_seq");
+    size_t e0, e1;
+    int rc = new_event(x, &e0);
+    if (rc) return rc;
+    int last_rows = 0;
+    for (int c0 = 0; c0 < n; c0 += kPrefillRows) {
+        const int M = std::min(kPrefillRows, n - c0);
+        const bool last = c0 + M >= n;
+        rc = run_pass(x, M, x->n_committed + c0, dev_tokens + c0, false, true, last, nullptr, false, nullptr);
+        if (rc) return rc;
+        last_rows = M;
+    }
+    rc = new_event(x, &e1);
+    if (rc) return rc;
+    x->spans.push_back({SPAN_PREFILL, e0, e1});
+    x->n_committed += n;
+    x->draft_cursor = x->n_committed;
+    x->n_sim_rows += n;
+    x->stats.prefill_rows += n;
+    if (first_token) {
+        ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax) + (last_rows - 1), 4, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+        *first_token = x->pinned[0];
+        if (resolve && (rc = resolve_spans(x))) return rc;
+    }
+    return ASD_OK;
+}
+
+extern "C" int asd_prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int32_t* first_token) {
+    if (!x || !dev_tokens) return ASD_ERR_ARG;
+    int32_t dummy;
+    return prefill_device(x, dev_tokens, n, first_token ? first_token : &dummy, true);
+}
+
+static int stage_tokens(asd_ctx* x, const int32_t* tokens, int32_t n, int32_t* dev_dst) {
+    for (int i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= x->c.vocab) return fail(x, ASD_ERR_ARG, "token id out of range");
+    ASD_CUDA(x, cudaMemcpyAsync(dev_dst, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));  // the host array is only borrowed for the call
+    return ASD_OK;
+}
+
+extern "C" int asd_prefill(asd_ctx* x, const int32_t* tokens, int32_t n, int32_t* first_token) {
+    if (!x || !tokens) return ASD_ERR_ARG;
+    if (n <= 0) return fail(x, ASD_ERR_ARG, "empty prompt");
+    if ((long long)x->n_committed + n > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "prompt exceeds max_seq");
+    int rc = stage_tokens(x, tokens, n, x->at<int>(x->lay.prompt_toks));
+    if (rc) return rc;
+    int32_t dummy;
+    return prefill_device(x, x->at<int>(x->lay.prompt_toks), n, first_token ? first_token : &dummy, true);
+}
+
+extern "C" int asd_get_similarity(asd_ctx* x, float* c_attn, float* c_mlp, int32_t* n_rows) {
+    if (!x) return ASD_ERR_ARG;
+    if (n_rows) *n_rows = (int32_t)x->n_sim_rows;
+    if (x->n_sim_rows == 0) return fail(x, ASD_ERR_STATE, "no prompt row has been processed");
+    const int L = x->c.n_layers;
+    std::vector<double> h(2 * (size_t)std::max(L, 1));
+    ASD_CUDA(x, cudaMemcpyAsync(h.data(), x->ws + x->lay.sumcos, h.size() * 8, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    for (int l = 0; l < L; ++l) {
+        if (c_attn) c_attn[l] = (float)(h[l] / (double)x->n_sim_rows);
+        if (c_mlp) c_mlp[l] = (float)(h[L + l] / (double)x->n_sim_rows);
+    }
+    return ASD_OK;
+}
+
+extern "C" int asd_set_skip_mask(asd_ctx* x, const uint8_t* skip_attn, const uint8_t* skip_mlp) {
+    if (!x || !skip_attn || !skip_mlp) return ASD_ERR_ARG;
+    for (int l = 0; l < x->c.n_layers; ++l) {
+        x->skip_attn[l] = skip_attn[l] ? 1 : 0;
+        x->skip_mlp[l] = skip_mlp[l] ? 1 : 0;
+    }
+    x->draft_cursor = x->n_committed;
+    return ASD_OK;
+}
+
+extern "C" int asd_admg_update(asd_ctx* x, const asd_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp) {
+    if (!x || !p) return ASD_ERR_ARG;
+    const int L = x->c.n_layers;
+    std::vector<float> C(std::max(L, 1));
+    int rc = asd_get_similarity(x, C.data(), nullptr, nullptr);
+    if (rc) return rc;
+    std::vector<uint8_t> a(std::max(L, 1)), b(std::max(L, 1));
+    rc = asd_admg(C.data(), L, p, a.data(), b.data());
+    if (rc) return fail(x, rc, "bad ADMG parameters");
+    asd_set_skip_mask(x, a.data(), b.data());
+    if (skip_attn) memcpy(skip_attn, a.data(), L);
+    if (skip_mlp) memcpy(skip_mlp, b.data(), L);
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- single passes
+static int timed_pass(asd_ctx* x, int kind, int M, int pos0, const int* dev_tokens, bool use_mask, int* dev_argmax_out, bool accept) {
+    size_t e0, e1;
+    int rc = new_event(x, &e0);
+    if (rc) return rc;
+    double bytes = 0;
+    rc = run_pass(x, M, pos0, dev_tokens, use_mask, false, true, dev_argmax_out, accept, &bytes);
+    if (rc) return rc;
+    rc = new_event(x, &e1);
+    if (rc) return rc;
+    x->spans.push_back({kind, e0, e1});
+    switch (kind) {
+        case SPAN_FULL: x->stats.full_passes += 1; x->stats.bytes_full += bytes; break;
+        case SPAN_DRAFT: x->stats.draft_passes += 1; x->stats.bytes_draft += bytes; break;
+        case SPAN_VERIFY: x->stats.verify_passes += 1; x->stats.bytes_verify += bytes; break;
+    }
+    return ASD_OK;
+}
+
+extern "C" int asd_decode_step(asd_ctx* x, int32_t token_in, int32_t* token_out) {
+    if (!x) return ASD_ERR_ARG;
+    if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (x->n_committed + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
+    int rc = stage_tokens(x, &token_in, 1, x->at<int>(x->lay.tok_in));
+    if (rc) return rc;
+    rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, x->at<int>(x->lay.tok_in), false, nullptr, false);
+    if (rc) return rc;
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax), 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    x->n_committed += 1;
+    x->draft_cursor = x->n_committed;
+    if (token_out) *token_out = x->pinned[0];
+    return resolve_spans(x);
+}
+
+extern "C" int asd_draft_step(asd_ctx* x, int32_t token_in, int32_t* token_out) {
+    if (!x) return ASD_ERR_ARG;
+    if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (x->draft_cursor + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
+    int rc = stage_tokens(x, &token_in, 1, x->at<int>(x->lay.tok_in));
+    if (rc) return rc;
+    rc = timed_pass(x, SPAN_DRAFT, 1, x->draft_cursor, x->at<int>(x->lay.tok_in), true, nullptr, false);
+    if (rc) return rc;
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax), 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    x->draft_cursor += 1;
+    if (token_out) *token_out = x->pinned[0];
+    return resolve_spans(x);
+}
+
+extern "C" int asd_verify(asd_ctx* x, const int32_t* tokens, int32_t k, int32_t* n_accepted, int32_t* out_tokens) {
+    if (!x || !tokens) return ASD_ERR_ARG;
+    if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (k < 0 || k > x->c.max_draft) return fail(x, ASD_ERR_ARG, "draft length out of range");
+    if ((long long)x->n_committed + k + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "verify would exceed max_seq");
+    int rc = stage_tokens(x, tokens, k + 1, x->at<int>(x->lay.draft_toks));
+    if (rc) return rc;
+    rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, x->at<int>(x->lay.draft_toks), false, nullptr, true);
+    if (rc) return rc;
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.accept), (size_t)(k + 2) * 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    const int a = x->pinned[0];
+    if (n_accepted) *n_accepted = a;
+    if (out_tokens)
+        for (int j = 0; j <= a; ++j) out_tokens[j] = x->pinned[1 + j];
+    x->n_committed += a + 1;
+    x->draft_cursor = x->n_committed;
+    x->stats.drafted += k;
+    x->stats.accepted += a;
+    return resolve_spans(x);
+}
+
+// ---------------------------------------------------------------- the whole method
+static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prompt, const asd_gen_params* gp,
+                           int32_t* dev_out, int32_t* n_out, asd_stats* stats) {
+    if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (n_prompt <= 0 || gp->max_new <= 0 || gp->draft_len < 0 || gp->draft_len > x->c.max_draft ||
+        gp->mode < ASD_MODE_AR || gp->mode > ASD_MODE_SPEC_MANUAL_MASK)
+        return fail(x, ASD_ERR_ARG, "bad generation parameters");
+    if (n_prompt > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "prompt exceeds max_seq");
+    std::vector<uint8_t> ka = x->skip_attn, km = x->skip_mlp;
+    int rc = asd_reset(x);
+    if (rc) return rc;
+    if (gp->mode == ASD_MODE_SPEC_MANUAL_MASK) asd_set_skip_mask(x, ka.data(), km.data());
+    cudaStream_t s = x->stream;
+    size_t ev_begin, ev_end;
+    if ((rc = new_event(x, &ev_begin))) return rc;
+
+    int32_t first = 0;
+    const bool need_host_token = gp->eos_id >= 0;
+    rc = prefill_device(x, dev_prompt, n_prompt, need_host_token ? &first : nullptr, false);
+    if (rc) return rc;
+    const int last_rows = (n_prompt - 1) % kPrefillRows + 1;
+    ASD_CUDA(x, cudaMemcpyAsync(dev_out, x->at<int>(x->lay.argmax) + (last_rows - 1), 4, cudaMemcpyDeviceToDevice, s));
+    int produced = 1;
+    bool stop = need_host_token && first == gp->eos_id;
+
+    if (gp->mode == ASD_MODE_SPEC) {
+        rc = asd_admg_update(x, &gp->admg, nullptr, nullptr);
+        if (rc) return rc;
+    }
+    int* draft = x->at<int>(x->lay.draft_toks);
+    int* accept = x->at<int>(x->lay.accept);
+
+    if (gp->mode == ASD_MODE_AR) {
+        // token i is read from dev_out[i-1] and written to dev_out[i]: no host round trip between steps
+        while (produced < gp->max_new && !stop) {
+            if (x->n_committed + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
+            rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, dev_out + produced - 1, false, dev_out + produced, false);
+            if (rc) return rc;
+            x->n_committed += 1;
+            if (need_host_token) {
+                ASD_CUDA(x, cudaMemcpyAsync(x->pinned, dev_out + produced, 4, cudaMemcpyDeviceToHost, s));
+                ASD_CUDA(x, cudaStreamSynchronize(s));
+                stop = x->pinned[0] == gp->eos_id;
+            }
+            ++produced;
+        }
+        x->draft_cursor = x->n_committed;
+    } else {
+        const int* last_src = dev_out;  // device address of the last emitted token
+        while (produced < gp->max_new && !stop) {
+            int k = std::min(gp->draft_len, gp->max_new - produced - 1);
+            k = std::min(k, x->c.max_seq - x->n_committed - 1);
+            if (k < 0) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
+            ASD_CUDA(x, cudaMemcpyAsync(draft, last_src, 4, cudaMemcpyDeviceToDevice, s));
+            for (int j = 0; j < k; ++j) {  // k steps of the draft model, chained on the device
+                rc = timed_pass(x, SPAN_DRAFT, 1, x->n_committed + j, draft + j, true, draft + j + 1, false);
+                if (rc) return rc;
+            }
+            rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, draft, false, nullptr, true);
+            if (rc) return rc;
+            ASD_CUDA(x, cudaMemcpyAsync(x->pinned, accept, (size_t)(k + 2) * 4, cudaMemcpyDeviceToHost, s));
+            ASD_CUDA(x, cudaStreamSynchronize(s));
+            const int a = x->pinned[0];
+            int emit = a + 1;
+            if (gp->eos_id >= 0)
+                for (int j = 0; j <= a; ++j)
+                    if (x->pinned[1 + j] == gp->eos_id) {
+                        emit = j + 1;
+                        stop = true;
+                        break;
+                    }
+            emit = std::min(emit, gp->max_new - produced);
+            ASD_CUDA(x, cudaMemcpyAsync(dev_out + produced, accept + 1, (size_t)emit * 4, cudaMemcpyDeviceToDevice, s));
+            produced += emit;
+            last_src = dev_out + produced - 1;
+            x->n_committed += a + 1;
+            x->draft_cursor = x->n_committed;
+            x->stats.rounds += 1;
+            x->stats.drafted += k;
+            x->stats.accepted += a;
+        }
+    }
+    if ((rc = new_event(x, &ev_end))) return rc;
+    ASD_CUDA(x, cudaStreamSynchronize(s));
+    float ms = 0.f;
+    ASD_CUDA(x, cudaEventElapsedTime(&ms, x->events[ev_begin], x->events[ev_end]));
+    x->stats.ms_total = ms;
+    rc = resolve_spans(x);
+    if (rc) return rc;
+    *n_out = produced;
+    if (stats) *stats = x->stats;
+    return ASD_OK;
+}
+
+extern "C" int asd_generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prompt, const asd_gen_params* p,
+                                   int32_t* dev_out, int32_t* n_out, asd_stats* stats) {
+    if (!x || !dev_prompt || !p || !dev_out || !n_out) return ASD_ERR_ARG;
+    return generate_device(x, dev_prompt, n_prompt, p, dev_out, n_out, stats);
+}
+
+extern "C" int asd_generate(asd_ctx* x, const int32_t* prompt, int32_t n_prompt, const asd_gen_params* p, int32_t* out,
+                            int32_t* n_out, asd_stats* stats) {
+    if (!x || !prompt || !p || !out || !n_out) return ASD_ERR_ARG;
+    if (n_prompt <= 0 || p->max_new <= 0) return fail(x, ASD_ERR_ARG, "bad generation parameters");
+    if (n_prompt > x->c.max_seq || p->max_new > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "request exceeds max_seq");
+    int rc = stage_tokens(x, prompt, n_prompt, x->at<int>(x->lay.prompt_toks));
+    if (rc) return rc;
+    int* gen = x->at<int>(x->lay.gen_toks);
+    rc = generate_device(x, x->at<int>(x->lay.prompt_toks), n_prompt, p, gen, n_out, stats);
+    if (rc) return rc;
+    ASD_CUDA(x, cudaMemcpyAsync(out, gen, (size_t)*n_out * 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- inspection
+extern "C" int asd_get_last_cosines(asd_ctx* x, int32_t* M, float* cos_attn, float* cos_mlp) {
+    if (!x) return ASD_ERR_ARG;
+    if (x->last_M == 0) return fail(x, ASD_ERR_STATE, "no pass has run");
+    const int L = x->c.n_layers, m = x->last_M;
+    if (M) *M = m;
+    std::vector<float> h((size_t)2 * std::max(L, 1) * kMaxRows);
+    ASD_CUDA(x, cudaMemcpyAsync(h.data(), x->ws + x->lay.cosv, h.size() * 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    for (int l = 0; l < L; ++l)
+        for (int r = 0; r < m; ++r) {
+            if (cos_attn) cos_attn[(size_t)l * m + r] = h[((size_t)0 * L + l) * kMaxRows + r];
+            if (cos_mlp) cos_mlp[(size_t)l * m + r] = h[((size_t)1 * L + l) * kMaxRows + r];
+        }
+    return ASD_OK;
+}
+
+extern "C" int asd_set_debug(asd_ctx* x, int32_t record_logits) {
+    if (!x) return ASD_ERR_ARG;
+    x->debug_logits = record_logits != 0;
+    return ASD_OK;
+}
+
+extern "C" int asd_get_last_logits(asd_ctx* x, int32_t* M, float* logits) {
+    if (!x) return ASD_ERR_ARG;
+    if (x->last_M == 0 || !x->last_has_logits) return fail(x, ASD_ERR_STATE, "no logits recorded (asd_set_debug)");
+    if (M) *M = x->last_M;
+    if (logits) {
+        ASD_CUDA(x, cudaMemcpyAsync(logits, x->ws + x->lay.logits, (size_t)x->last_M * x->c.vocab * 4, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    }
+    return ASD_OK;
+}
+
+extern "C" int asd_get_kv(asd_ctx* x, int32_t layer, int32_t pos, uint16_t* k, uint16_t* v) {
+    if (!x || layer < 0 || layer >= x->c.n_layers || pos < 0 || pos >= x->c.max_seq) return ASD_ERR_ARG;
+    const size_t off = (size_t)layer * x->lay.kv_layer_stride + (size_t)pos * x->kv_dim * 2;
+    if (k) ASD_CUDA(x, cudaMemcpyAsync(k, x->ws + x->lay.kcache + off, (size_t)x->kv_dim * 2, cudaMemcpyDeviceToHost, x->stream));
+    if (v) ASD_CUDA(x, cudaMemcpyAsync(v, x->ws + x->lay.vcache + off, (size_t)x->kv_dim * 2, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    return ASD_OK;
+}
+
+extern "C" int asd_get_positions(asd_ctx* x, int32_t* n_committed, int32_t* draft_cursor) {
+    if (!x) return ASD_ERR_ARG;
+    if (n_committed) *n_committed = x->n_committed;
+    if (draft_cursor) *draft_cursor = x->draft_cursor;
+    return ASD_OK;
+}
+
+extern "C" int asd_get_stats(asd_ctx* x, asd_stats* stats) {
+    if (!x || !stats) return ASD_ERR_ARG;
+    *stats = x->stats;
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- the sublayer building block on its own
+extern "C" size_t asd_fused_gemv_scratch_bytes(void) { return 256 + (size_t)kMaxGemvGrid * kMaxRows * 4 * 4; }
+
+extern "C" int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, const void* x, const uint16_t* gain,
+                              float eps, const uint16_t* W, int32_t epilogue, void* out, float* cosv, void* scratch,
+                              size_t scratch_bytes) {
+    if (!x || !W || !out || !scratch || M < 1 || M > kMaxRows || n_in <= 0 || n_in % 8 || n_rows <= 0) return ASD_ERR_ARG;
+    if (epilogue < ASD_EPI_PLAIN || epilogue > ASD_EPI_RESIDUAL) return ASD_ERR_ARG;
+    if (epilogue == ASD_EPI_SWIGLU && (n_rows & 1)) return ASD_ERR_ARG;
+    if (epilogue == ASD_EPI_RESIDUAL && !cosv) return ASD_ERR_ARG;
+    if (scratch_bytes < asd_fused_gemv_scratch_bytes() || ((uintptr_t)scratch % kAlign)) return ASD_ERR_NOMEM;
+    DeviceInfo* dv = nullptr;
+    if (device_info(&dv) != cudaSuccess) return ASD_ERR_CUDA;
+    GemvParams p{};
+    p.W = reinterpret_cast<const __nv_bfloat16*>(W);
+    p.n_rows = n_rows;
+    p.n_in = n_in;
+    p.x = x;
+    p.gain = reinterpret_cast<const __nv_bfloat16*>(gain);
+    p.eps = eps;
+    p.out = out;
+    p.cos_out = cosv;
+    p.counter = reinterpret_cast<unsigned*>(scratch);
+    p.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + 256);
+    int grid, xin;
+    size_t smem;
+    if (!plan_gemv(*dv, M, n_rows, n_in, gain != nullptr, &grid, &xin, &smem)) return ASD_ERR_ARG;
+    p.x_in_smem = xin;
+    if (launch_gemv(M, epilogue, gain != nullptr, p, grid, smem, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return ASD_ERR_CUDA;
+    return ASD_OK;
+}

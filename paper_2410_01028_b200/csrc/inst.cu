@@ -1,0 +1,56 @@
+// Instantiations of the row-count-templated kernels; compiled once per ASD_M in 1..9.
+#include "attn.cuh"
+#include "gemv.cuh"
+
+#ifndef ASD_M
+#error "compile with -DASD_M=<rows>"
+#endif
+
+namespace asd {
+
+#define ASD_CAT2(a, b) a##b
+#define ASD_CAT(a, b) ASD_CAT2(a, b)
+
+template <int EPI, bool NORM>
+static cudaError_t launch_one(const GemvParams& p, int grid, size_t smem, cudaStream_t s) {
+    gemv_kernel<ASD_M, EPI, NORM><<<grid, kGemvThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t ASD_CAT(launch_gemv_m, ASD_M)(int epi, bool norm, const GemvParams& p, int grid, size_t smem, cudaStream_t s) {
+    switch (epi) {
+        case kEpiPlain: return norm ? launch_one<kEpiPlain, true>(p, grid, smem, s) : launch_one<kEpiPlain, false>(p, grid, smem, s);
+        case kEpiSwiglu: return norm ? launch_one<kEpiSwiglu, true>(p, grid, smem, s) : launch_one<kEpiSwiglu, false>(p, grid, smem, s);
+        case kEpiResidual: return norm ? launch_one<kEpiResidual, true>(p, grid, smem, s) : launch_one<kEpiResidual, false>(p, grid, smem, s);
+        case kEpiQkv: return norm ? launch_one<kEpiQkv, true>(p, grid, smem, s) : cudaErrorInvalidValue;
+        case kEpiArgmax: return norm ? launch_one<kEpiArgmax, true>(p, grid, smem, s) : cudaErrorInvalidValue;
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t ASD_CAT(launch_attn_m, ASD_M)(const AttnParams& p, size_t smem, cudaStream_t s) {
+    dim3 grid(p.n_chunks, p.n_kv_heads);
+    attn_kernel<ASD_M><<<grid, kAttnThreads, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+// opt every instantiation in to large dynamic shared memory
+cudaError_t ASD_CAT(configure_m, ASD_M)(int max_smem) {
+    cudaError_t e;
+#define ASD_SET(k)                                                                              \
+    e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);         \
+    if (e != cudaSuccess) return e;
+    ASD_SET((gemv_kernel<ASD_M, kEpiPlain, true>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiPlain, false>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiSwiglu, true>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiSwiglu, false>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiResidual, true>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiResidual, false>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiQkv, true>))
+    ASD_SET((gemv_kernel<ASD_M, kEpiArgmax, true>))
+    ASD_SET((attn_kernel<ASD_M>))
+#undef ASD_SET
+    return cudaSuccess;
+}
+
+}  // namespace asd

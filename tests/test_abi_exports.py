@@ -1,0 +1,66 @@
+"""The C-ABI library builds, loads and exports every symbol include/asd.h declares (no GPU needed)."""
+import os
+import re
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "asd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(asd_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    import paper_2410_01028_b200 as asd
+    from paper_2410_01028_b200 import binding
+    L = asd.lib()
+    declared = _declared_symbols()
+    assert len(declared) >= 20
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(binding.EXPORTS) == declared
+
+
+def test_workspace_bytes_and_config_validation():
+    import paper_2410_01028_b200 as asd
+    import synth
+    from paper_2410_01028_b200.binding import make_config
+    cfg = make_config(synth.TINY, 128, 4)
+    n = asd.workspace_bytes(cfg)
+    weights = 2 * synth.make_model(synth.TINY).nbytes() // 2
+    assert n > weights
+    bad = make_config(synth.TINY, 128, 4)
+    bad.head_dim = 60  # heads * head_dim != d_model
+    assert asd.workspace_bytes(bad) == 0
+    bad = make_config(synth.TINY, 128, 9)  # draft length beyond the kernels' row limit
+    assert asd.workspace_bytes(bad) == 0
+    # 7B shape with room for 8192 + 512 positions fits one 180 GB device many times over
+    big = asd.workspace_bytes(make_config(synth.LLAMA_7B, 8192 + 512 + 16, 8))
+    assert 17e9 < big < 20e9
+
+
+def test_host_admg_matches_hand_derived_sets():
+    import paper_2410_01028_b200 as asd
+    C = np.full(40, 0.5, np.float32)
+    C[[0, 1, 38, 39]] = 0.99
+    ra, rm = asd.admg(C, 0.985, 3, 2)
+    assert {i + 1 for i in np.flatnonzero(rm)} == set(range(3, 37, 3))
+    assert {i + 1 for i in np.flatnonzero(ra)} == set(range(3, 37, 3)) | {1, 2}
+    ra, rm = asd.admg(C, 0.985, 3, 2, asd.USE_CS)
+    assert {i + 1 for i in np.flatnonzero(ra)} == {1, 2, 39, 40} and rm.sum() == 0
+
+
+def test_host_admg_agrees_with_oracle_on_random_inputs():
+    import oracle
+    import paper_2410_01028_b200 as asd
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        L = int(rng.integers(1, 48))
+        C = rng.uniform(0.9, 1.0, L).astype(np.float32)
+        m, n, flags = int(rng.integers(0, 6)), int(rng.integers(0, 6)), int(rng.integers(0, 8))
+        a1, b1 = asd.admg(C, 0.95, m, n, flags)
+        a2, b2 = oracle.admg(C, 0.95, m, n, flags)
+        assert a1.tolist() == a2.tolist() and b1.tolist() == b2.tolist()

@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the adaptive self-speculative decoding hot path on B200.
+
+One step = one whole generation on one sequence: prefill of the prompt with the per-sublayer cosine
+similarities, Algorithm 1 (ADMG), then rounds of draft steps under the skip mask and one (k+1)-row greedy
+verify, until ``max_new`` tokens.  Default workload: the Llama-2-7B-shaped decoder with a 512-token random
+prompt and 256 generated tokens.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 7b|13b|7b_long|tiny]
+
+With N > 1 (launched by torch.distributed.run) every rank decodes its own sequence on its own GPU: the path
+has no exchange step, so ranks are independent replicas and the value is the sum over ranks.
+``--impl reference`` times the CPU oracle on a bounded sample of the same workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (shape, prompt_len, max_new, description)
+    "tiny": (synth.TINY, 32, 64, "tiny decoder L=4 d=256, prompt 32, generate 64"),
+    "7b": (synth.LLAMA_7B, 512, 256, "Llama-2-7B-shaped decoder, prompt 512, generate 256"),
+    "13b": (synth.LLAMA_13B, 1024, 256, "Llama-2-13B-shaped decoder, prompt 1024, generate 256"),
+    "7b_long": (synth.LLAMA_7B, 8192, 512, "Llama-2-7B-shaped decoder, prompt 8192, generate 512"),
+}
+METRIC = "speculative decode tokens/s"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
+    ap.add_argument("--draft-len", type=int, default=4)
+    ap.add_argument("--alpha", type=float, default=0.9995)
+    ap.add_argument("--m", type=int, default=3)
+    ap.add_argument("--n", type=int, default=2)
+    ap.add_argument("--flags", type=int, default=5, help="ADMG rule subset: 1=CS thresholding, 2=rule 1, 4=rule 2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    # reduced cases for profiler captures only (never for a reported number)
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
+    ap.add_argument("--max-new", type=int, default=0, help="override the workload's generation length")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload(args):
+    import dataclasses
+    shape, S, new, desc = WORKLOADS[args.workload]
+    reduced = []
+    if args.layers:
+        shape = dataclasses.replace(shape, n_layers=args.layers); reduced.append("%d layers" % args.layers)
+    if args.prompt_len:
+        S = args.prompt_len; reduced.append("prompt %d" % S)
+    if args.max_new:
+        new = args.max_new; reduced.append("generate %d" % new)
+    if reduced:
+        desc += " [REDUCED for profiling: " + ", ".join(reduced) + "]"
+    return shape, S, new, desc
+
+
+def admg_kwargs(a):
+    return dict(draft_len=a.draft_len, alpha=a.alpha, m=a.m, n=a.n, flags=a.flags)
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(args, model, shape, prompt, steps, warmup):
+    """The oracle, as it stands, on a bounded sample of the workload: the first 64 prompt tokens, 12 new tokens."""
+    import oracle
+    n_prompt, max_new = min(64, len(prompt)), 12
+    orc = oracle.Oracle(model, max_seq=n_prompt + max_new + 8)
+    kw = admg_kwargs(args)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        toks, _, st = orc.generate(prompt[:n_prompt], max_new, mode=oracle.MODE_SPEC, **kw)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    per_step = sum(times) / len(times)
+    return {"value": max_new / per_step, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "first %d prompt tokens, %d generated tokens, same ADMG and draft settings; %.1f s per step"
+                      % (n_prompt, max_new, per_step)}, per_step
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape, S, new, desc = workload(args)
+    model = synth.make_model(shape, seed=0)
+    prompt = synth.make_prompt(shape.vocab, S, seed=1)
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    cb, per_step = oracle_sample(args, model, shape, prompt, steps, warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": desc, "sample": cb["sample"], **admg_kwargs(args)},
+            "cpu_baseline": cb,
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------- GPU legs
+def gemv_roofline(torch, asd, shape, hbm_peak):
+    """Times the dominant kernel alone: the fused RMSNorm -> gate/up GEMV -> SwiGLU sublayer product at M = 1,
+    over a pool of distinct weight matrices larger than L2, with CUDA events on the launching stream."""
+    d, f = shape.d_model, shape.d_ffn
+    n_rows = 2 * f
+    per_launch = n_rows * d * 2
+    pool = max(2, int(400e6 // per_launch) + 1)
+    dev = torch.device("cuda")
+    W = [torch.from_numpy(synth.make_matrix_bf16((n_rows, d), seed=7, stream=100 + i).view(np.int16)).to(dev)
+         .view(torch.bfloat16) for i in range(min(pool, 4))]
+    while len(W) < pool:
+        W.append(W[len(W) % 4].clone())
+    x = torch.from_numpy(synth.make_array_f32((1, d), seed=7, stream=99)).to(dev)
+    gain = torch.from_numpy(synth.make_matrix_bf16((d,), seed=7, stream=98, mean=1.0).view(np.int16)).to(dev).view(torch.bfloat16)
+    out = torch.empty((1, f), dtype=torch.bfloat16, device=dev)
+    scratch = torch.zeros(asd.fused_gemv_scratch_bytes(), dtype=torch.uint8, device=dev)
+    n = 200
+    for i in range(20):
+        asd.fused_gemv(x, W[i % pool], asd.EPI_SWIGLU, out, gain=gain, scratch=scratch)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        asd.fused_gemv(x, W[i % pool], asd.EPI_SWIGLU, out, gain=gain, scratch=scratch)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    achieved = per_launch / (us * 1e-6) / 1e9
+    return {"kernel": "gemv_kernel<M=1, swiglu, rmsnorm> %dx%d" % (n_rows, d), "bytes_per_launch": per_launch,
+            "us_per_launch": us, "achieved": achieved, "pool_matrices": pool}
+
+
+def run_ours(args):
+    import torch
+    import paper_2410_01028_b200 as asd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    shape, S, new, desc = workload(args)
+    hbm_peak, peak_kind = peaks()
+
+    model = synth.make_model(shape, seed=0)
+    dec = asd.Decoder(shape, max_seq=S + new + 16, max_draft=8, device="cuda:%d" % local)
+    dec.load_weights_host(model)
+    prompt = synth.make_prompt(shape.vocab, S, seed=1 + rank)       # every replica decodes its own sequence
+    dev_prompt = torch.from_numpy(prompt).cuda()
+    dev_out = torch.zeros(new, dtype=torch.int32, device="cuda")
+    kw = admg_kwargs(args)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # plain greedy decoding of the same workload by the same library (comparison value, outside the timed region)
+    n_ar, st_ar = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_AR)
+    ar_tokens = dev_out.cpu().numpy().copy()
+
+    for _ in range(args.warmup):
+        dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+    sampler = ClockSampler(local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    launches = 0
+    agg = None
+    for _ in range(args.steps):
+        n_out, st = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        launches += st["kernel_launches"]
+        agg = st if agg is None else {k: agg[k] + st[k] for k in st}
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    lossless = bool((dev_out.cpu().numpy() == ar_tokens).all())
+    value = world * args.steps * new / (ms * 1e-3)
+
+    # end to end through the host-buffer entry point: prompt from pinned host memory, tokens back to the host
+    pinned = torch.from_numpy(prompt).pin_memory()
+    host_prompt = pinned.numpy()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        toks, _ = dec.generate(host_prompt, new, mode=asd.MODE_SPEC, **kw)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * args.steps * new / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
+           "d2h_bytes_per_step": int(toks.nbytes) + 4 * int(agg["rounds"] // args.steps) * (args.draft_len + 2)}
+
+    if rank != 0:
+        return
+
+    def per_pass(kind, st):
+        n = st[kind + "_passes"]
+        if not n:
+            return None
+        msp = st["ms_" + kind] / n
+        gbs = st["bytes_" + kind] / st["ms_" + kind] / 1e6
+        return {"ms": msp, "GBps": gbs, "frac_of_%s_peak" % peak_kind: gbs / hbm_peak, "frac_of_8TBps": gbs / 8000.0}
+
+    passes = {"full": per_pass("full", st_ar), "draft": per_pass("draft", agg), "verify": per_pass("verify", agg)}
+    roof = gemv_roofline(torch, asd, shape, hbm_peak)
+    roofline = {"bound": "hbm", "achieved": roof["achieved"], "peak": hbm_peak, "unit": "GB/s",
+                "frac": roof["achieved"] / hbm_peak, "traffic": None, "peak_kind": peak_kind, "kernel": roof["kernel"],
+                "bytes_per_launch": roof["bytes_per_launch"], "us_per_launch": roof["us_per_launch"],
+                "how": "CUDA events over 200 launches rotating over %d weight matrices (> L2)" % roof["pool_matrices"]}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 weights and activations, f32 accumulate", "data": "synthetic",
+        "config": {"workload": desc, "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (model.nbytes() / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU", **kw},
+        "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": roofline, "passes": passes,
+        "decode_tokens_per_s": (new - 1) / ((agg["ms_total"] - agg["ms_prefill"]) / args.steps * 1e-3),
+        "prefill_ms": agg["ms_prefill"] / args.steps,
+        "ar_tokens_per_s": new / (st_ar["ms_total"] * 1e-3),
+        "ar_decode_tokens_per_s": (new - 1) / ((st_ar["ms_total"] - st_ar["ms_prefill"]) * 1e-3),
+        "acceptance": agg["accepted"] / max(agg["drafted"], 1), "rounds_per_step": agg["rounds"] / args.steps,
+        "spec_equals_ar": lossless,
+    }
+    if not args.no_cpu_baseline:
+        cb, _ = oracle_sample(args, model, shape, synth.make_prompt(shape.vocab, S, seed=1), 1, 0)
+        line["cpu_baseline"] = cb
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

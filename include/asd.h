@@ -189,6 +189,25 @@ int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, c
                    float eps, const uint16_t* W, int32_t epilogue, void* out, float* cos, void* scratch,
                    size_t scratch_bytes);
 
+/* The same fused sublayer product for callers that must not allocate (the paper has no counterpart; this is
+ * a deployment convenience). Some hosts of this library cannot call cudaMalloc at the point where they need
+ * the kernel: code running inside a memory pool that owns the whole device, a plug-in whose host forbids
+ * driver allocations after start-up, or a latency-critical loop in which an allocation would synchronise the
+ * device. For them the cross-CTA scratch of asd_fused_gemv lives in a fixed array inside the library image
+ * (about 42 KB of device memory per GPU that loads the library, held until the process exits), so the caller
+ * passes only inputs and outputs. Arguments and results are exactly those of asd_fused_gemv.
+ *   - Limit: the array covers launch plans of up to 296 CTAs. A shape whose plan needs more (very many rows
+ *     with a long reduction dimension and many activation rows) is rejected with ASD_ERR_NOMEM and a message on
+ *     stderr; use asd_fused_gemv with your own scratch for those.
+ *   - The first call on each device looks up the array's device address (that device must be current) and
+ *     configures the kernels; make that first call outside any stream capture.
+ *   - All calls on a device share the one array: two calls whose kernels can overlap on the GPU (different
+ *     streams without ordering, or several host threads) race on it. Order them on one stream.
+ *   - The call itself allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
+ * Errors: ARG, NOMEM (plan larger than the built-in array), CUDA. Asynchronous on the stream. */
+int asd_fused_gemv_static(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, const void* x,
+                          const uint16_t* gain, float eps, const uint16_t* W, int32_t epilogue, void* out, float* cos);
+
 /* Algorithm 1 as a pure host function (no context): C[L] -> remove_attn[L], remove_mlp[L]. */
 int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp);
 

@@ -51,7 +51,7 @@ EXPORTS = (
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
     "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_kv", "asd_get_positions", "asd_get_stats",
-    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_admg",
+    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg",
 )
 
 _lib = None
@@ -126,6 +126,20 @@ def fused_gemv(x, W, epilogue, out, gain=None, eps=1e-5, cos=None, scratch=None,
                               _vp(cos), _vp(scratch), ctypes.c_size_t(scratch.numel() * scratch.element_size()))
     if rc:
         raise AsdError(rc, "asd_fused_gemv")
+
+
+def fused_gemv_static(x, W, epilogue, out, gain=None, eps=1e-5, cos=None, stream=None):
+    """asd_fused_gemv_static: as ``fused_gemv`` but with the library's built-in scratch array, for callers that
+    cannot allocate device memory. Calls that may overlap on the GPU must be ordered on one stream."""
+    import torch
+    M, n_in = x.shape
+    n_rows = W.shape[0]
+    st = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    rc = lib().asd_fused_gemv_static(ctypes.c_void_p(st), ctypes.c_int32(M), ctypes.c_int32(n_in),
+                                     ctypes.c_int32(n_rows), _vp(x), _vp(gain), ctypes.c_float(eps), _vp(W),
+                                     ctypes.c_int32(epilogue), _vp(out), _vp(cos))
+    if rc:
+        raise AsdError(rc, "asd_fused_gemv_static")
 
 
 class Decoder:

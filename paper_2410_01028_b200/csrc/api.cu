@@ -927,3 +927,61 @@ extern "C" int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_
         return ASD_ERR_CUDA;
     return ASD_OK;
 }
+
+// ---------------------------------------------------------------- the same product without any allocation
+// Scratch for callers that cannot allocate device memory: a fixed array in the library image. In host code
+// the symbol below is only a handle; its device address is looked up once per device.
+constexpr int kStaticMaxGrid = 296;
+constexpr size_t kStaticScratchBytes = 256 + (size_t)kStaticMaxGrid * kMaxRows * 4 * 4;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static void* g_static_scratch_addr[64];
+
+extern "C" int asd_fused_gemv_static(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, const void* x,
+                                     const uint16_t* gain, float eps, const uint16_t* W, int32_t epilogue, void* out,
+                                     float* cosv) {
+    if (!x || !W || !out || M < 1 || M > kMaxRows || n_in <= 0 || n_in % 8 || n_rows <= 0) return ASD_ERR_ARG;
+    if (epilogue < ASD_EPI_PLAIN || epilogue > ASD_EPI_RESIDUAL) return ASD_ERR_ARG;
+    if (epilogue == ASD_EPI_SWIGLU && (n_rows & 1)) return ASD_ERR_ARG;
+    if (epilogue == ASD_EPI_RESIDUAL && !cosv) return ASD_ERR_ARG;
+    DeviceInfo* dv = nullptr;
+    if (device_info(&dv) != cudaSuccess) return ASD_ERR_CUDA;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ASD_ERR_CUDA;
+    if (!g_static_scratch_addr[dev]) {  // first call on this device: resolve the array's device address
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) {
+            fprintf(stderr, "asd_fused_gemv_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+            return ASD_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = ptr;
+    }
+    unsigned char* scratch = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
+    int grid, xin;
+    size_t smem;
+    if (!plan_gemv(*dv, M, n_rows, n_in, gain != nullptr, &grid, &xin, &smem)) return ASD_ERR_ARG;
+    if (grid > kStaticMaxGrid) {
+        fprintf(stderr,
+                "asd_fused_gemv_static: this shape needs a %d-CTA launch plan but the built-in scratch array holds "
+                "partials for at most %d CTAs; call asd_fused_gemv with caller-provided scratch instead\n",
+                grid, kStaticMaxGrid);
+        return ASD_ERR_NOMEM;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps whatever the previous call left: the arrival counter must start at zero
+    if (cudaMemsetAsync(scratch, 0, 256, s) != cudaSuccess) return ASD_ERR_CUDA;
+    GemvParams p{};
+    p.W = reinterpret_cast<const __nv_bfloat16*>(W);
+    p.n_rows = n_rows;
+    p.n_in = n_in;
+    p.x = x;
+    p.gain = reinterpret_cast<const __nv_bfloat16*>(gain);
+    p.eps = eps;
+    p.out = out;
+    p.cos_out = cosv;
+    p.counter = reinterpret_cast<unsigned*>(scratch);
+    p.partials = reinterpret_cast<float*>(scratch + 256);
+    p.x_in_smem = xin;
+    if (launch_gemv(M, epilogue, gain != nullptr, p, grid, smem, s) != cudaSuccess) return ASD_ERR_CUDA;
+    return ASD_OK;
+}

@@ -10,6 +10,7 @@
 
 #include "../../include/asd.h"
 #include "common.cuh"
+#include "pass.cuh"
 
 namespace asd {
 
@@ -29,11 +30,6 @@ size_t gemv_smem_bytes(int M, int n_rows, int n_in, int grid, bool x_in_smem) {
     if (x_in_smem) b += (size_t)M * n_in * 2;
     return b;
 }
-size_t attn_smem_bytes(int M, int head_dim) {
-    return (size_t)kAttnChunk * (head_dim + 8) * 2 + (size_t)kAttnChunk * head_dim * 2 + (size_t)M * head_dim * 4 +
-           (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16;
-}
-
 static cudaError_t launch_gemv(int M, int epi, bool norm, const GemvParams& p, int grid, size_t smem, cudaStream_t s) {
     switch (M) {
         case 1: return launch_gemv_m1(epi, norm, p, grid, smem, s);
@@ -48,17 +44,17 @@ static cudaError_t launch_gemv(int M, int epi, bool norm, const GemvParams& p, i
     }
     return cudaErrorInvalidValue;
 }
-static cudaError_t launch_attn(int M, const AttnParams& p, size_t smem, cudaStream_t s) {
+static cudaError_t launch_pass(int M, const PassParams& p, int grid, size_t smem, cudaStream_t s) {
     switch (M) {
-        case 1: return launch_attn_m1(p, smem, s);
-        case 2: return launch_attn_m2(p, smem, s);
-        case 3: return launch_attn_m3(p, smem, s);
-        case 4: return launch_attn_m4(p, smem, s);
-        case 5: return launch_attn_m5(p, smem, s);
-        case 6: return launch_attn_m6(p, smem, s);
-        case 7: return launch_attn_m7(p, smem, s);
-        case 8: return launch_attn_m8(p, smem, s);
-        case 9: return launch_attn_m9(p, smem, s);
+        case 1: return launch_pass_m1(p, grid, smem, s);
+        case 2: return launch_pass_m2(p, grid, smem, s);
+        case 3: return launch_pass_m3(p, grid, smem, s);
+        case 4: return launch_pass_m4(p, grid, smem, s);
+        case 5: return launch_pass_m5(p, grid, smem, s);
+        case 6: return launch_pass_m6(p, grid, smem, s);
+        case 7: return launch_pass_m7(p, grid, smem, s);
+        case 8: return launch_pass_m8(p, grid, smem, s);
+        case 9: return launch_pass_m9(p, grid, smem, s);
     }
     return cudaErrorInvalidValue;
 }
@@ -114,11 +110,34 @@ static bool plan_gemv(const DeviceInfo& dv, int M, int n_rows, int n_in, bool no
     return false;
 }
 
-__global__ void embed_kernel(const int* tokens, const __nv_bfloat16* E, float* x, int d, int vocab) {
-    const int m = blockIdx.x;
-    int t = tokens[m];
-    t = min(max(t, 0), vocab - 1);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)m * d + i] = __bfloat162float(E[(size_t)t * d + i]);
+// Shared-memory plan of the persistent pass kernel for M rows: ring slots, barriers, reduction scratch,
+// per-pair partial sums, activation window / attention scratch.
+struct PassPlan {
+    int ns, attn_groups, off_bars, off_misc, off_psum, off_reg_a;
+    size_t smem;
+};
+
+static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan* pl) {
+    const int kvd = c.n_kv_heads * c.head_dim;
+    const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
+    const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
+    const size_t psum = ((size_t)np_max * 2 * M * 4 + 15) & ~(size_t)15;
+    const size_t misc = ((size_t)16 * kMaxRows * 4 * 4 + 32 + 15) & ~(size_t)15;
+    const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16 + 15) & ~(size_t)15;
+    const size_t xs = (size_t)M * pass_wseg(M) * kSeg * 2;
+    const size_t reg_a = (std::max(xs, 2 * attn_scratch) + 15) & ~(size_t)15;
+    const long long avail = (long long)dv.max_smem - 1024 - (long long)(psum + misc + reg_a) - 2 * 64 * 8;
+    int ns = (int)std::min<long long>(64, avail / kSlotBytes);
+    const int tile_slots = 4 * std::max(1, c.head_dim / 64);
+    if (ns < 2 * tile_slots || ns < 8) return false;
+    pl->ns = ns;
+    pl->attn_groups = ns >= 4 * tile_slots ? 2 : 1;
+    pl->off_bars = ns * kSlotBytes;
+    pl->off_misc = pl->off_bars + 2 * 64 * 8;
+    pl->off_psum = pl->off_misc + (int)misc;
+    pl->off_reg_a = pl->off_psum + (int)psum;
+    pl->smem = (size_t)pl->off_reg_a + reg_a + 1024;
+    return pl->smem <= (size_t)dv.max_smem;
 }
 
 // ---------------------------------------------------------------- workspace layout
@@ -128,6 +147,8 @@ struct Layout {
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
     size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
     size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits;
+    size_t stage_tab, tmaps, sync_words;
+    int max_stages;
     size_t total;
     int chunk_stride;
 };
@@ -137,7 +158,9 @@ static bool check_config(const asd_config& c) {
         c.vocab <= 0 || c.max_seq <= 0)
         return false;
     if ((long long)c.n_heads * c.head_dim != c.d_model || c.n_heads % c.n_kv_heads) return false;
-    if (c.head_dim % 8 || c.head_dim > 256 || c.d_model % 8 || c.d_ffn % 8) return false;
+    if ((c.head_dim != 16 && c.head_dim != 32 && c.head_dim != 64 && c.head_dim != 128 && c.head_dim != 256) || c.d_model % 8 ||
+        c.d_ffn % 8)
+        return false;
     if (c.max_draft < 0 || c.max_draft > kMaxRows - 1) return false;
     if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return false;
     return true;
@@ -194,6 +217,10 @@ static Layout make_layout(const asd_config& c) {
     L.argmax = take(64 * 4);
     L.accept = take(64 * 4);
     L.logits = take((size_t)kMaxRows * V * 4);
+    L.max_stages = 5 * c.n_layers + 2;
+    L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
+    L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
+    L.sync_words = take(256);
     L.total = o;
     return L;
 }
@@ -218,6 +245,8 @@ struct asd_ctx {
     bool debug_logits = false, last_has_logits = false;
     asd_stats stats{};
     int32_t* pinned = nullptr;  // small host staging buffer
+    uint32_t bar_base = 0;      // value of the grid-barrier counter at the start of the next pass
+    int n_stages_full = 0, n_stages_draft = 0;
     std::vector<cudaEvent_t> events;
     size_t events_used = 0;
     struct Span { int kind; size_t e0, e1; };
@@ -270,9 +299,107 @@ static int resolve_spans(asd_ctx* x) {
     return ASD_OK;
 }
 
+// ---------------------------------------------------------------- stage tables and tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// One 2-D tensor map per layer and per cache: [max_seq rows, kv_dim columns] bf16, boxes of 32 keys x (up to) 64
+// columns; 128-byte rows are stored with the 128-byte swizzle so that one thread per key reads its row without
+// shared-memory bank conflicts.
+static int make_tensor_maps(asd_ctx* x) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    ASD_CUDA(x, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return fail(x, ASD_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+    const asd_config& c = x->c;
+    const int L = c.n_layers;
+    std::vector<CUtensorMap> maps((size_t)2 * std::max(L, 1));
+    const int box_cols = c.head_dim > 64 ? 64 : c.head_dim;
+    const cuuint64_t gdim[2] = {(cuuint64_t)x->kv_dim, (cuuint64_t)c.max_seq};
+    const cuuint64_t gstride[1] = {(cuuint64_t)x->kv_dim * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, 32u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUtensorMapSwizzle swz = (box_cols * 2 == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    for (int l = 0; l < L; ++l)
+        for (int which = 0; which < 2; ++which) {
+            void* base = x->ws + (which ? x->lay.vcache : x->lay.kcache) + (size_t)l * x->lay.kv_layer_stride;
+            const CUresult r = encode(&maps[(size_t)l * 2 + which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box,
+                                      estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(x, ASD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the KV cache");
+        }
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + x->lay.tmaps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    return ASD_OK;
+}
+
+// Stage tables of the persistent pass kernel: table 0 = the full model M, table 1 = the draft model D (M
+// without the sublayers in the skip mask: they get no stage, so nothing is streamed or touched for them).
+static int build_stage_tables(asd_ctx* x) {
+    const asd_config& c = x->c;
+    const Layout& ly = x->lay;
+    const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
+    float* cosv = x->at<float>(ly.cosv);
+    const CUtensorMap* maps = x->at<CUtensorMap>(ly.tmaps);
+    std::vector<StageDesc> tab((size_t)2 * ly.max_stages);
+    for (int which = 0; which < 2; ++which) {
+        StageDesc* t = tab.data() + (size_t)which * ly.max_stages;
+        int n = 0;
+        t[n] = StageDesc{};
+        t[n++].type = kStEmbed;
+        for (int l = 0; l < L; ++l) {
+            unsigned char* lw = x->layer(l);
+            __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.kcache + (size_t)l * ly.kv_layer_stride);
+            __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.vcache + (size_t)l * ly.kv_layer_stride);
+            if (!(which && x->skip_attn[l])) {
+                StageDesc q{};
+                q.type = kStQkv, q.layer = l, q.n_rows = d + 2 * kvd, q.n_in = d;
+                q.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wqkv);
+                q.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_attn_norm);
+                q.k_cache = kc, q.v_cache = vc;
+                t[n++] = q;
+                StageDesc a{};
+                a.type = kStAttn, a.layer = l;
+                a.k_cache = kc, a.v_cache = vc;
+                a.tm_k = maps + (size_t)l * 2, a.tm_v = maps + (size_t)l * 2 + 1;
+                t[n++] = a;
+                StageDesc o{};
+                o.type = kStOproj, o.layer = l, o.n_rows = d, o.n_in = d;
+                o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wo);
+                o.cos_out = cosv + (size_t)(0 * L + l) * kMaxRows;
+                o.sumcos = x->at<double>(ly.sumcos) + l;
+                t[n++] = o;
+            }
+            if (!(which && x->skip_mlp[l])) {
+                StageDesc g{};
+                g.type = kStGateUp, g.layer = l, g.n_rows = 2 * f, g.n_in = d;
+                g.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wgu);
+                g.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_mlp_norm);
+                t[n++] = g;
+                StageDesc w{};
+                w.type = kStDown, w.layer = l, w.n_rows = d, w.n_in = f;
+                w.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wd);
+                w.cos_out = cosv + (size_t)(1 * L + l) * kMaxRows;
+                w.sumcos = x->at<double>(ly.sumcos) + L + l;
+                t[n++] = w;
+            }
+        }
+        StageDesc h{};
+        h.type = kStLmHead, h.layer = L, h.n_rows = c.vocab, h.n_in = d;
+        h.W = x->at<__nv_bfloat16>(ly.lm_head);
+        h.gain = x->at<__nv_bfloat16>(ly.final_norm);
+        t[n++] = h;
+        (which ? x->n_stages_draft : x->n_stages_full) = n;
+    }
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.stage_tab, tab.data(), tab.size() * sizeof(StageDesc), cudaMemcpyHostToDevice, x->stream));
+    return ASD_OK;
+}
+
 // ---------------------------------------------------------------- one pass of M rows through the decoder
-// tokens (DEVICE) feed rows at positions pos0..pos0+M-1. use_mask selects the draft model D: sublayers in the
-// skip sets are the identity and launch nothing. acc_sim adds the rows' cosines to the prompt sums behind C_l.
+// tokens (DEVICE) feed rows at positions pos0..pos0+M-1. use_mask selects the draft model D. acc_sim adds the
+// rows' cosines to the prompt sums behind C_l. One cooperative launch of the persistent pass kernel.
 static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use_mask, bool acc_sim, bool lm_head,
                     int* dev_argmax_out, bool accept, double* bytes_out) {
     const asd_config& c = x->c;
@@ -281,126 +408,79 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     cudaStream_t s = x->stream;
     if (M < 1 || M > kMaxRows) return fail(x, ASD_ERR_ARG, "row count out of range");
     if ((long long)pos0 + M > c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "pass would exceed max_seq positions");
-    double bytes = 0;
+    PassPlan pl;
+    if (!plan_pass(*x->dev, c, M, &pl)) return fail(x, ASD_ERR_ARG, "decoder shape does not fit the pass kernel's shared-memory plan");
 
     float* cosv = x->at<float>(ly.cosv);
     ASD_CUDA(x, cudaMemsetAsync(cosv, 0xFF, (size_t)2 * std::max(L, 1) * kMaxRows * 4, s));  // NaN = skipped
-    embed_kernel<<<M, 256, 0, s>>>(dev_tokens, x->at<__nv_bfloat16>(ly.embed), x->at<float>(ly.x), d, c.vocab);
-    ASD_CUDA(x, cudaGetLastError());
+
+    unsigned* words = x->at<unsigned>(ly.sync_words);
+    PassParams p{};
+    p.pos0 = pos0;
+    p.tokens = dev_tokens;
+    p.embed = x->at<__nv_bfloat16>(ly.embed);
+    p.d_model = d, p.vocab = c.vocab, p.kv_dim = kvd, p.head_dim = c.head_dim, p.n_heads = c.n_heads;
+    p.n_kv_heads = c.n_kv_heads, p.d_ffn = f;
+    p.eps = c.rms_eps;
+    p.attn_scale = 1.0f / sqrtf((float)c.head_dim);
+    p.rope_cos = x->at<float>(ly.rope_cos);
+    p.rope_sin = x->at<float>(ly.rope_sin);
+    p.x = x->at<float>(ly.x);
+    p.q = x->at<__nv_bfloat16>(ly.q);
+    p.a = x->at<__nv_bfloat16>(ly.a);
+    p.t = x->at<__nv_bfloat16>(ly.t);
+    p.part_acc = x->at<float>(ly.part_acc);
+    p.part_ml = x->at<float>(ly.part_ml);
+    p.attn_counters = x->at<unsigned>(ly.counters) + 64;
+    p.chunk_stride = ly.chunk_stride;
+    p.partials = x->at<float>(ly.partials);
+    p.fin_counter = words + 0;
+    p.grid_bar = words + 16;
+    p.err = reinterpret_cast<int*>(x->at<int>(ly.accept) + 15);
+    p.bar_base = x->bar_base;
+    const int table = use_mask ? 1 : 0;
+    p.stages = x->at<StageDesc>(ly.stage_tab) + (size_t)table * ly.max_stages;
+    const int n_table = use_mask ? x->n_stages_draft : x->n_stages_full;
+    p.n_stages = lm_head ? n_table : n_table - 1;
+    p.row_tokens = accept ? dev_tokens : nullptr;
+    p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
+    p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
+    p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
+    p.acc_sim = acc_sim ? 1 : 0;
+    p.ns = pl.ns, p.attn_groups = pl.attn_groups;
+    p.off_bars = pl.off_bars, p.off_misc = pl.off_misc, p.off_psum = pl.off_psum, p.off_reg_a = pl.off_reg_a;
+    const int grid = x->dev->num_sms;
+    ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));
+    x->bar_base += (uint32_t)p.n_stages * (uint32_t)grid;
     x->stats.kernel_launches += 1;
 
-    GemvParams base{};
-    base.eps = c.rms_eps;
-    base.partials = x->at<float>(ly.partials);
-    base.counter = x->at<unsigned>(ly.counters);  // slot 0; attention uses slots 64..
-    base.pos0 = pos0;
-    base.d_model = d;
-    base.kv_dim = kvd;
-    base.head_dim = c.head_dim;
-    base.rope_cos = x->at<float>(ly.rope_cos);
-    base.rope_sin = x->at<float>(ly.rope_sin);
-
-    auto gemv = [&](int epi, bool norm, GemvParams& p) -> int {
-        int grid, xin;
-        size_t smem;
-        if (!plan_gemv(*x->dev, M, p.n_rows, p.n_in, norm, &grid, &xin, &smem))
-            return fail(x, ASD_ERR_ARG, "matrix shape does not fit the kernel's shared-memory plan");
-        p.x_in_smem = xin;
-        ASD_CUDA(x, launch_gemv(M, epi, norm, p, grid, smem, s));
-        x->stats.kernel_launches += 1;
-        return ASD_OK;
-    };
-
+    // algorithmic bytes of the pass: weights of the stages that ran, plus K/V read by the kept attention sublayers
+    double bytes = 0;
     for (int l = 0; l < L; ++l) {
-        unsigned char* lw = x->layer(l);
-        if (!(use_mask && x->skip_attn[l])) {
-            GemvParams p = base;
-            p.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wqkv);
-            p.n_rows = d + 2 * kvd;
-            p.n_in = d;
-            p.x = x->at<float>(ly.x);
-            p.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_attn_norm);
-            p.q_out = x->at<__nv_bfloat16>(ly.q);
-            p.k_cache = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.kcache + (size_t)l * ly.kv_layer_stride);
-            p.v_cache = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.vcache + (size_t)l * ly.kv_layer_stride);
-            int rc = gemv(kEpiQkv, true, p);
-            if (rc) return rc;
-
-            AttnParams ap{};
-            ap.q = p.q_out;
-            ap.k_cache = p.k_cache;
-            ap.v_cache = p.v_cache;
-            ap.pos0 = pos0;
-            ap.n_heads = c.n_heads;
-            ap.n_kv_heads = c.n_kv_heads;
-            ap.head_dim = c.head_dim;
-            ap.kv_dim = kvd;
-            ap.d_model = d;
-            ap.scale = 1.0f / sqrtf((float)c.head_dim);
-            ap.part_acc = x->at<float>(ly.part_acc);
-            ap.part_ml = x->at<float>(ly.part_ml);
-            ap.counters = x->at<unsigned>(ly.counters) + 64;
-            ap.a_out = x->at<__nv_bfloat16>(ly.a);
-            ap.n_chunks = (pos0 + M - 1) / kAttnChunk + 1;
-            ap.chunk_stride = ly.chunk_stride;
-            ASD_CUDA(x, launch_attn(M, ap, attn_smem_bytes(M, c.head_dim), s));
-            x->stats.kernel_launches += 1;
-
-            GemvParams o = base;
-            o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wo);
-            o.n_rows = d;
-            o.n_in = d;
-            o.x = x->at<__nv_bfloat16>(ly.a);
-            o.out = x->at<float>(ly.x);
-            o.cos_out = cosv + (size_t)(0 * L + l) * kMaxRows;
-            o.sumcos = acc_sim ? x->at<double>(ly.sumcos) + l : nullptr;
-            rc = gemv(kEpiResidual, false, o);
-            if (rc) return rc;
+        if (!(use_mask && x->skip_attn[l]))
             bytes += 2.0 * ((double)(d + 2 * kvd) * d + (double)d * d) + 2.0 * 2.0 * kvd * (double)(pos0 + M);
-        }
-        if (!(use_mask && x->skip_mlp[l])) {
-            GemvParams p = base;
-            p.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wgu);
-            p.n_rows = 2 * f;
-            p.n_in = d;
-            p.x = x->at<float>(ly.x);
-            p.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_mlp_norm);
-            p.out = x->at<__nv_bfloat16>(ly.t);
-            int rc = gemv(kEpiSwiglu, true, p);
-            if (rc) return rc;
-            GemvParams o = base;
-            o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wd);
-            o.n_rows = d;
-            o.n_in = f;
-            o.x = x->at<__nv_bfloat16>(ly.t);
-            o.out = x->at<float>(ly.x);
-            o.cos_out = cosv + (size_t)(1 * L + l) * kMaxRows;
-            o.sumcos = acc_sim ? x->at<double>(ly.sumcos) + L + l : nullptr;
-            rc = gemv(kEpiResidual, false, o);
-            if (rc) return rc;
-            bytes += 2.0 * 3.0 * (double)d * f;
-        }
+        if (!(use_mask && x->skip_mlp[l])) bytes += 2.0 * 3.0 * (double)d * f;
     }
-    x->last_has_logits = false;
-    if (lm_head) {
-        GemvParams p = base;
-        p.W = x->at<__nv_bfloat16>(ly.lm_head);
-        p.n_rows = c.vocab;
-        p.n_in = d;
-        p.x = x->at<float>(ly.x);
-        p.gain = x->at<__nv_bfloat16>(ly.final_norm);
-        p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
-        p.row_tokens = accept ? dev_tokens : nullptr;
-        p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
-        p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
-        int rc = gemv(kEpiArgmax, true, p);
-        if (rc) return rc;
-        x->last_has_logits = x->debug_logits;
-        bytes += 2.0 * (double)c.vocab * d;
-    }
+    if (lm_head) bytes += 2.0 * (double)c.vocab * d;
+    x->last_has_logits = lm_head && x->debug_logits;
     x->last_M = M;
     if (bytes_out) *bytes_out = bytes;
     return ASD_OK;
+}
+
+// the bounded waits of the pass kernel report through a device word; 0 = no error
+static int check_device_error(asd_ctx* x, int word) {
+    if (word == 0) return ASD_OK;
+    static const char* names[] = {"", "a ring slot was never filled", "a ring slot was never released", "the grid barrier never completed"};
+    return fail(x, ASD_ERR_DEVICE_TIMEOUT, std::string("pass kernel gave up waiting: ") + (word >= 1 && word <= 3 ? names[word] : "unknown"));
+}
+
+// copy n ints from the device and the pass kernel's error word to the pinned buffer, wait, and check the word
+static int read_back(asd_ctx* x, const int* dev_src, int n) {
+    if (n > 0) ASD_CUDA(x, cudaMemcpyAsync(x->pinned, dev_src, (size_t)n * 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned + 32, x->at<int>(x->lay.accept) + 15, 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    return check_device_error(x, x->pinned[32]);
 }
 
 // ---------------------------------------------------------------- Algorithm 1
@@ -445,10 +525,12 @@ extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t byt
     };
     cudaError_t e = device_info(&x->dev);
     if (e != cudaSuccess) return bail(e);
-    const size_t worst_attn = attn_smem_bytes(kMaxRows, cfg->head_dim);
-    if (worst_attn > (size_t)x->dev->max_smem) {
-        delete x;
-        return ASD_ERR_ARG;
+    {
+        PassPlan pl;
+        if (!plan_pass(*x->dev, *cfg, kMaxRows, &pl) || !plan_pass(*x->dev, *cfg, 1, &pl)) {
+            delete x;
+            return ASD_ERR_ARG;
+        }
     }
     if ((e = cudaHostAlloc((void**)&x->pinned, 4096, cudaHostAllocDefault)) != cudaSuccess) return bail(e);
     // rotary table: angle(p, j) = p * theta^(-2j/head_dim), evaluated in double, stored as float
@@ -469,6 +551,13 @@ extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t byt
     }
     // zero everything behind the weights: KV cache, scratch, counters
     if ((e = cudaMemsetAsync(x->ws + lay.kcache, 0, lay.total - lay.kcache, x->stream)) != cudaSuccess) return bail(e);
+    if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e);
+    if (make_tensor_maps(x) != ASD_OK || build_stage_tables(x) != ASD_OK) {
+        fprintf(stderr, "asd_create: %s\n", x->err.c_str());
+        cudaFreeHost(x->pinned);
+        delete x;
+        return ASD_ERR_CUDA;
+    }
     if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e);
     *out = x;
     return ASD_OK;
@@ -553,7 +642,8 @@ extern "C" int asd_reset(asd_ctx* x) {
     x->spans.clear();
     x->events_used = 0;
     ASD_CUDA(x, cudaMemsetAsync(x->ws + x->lay.sumcos, 0, (size_t)2 * std::max(x->c.n_layers, 1) * 8, x->stream));
-    return ASD_OK;
+    ASD_CUDA(x, cudaMemsetAsync(x->at<int>(x->lay.accept), 0, 64 * 4, x->stream));
+    return build_stage_tables(x);
 }
 
 // ---------------------------------------------------------------- prefill (Section 3.2)
@@ -580,8 +670,7 @@ static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int3
     x->n_sim_rows += n;
     x->stats.prefill_rows += n;
     if (first_token) {
-        ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax) + (last_rows - 1), 4, cudaMemcpyDeviceToHost, x->stream));
-        ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+        if ((rc = read_back(x, x->at<int>(x->lay.argmax) + (last_rows - 1), 1))) return rc;
         *first_token = x->pinned[0];
         if (resolve && (rc = resolve_spans(x))) return rc;
     }
@@ -634,7 +723,7 @@ extern "C" int asd_set_skip_mask(asd_ctx* x, const uint8_t* skip_attn, const uin
         x->skip_mlp[l] = skip_mlp[l] ? 1 : 0;
     }
     x->draft_cursor = x->n_committed;
-    return ASD_OK;
+    return build_stage_tables(x);
 }
 
 extern "C" int asd_admg_update(asd_ctx* x, const asd_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp) {
@@ -646,7 +735,8 @@ extern "C" int asd_admg_update(asd_ctx* x, const asd_admg_params* p, uint8_t* sk
     std::vector<uint8_t> a(std::max(L, 1)), b(std::max(L, 1));
     rc = asd_admg(C.data(), L, p, a.data(), b.data());
     if (rc) return fail(x, rc, "bad ADMG parameters");
-    asd_set_skip_mask(x, a.data(), b.data());
+    rc = asd_set_skip_mask(x, a.data(), b.data());
+    if (rc) return rc;
     if (skip_attn) memcpy(skip_attn, a.data(), L);
     if (skip_mlp) memcpy(skip_mlp, b.data(), L);
     return ASD_OK;
@@ -679,8 +769,7 @@ extern "C" int asd_decode_step(asd_ctx* x, int32_t token_in, int32_t* token_out)
     if (rc) return rc;
     rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, x->at<int>(x->lay.tok_in), false, nullptr, false);
     if (rc) return rc;
-    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax), 4, cudaMemcpyDeviceToHost, x->stream));
-    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    if ((rc = read_back(x, x->at<int>(x->lay.argmax), 1))) return rc;
     x->n_committed += 1;
     x->draft_cursor = x->n_committed;
     if (token_out) *token_out = x->pinned[0];
@@ -695,8 +784,7 @@ extern "C" int asd_draft_step(asd_ctx* x, int32_t token_in, int32_t* token_out) 
     if (rc) return rc;
     rc = timed_pass(x, SPAN_DRAFT, 1, x->draft_cursor, x->at<int>(x->lay.tok_in), true, nullptr, false);
     if (rc) return rc;
-    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.argmax), 4, cudaMemcpyDeviceToHost, x->stream));
-    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    if ((rc = read_back(x, x->at<int>(x->lay.argmax), 1))) return rc;
     x->draft_cursor += 1;
     if (token_out) *token_out = x->pinned[0];
     return resolve_spans(x);
@@ -711,8 +799,7 @@ extern "C" int asd_verify(asd_ctx* x, const int32_t* tokens, int32_t k, int32_t*
     if (rc) return rc;
     rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, x->at<int>(x->lay.draft_toks), false, nullptr, true);
     if (rc) return rc;
-    ASD_CUDA(x, cudaMemcpyAsync(x->pinned, x->at<int>(x->lay.accept), (size_t)(k + 2) * 4, cudaMemcpyDeviceToHost, x->stream));
-    ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    if ((rc = read_back(x, x->at<int>(x->lay.accept), k + 2))) return rc;
     const int a = x->pinned[0];
     if (n_accepted) *n_accepted = a;
     if (out_tokens)
@@ -764,8 +851,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             if (rc) return rc;
             x->n_committed += 1;
             if (need_host_token) {
-                ASD_CUDA(x, cudaMemcpyAsync(x->pinned, dev_out + produced, 4, cudaMemcpyDeviceToHost, s));
-                ASD_CUDA(x, cudaStreamSynchronize(s));
+                if ((rc = read_back(x, dev_out + produced, 1))) return rc;
                 stop = x->pinned[0] == gp->eos_id;
             }
             ++produced;
@@ -784,8 +870,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             }
             rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, draft, false, nullptr, true);
             if (rc) return rc;
-            ASD_CUDA(x, cudaMemcpyAsync(x->pinned, accept, (size_t)(k + 2) * 4, cudaMemcpyDeviceToHost, s));
-            ASD_CUDA(x, cudaStreamSynchronize(s));
+            if ((rc = read_back(x, accept, k + 2))) return rc;
             const int a = x->pinned[0];
             int emit = a + 1;
             if (gp->eos_id >= 0)
@@ -807,7 +892,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
         }
     }
     if ((rc = new_event(x, &ev_end))) return rc;
-    ASD_CUDA(x, cudaStreamSynchronize(s));
+    if ((rc = read_back(x, nullptr, 0))) return rc;
     float ms = 0.f;
     ASD_CUDA(x, cudaEventElapsedTime(&ms, x->events[ev_begin], x->events[ev_end]));
     x->stats.ms_total = ms;

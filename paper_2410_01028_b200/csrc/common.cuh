@@ -10,7 +10,6 @@ constexpr int kMaxRows = 9;        // rows per pass: max draft length 8, plus th
 constexpr int kGemvThreads = 512;  // 16 warps per CTA, one CTA per SM
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kSeg = 1024;         // elements of the reduction dimension per warp work item
-constexpr int kAttnThreads = 128;
 constexpr int kAttnChunk = 128;    // keys per attention work item; chunks are aligned to absolute positions
 
 enum Epilogue : int { kEpiPlain = 0, kEpiSwiglu = 1, kEpiResidual = 2, kEpiQkv = 3, kEpiArgmax = 4 };
@@ -40,22 +39,12 @@ struct GemvParams {
     float* logits_out;      // [M, n_rows] or null
 };
 
-struct AttnParams {
-    const __nv_bfloat16* q;  // [M, d_model]
-    const __nv_bfloat16 *k_cache, *v_cache;  // this layer: [max_seq, kv_dim]
-    int pos0, n_heads, n_kv_heads, head_dim, kv_dim, d_model;
-    float scale;
-    float* part_acc;  // [n_heads][chunk_stride][kMaxRows][head_dim]
-    float* part_ml;   // [n_heads][chunk_stride][kMaxRows][2]
-    unsigned* counters;  // [n_kv_heads], zero before launch, reset by the merging CTA
-    __nv_bfloat16* a_out;  // [M, d_model]
-    int n_chunks, chunk_stride;
-};
+struct PassParams;
 
 // launchers, one translation unit per row count (inst.cu compiled with -DASD_M=1..9)
 #define ASD_DECLARE_LAUNCHERS(M)                                                                                 \
     cudaError_t launch_gemv_m##M(int epi, bool norm, const GemvParams& p, int grid, size_t smem, cudaStream_t s); \
-    cudaError_t launch_attn_m##M(const AttnParams& p, size_t smem, cudaStream_t s);                              \
+    cudaError_t launch_pass_m##M(const PassParams& p, int grid, size_t smem, cudaStream_t s);                    \
     cudaError_t configure_m##M(int max_smem);
 ASD_DECLARE_LAUNCHERS(1)
 ASD_DECLARE_LAUNCHERS(2)
@@ -68,7 +57,6 @@ ASD_DECLARE_LAUNCHERS(8)
 ASD_DECLARE_LAUNCHERS(9)
 
 size_t gemv_smem_bytes(int M, int n_rows, int n_in, int grid, bool x_in_smem);
-size_t attn_smem_bytes(int M, int head_dim);
 
 // ---------------------------------------------------------------- device helpers
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }

@@ -1,6 +1,6 @@
 // Instantiations of the row-count-templated kernels; compiled once per ASD_M in 1..9.
-#include "attn.cuh"
 #include "gemv.cuh"
+#include "pass.cuh"
 
 #ifndef ASD_M
 #error "compile with -DASD_M=<rows>"
@@ -22,16 +22,14 @@ cudaError_t ASD_CAT(launch_gemv_m, ASD_M)(int epi, bool norm, const GemvParams& 
         case kEpiPlain: return norm ? launch_one<kEpiPlain, true>(p, grid, smem, s) : launch_one<kEpiPlain, false>(p, grid, smem, s);
         case kEpiSwiglu: return norm ? launch_one<kEpiSwiglu, true>(p, grid, smem, s) : launch_one<kEpiSwiglu, false>(p, grid, smem, s);
         case kEpiResidual: return norm ? launch_one<kEpiResidual, true>(p, grid, smem, s) : launch_one<kEpiResidual, false>(p, grid, smem, s);
-        case kEpiQkv: return norm ? launch_one<kEpiQkv, true>(p, grid, smem, s) : cudaErrorInvalidValue;
-        case kEpiArgmax: return norm ? launch_one<kEpiArgmax, true>(p, grid, smem, s) : cudaErrorInvalidValue;
     }
     return cudaErrorInvalidValue;
 }
 
-cudaError_t ASD_CAT(launch_attn_m, ASD_M)(const AttnParams& p, size_t smem, cudaStream_t s) {
-    dim3 grid(p.n_chunks, p.n_kv_heads);
-    attn_kernel<ASD_M><<<grid, kAttnThreads, smem, s>>>(p);
-    return cudaGetLastError();
+cudaError_t ASD_CAT(launch_pass_m, ASD_M)(const PassParams& p, int grid, size_t smem, cudaStream_t s) {
+    void* args[] = {const_cast<PassParams*>(&p)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&pass_kernel<ASD_M>), dim3(grid), dim3(kPassThreads),
+                                       args, smem, s);
 }
 
 // opt every instantiation in to large dynamic shared memory
@@ -46,9 +44,7 @@ cudaError_t ASD_CAT(configure_m, ASD_M)(int max_smem) {
     ASD_SET((gemv_kernel<ASD_M, kEpiSwiglu, false>))
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, true>))
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, false>))
-    ASD_SET((gemv_kernel<ASD_M, kEpiQkv, true>))
-    ASD_SET((gemv_kernel<ASD_M, kEpiArgmax, true>))
-    ASD_SET((attn_kernel<ASD_M>))
+    ASD_SET((pass_kernel<ASD_M>))
 #undef ASD_SET
     return cudaSuccess;
 }

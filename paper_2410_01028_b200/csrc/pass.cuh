@@ -1,0 +1,831 @@
+// One persistent kernel per decoder pass (decode, draft, verify, prefill chunk).
+//
+// Why: at batch 1 a pass is ~200 dependent sublayer stages of 5-30 us each. Launching them one by one leaves
+// HBM idle at every boundary (launch latency, RMSNorm prologue, drain). Weights, however, never depend on
+// activations. So here one CTA per SM stays resident for the whole pass (cooperative launch) and is split in
+// two roles:
+//   * a producer thread walks this CTA's share of EVERY stage's weights (and of the old part of the KV cache)
+//     in order and keeps a shared-memory ring of 4 KB slots full with TMA copies (cp.async.bulk, and
+//     cp.async.bulk.tensor with 128-byte swizzle for K/V boxes). It never waits for activations, so HBM keeps
+//     streaming across stage boundaries, grid barriers and prologues;
+//   * 15 consumer warps wait for the previous stage of all CTAs (a grid barrier on a monotonically increasing
+//     counter, bounded spin), stage the activations in shared memory (RMSNorm fused), multiply the ring slots
+//     with packed fp32 FMAs, and run the epilogue: RoPE + KV append, SwiGLU, residual add + cosine
+//     similarity (summand of C_l, Section 3.2), LM-head argmax + greedy acceptance (Section 1).
+// Sublayers in the skip mask (the draft model D, Algorithm 1) simply do not appear in the stage table: no
+// weights are streamed and no K/V is touched for them.
+//
+// Reduction order is fixed and independent of the row count M: per (weight row, activation row) a lane adds
+// the even and the odd elements of its 16-byte chunks of a 1024-element segment in order, the two halves are
+// added, lanes are combined by an xor butterfly, segments are added in ascending order. Attention chunks are
+// aligned to absolute positions and merged in order. Row m of a (k+1)-row verify pass is therefore
+// bit-identical to a 1-row decode pass at the same position, so speculative output equals autoregressive
+// output bit for bit.
+#pragma once
+#include <limits.h>
+
+#include "common.cuh"
+#include "ring.cuh"
+
+namespace asd {
+
+constexpr int kPassConsumerWarps = 15;
+constexpr int kPassConsumers = kPassConsumerWarps * 32;
+constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
+constexpr int kWsegMax = 4;                         // at most 4 segments of the reduction dimension per activation window
+constexpr int kXsBudget = 40960;                    // bytes of shared memory for the activation window / attention scratch
+
+enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead };
+
+struct StageDesc {
+    int type, layer;
+    int n_rows, n_in;
+    const __nv_bfloat16* W;
+    const __nv_bfloat16* gain;
+    __nv_bfloat16 *k_cache, *v_cache;   // this layer's cache [max_seq, kv_dim]
+    const CUtensorMap *tm_k, *tm_v;     // tensor maps over the same
+    float* cos_out;                     // [kMaxRows] cosine of this sublayer, per row
+    double* sumcos;                     // running sum over prompt rows
+};
+
+struct PassParams {
+    int pos0;
+    const int* tokens;
+    const __nv_bfloat16* embed;
+    int d_model, vocab, kv_dim, head_dim, n_heads, n_kv_heads, d_ffn;
+    float eps, attn_scale;
+    const float *rope_cos, *rope_sin;
+    float* x;
+    __nv_bfloat16 *q, *a, *t;
+    float *part_acc, *part_ml;
+    unsigned* attn_counters;
+    int chunk_stride;
+    float* partials;
+    unsigned* fin_counter;
+    unsigned* grid_bar;
+    unsigned bar_base;
+    int* err;
+    const StageDesc* stages;
+    int n_stages;
+    const int* row_tokens;
+    int* argmax_out;
+    int* accept_out;
+    float* logits_out;
+    int acc_sim;
+    // shared-memory plan (bytes from the 1024-aligned base)
+    int ns;            // ring slots
+    int attn_groups;   // 1 or 2 groups of 4 warps work on attention items
+    int off_bars, off_misc, off_psum, off_reg_a;
+};
+
+__host__ __device__ inline int pass_wseg(int M) {
+    int w = kXsBudget / (M * 2048);
+    return w < 1 ? 1 : (w > kWsegMax ? kWsegMax : w);
+}
+
+struct PassSmem {
+    unsigned char* ring;
+    uint64_t *full, *empty;
+    float* red;   // [16][kMaxRows*4]
+    int* flag;    // [8]
+    float* psum;
+    unsigned char* reg_a;
+};
+
+__device__ __forceinline__ void stage_pair_rows(int type, const PassParams& p, int pair, int& ra, int& rb) {
+    if (type == kStQkv) {
+        const int half = p.head_dim >> 1;
+        const int nq = p.d_model >> 1, nk = p.kv_dim >> 1;
+        int base, pp;
+        if (pair < nq) {
+            base = 0;
+            pp = pair;
+        } else if (pair < nq + nk) {
+            base = p.d_model;
+            pp = pair - nq;
+        } else {
+            base = p.d_model + p.kv_dim;
+            pp = pair - nq - nk;
+        }
+        const int head = pp / half, j = pp - head * half;
+        ra = base + head * p.head_dim + j;
+        rb = ra + half;
+    } else {
+        ra = 2 * pair;
+        rb = 2 * pair + 1;
+    }
+}
+
+__device__ __forceinline__ void cta_pairs(int n_rows, int& pair0, int& np) {
+    const int n_pairs = (n_rows + 1) >> 1;
+    pair0 = (int)((long long)blockIdx.x * n_pairs / gridDim.x);
+    const int pair1 = (int)((long long)(blockIdx.x + 1) * n_pairs / gridDim.x);
+    np = pair1 - pair0;
+}
+
+__device__ __forceinline__ int attn_local_items(const PassParams& p, int M, int& n_chunks) {
+    n_chunks = (p.pos0 + M - 1) / kAttnChunk + 1;
+    const int total = p.n_kv_heads * n_chunks;
+    return ((int)blockIdx.x < total) ? (total - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+}
+
+// ============================================================================================ producer
+template <int M>
+__device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
+    volatile int* err = p.err;
+    uint32_t gi = 0;
+    const int ns = p.ns;
+    auto acquire = [&](uint32_t g) -> int {   // wait until the slot of ring item g may be overwritten
+        const int slot = g % ns;
+        const uint32_t gen = g / ns;
+        if (gen > 0) mbar_wait(&sm.empty[slot], (gen - 1) & 1, err, kErrEmptyWait);
+        return slot;
+    };
+    for (int s = 0; s < p.n_stages; ++s) {
+        const StageDesc st = p.stages[s];
+        if (st.type == kStEmbed) continue;
+        if (st.type == kStAttn) {
+            int n_chunks;
+            const int n_local = attn_local_items(p, M, n_chunks);
+            const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
+            const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
+            const uint32_t box_bytes = 32u * box_cols * 2u;
+            for (int j = 0; j < n_local; ++j) {
+                const int idx = blockIdx.x + j * gridDim.x;
+                const int kvh = idx / n_chunks, chunk = idx - kvh * n_chunks;
+                for (int which = 0; which < 2; ++which) {
+                    const CUtensorMap* tm = which ? st.tm_v : st.tm_k;
+                    for (int rg = 0; rg < 4; ++rg)
+                        for (int hb = 0; hb < nhb; ++hb) {
+                            const int slot = acquire(gi);
+                            mbar_expect_tx(&sm.full[slot], box_bytes);
+                            tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, tm, kvh * p.head_dim + hb * 64,
+                                        chunk * kAttnChunk + rg * 32, &sm.full[slot]);
+                            ++gi;
+                        }
+                }
+            }
+            continue;
+        }
+        // GEMV stage: windows of segments, pairs inside a window, segments of a pair consecutively
+        int pair0, np;
+        cta_pairs(st.n_rows, pair0, np);
+        const int n_seg = (st.n_in + kSeg - 1) / kSeg;
+        const int wseg = pass_wseg(M);
+        for (int w0 = 0; w0 < n_seg; w0 += wseg) {
+            const int ws = min(wseg, n_seg - w0);
+            for (int pl = 0; pl < np; ++pl) {
+                int ra, rb;
+                stage_pair_rows(st.type, p, pair0 + pl, ra, rb);
+                rb = min(rb, st.n_rows - 1);
+                for (int sg = w0; sg < w0 + ws; ++sg) {
+                    const int k0 = sg * kSeg;
+                    const uint32_t bytes = (uint32_t)min(kSeg, st.n_in - k0) * 2u;
+                    const int slot = acquire(gi);
+                    unsigned char* dst = sm.ring + (size_t)slot * kSlotBytes;
+                    mbar_expect_tx(&sm.full[slot], 2u * bytes);
+                    tma_load_1d(dst, st.W + (size_t)ra * st.n_in + k0, bytes, &sm.full[slot]);
+                    tma_load_1d(dst + kSlotBytes / 2, st.W + (size_t)rb * st.n_in + k0, bytes, &sm.full[slot]);
+                    ++gi;
+                }
+            }
+        }
+    }
+    // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let them land
+    // (bounded) before the CTA exits.
+    if (*err != kErrNone) {
+        const uint32_t n_wait = gi < (uint32_t)ns ? gi : (uint32_t)ns;
+        for (uint32_t k = 0; k < n_wait; ++k) {
+            const uint32_t g = gi - 1 - k;
+            const int slot = g % ns;
+            const uint32_t par = (g / ns) & 1;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(&sm.full[slot], par) && clock64() - t0 < 20000000LL) {
+            }
+        }
+    }
+}
+
+// ============================================================================================ grid barrier
+__device__ __forceinline__ void consumers_sync() { bar_sync(1, kPassConsumers); }
+
+__device__ __forceinline__ void grid_arrive(const PassParams& p) {
+    consumers_sync();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(p.grid_bar, 1u);
+    }
+}
+__device__ __forceinline__ void grid_wait(const PassParams& p, unsigned target) {
+    if (threadIdx.x == 0) {
+        volatile int* err = p.err;
+        const long long t0 = clock64();
+        while ((int)(ld_acquire_gpu(p.grid_bar) - target) < 0) {
+            if (*err != kErrNone) break;
+            if (clock64() - t0 > kWaitCycles) {
+                atomicCAS(p.err, kErrNone, kErrGridWait);
+                break;
+            }
+        }
+    }
+    consumers_sync();
+}
+
+// consumers only: true in every thread of the last CTA to arrive on a global counter
+__device__ __forceinline__ bool last_cta_consumers(unsigned* counter, int* flag_smem) {
+    __threadfence();
+    consumers_sync();
+    if (threadIdx.x == 0) {
+        const unsigned t = atomicAdd(counter, 1u);
+        *flag_smem = (t == gridDim.x - 1) ? 1 : 0;
+    }
+    consumers_sync();
+    const bool last = *flag_smem != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+// ============================================================================================ GEMV stage
+template <int M>
+__device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int type = st.type;
+    const bool norm = (type == kStQkv || type == kStGateUp || type == kStLmHead);
+    const int n_in = st.n_in, n_rows = st.n_rows;
+    int pair0, np;
+    cta_pairs(n_rows, pair0, np);
+    const int n_seg = (n_in + kSeg - 1) / kSeg;
+    const int wseg = pass_wseg(M);
+    const int xstride = wseg * kSeg;
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
+    float* red = sm.red;
+    float* psum = sm.psum;
+    volatile int* err = p.err;
+
+    const float* xf = p.x;
+    const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
+
+    // ---- RMSNorm statistics (same arithmetic for every row count)
+    float inv[M];
+    if (norm) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float s = 0.f;
+            for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
+                s = fmaf(v.x, v.x, s);
+                s = fmaf(v.y, v.y, s);
+                s = fmaf(v.z, v.z, s);
+                s = fmaf(v.w, v.w, s);
+            }
+            s = warp_sum(s);
+            if (lane == 0) red[warp * (kMaxRows * 4) + m] = s;
+        }
+        consumers_sync();
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < kPassConsumerWarps; ++w) s += red[w * (kMaxRows * 4) + m];
+            inv[m] = 1.0f / sqrtf(s / (float)n_in + p.eps);
+        }
+    }
+    for (int i = tid; i < np * 2 * M; i += kPassConsumers) psum[i] = 0.f;
+
+    // ---- stream the slab window by window
+    for (int w0 = 0; w0 < n_seg; w0 += wseg) {
+        const int ws = min(wseg, n_seg - w0);
+        const int k0 = w0 * kSeg;
+        const int klen = min(n_in - k0, ws * kSeg);
+        consumers_sync();  // previous window fully consumed; psum zeroed; red free
+        if (norm) {
+            for (int i = tid * 4; i < klen; i += kPassConsumers * 4) {
+                const uint2 gv = *reinterpret_cast<const uint2*>(st.gain + k0 + i);
+                const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + k0 + i));
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv[m] * g0, v.y * inv[m] * g1);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv[m] * g2, v.w * inv[m] * g3);
+                    uint2 o;
+                    o.x = *reinterpret_cast<uint32_t*>(&lo);
+                    o.y = *reinterpret_cast<uint32_t*>(&hi);
+                    *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                }
+            }
+        } else {
+            for (int i = tid * 8; i < klen; i += kPassConsumers * 8) {
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+                    *reinterpret_cast<uint4*>(xs + (size_t)m * xstride + i) =
+                        __ldcg(reinterpret_cast<const uint4*>(xb + (size_t)m * n_in + k0 + i));
+            }
+        }
+        consumers_sync();
+
+        for (int pl = warp; pl < np; pl += kPassConsumerWarps) {
+            float sa[M], sb[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                sa[m] = psum[(pl * 2 + 0) * M + m];
+                sb[m] = psum[(pl * 2 + 1) * M + m];
+            }
+            for (int sg = 0; sg < ws; ++sg) {
+                const uint32_t g = gi + (uint32_t)(np * w0 + pl * ws + sg);
+                const int slot = g % p.ns;
+                mbar_wait(&sm.full[slot], (g / p.ns) & 1, err, kErrFullWait);
+                const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes;
+                const int seglen = min(kSeg, n_in - (w0 + sg) * kSeg);
+                unsigned long long acc_a[M], acc_b[M];
+#pragma unroll
+                for (int m = 0; m < M; ++m) acc_a[m] = acc_b[m] = 0ull;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int kk = i * 256 + lane * 8;
+                    if (kk < seglen) {
+                        const uint4 wa = *reinterpret_cast<const uint4*>(sl + kk * 2);
+                        const uint4 wb = *reinterpret_cast<const uint4*>(sl + kSlotBytes / 2 + kk * 2);
+                        const unsigned long long a0 = bf2_to_f2(wa.x), a1 = bf2_to_f2(wa.y), a2 = bf2_to_f2(wa.z), a3 = bf2_to_f2(wa.w);
+                        const unsigned long long b0 = bf2_to_f2(wb.x), b1 = bf2_to_f2(wb.y), b2 = bf2_to_f2(wb.z), b3 = bf2_to_f2(wb.w);
+#pragma unroll
+                        for (int m = 0; m < M; ++m) {
+                            const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)m * xstride + sg * kSeg + kk);
+                            const unsigned long long x0 = bf2_to_f2(xv.x), x1 = bf2_to_f2(xv.y), x2 = bf2_to_f2(xv.z), x3 = bf2_to_f2(xv.w);
+                            acc_a[m] = ffma2(a0, x0, acc_a[m]);
+                            acc_a[m] = ffma2(a1, x1, acc_a[m]);
+                            acc_a[m] = ffma2(a2, x2, acc_a[m]);
+                            acc_a[m] = ffma2(a3, x3, acc_a[m]);
+                            acc_b[m] = ffma2(b0, x0, acc_b[m]);
+                            acc_b[m] = ffma2(b1, x1, acc_b[m]);
+                            acc_b[m] = ffma2(b2, x2, acc_b[m]);
+                            acc_b[m] = ffma2(b3, x3, acc_b[m]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[slot]);
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    float e, o;
+                    unpack2(acc_a[m], e, o);
+                    sa[m] += warp_sum(e + o);
+                    unpack2(acc_b[m], e, o);
+                    sb[m] += warp_sum(e + o);
+                }
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    psum[(pl * 2 + 0) * M + m] = sa[m];
+                    psum[(pl * 2 + 1) * M + m] = sb[m];
+                }
+            }
+        }
+    }
+    gi += (uint32_t)(np * n_seg);
+    consumers_sync();
+
+    // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
+    float s_loc[M][3];
+    float best_v[M];
+    int best_i[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        s_loc[m][0] = s_loc[m][1] = s_loc[m][2] = 0.f;
+        best_v[m] = -INFINITY;
+        best_i[m] = INT_MAX;
+    }
+    for (int pl = tid; pl < np; pl += kPassConsumers) {
+        int ra, rb;
+        stage_pair_rows(type, p, pair0 + pl, ra, rb);
+        const bool has_b = rb < n_rows;
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float va = psum[(pl * 2 + 0) * M + m], vb = psum[(pl * 2 + 1) * M + m];
+            if (type == kStGateUp) {
+                const float t = va / (1.0f + expf(-va)) * vb;
+                p.t[(size_t)m * (n_rows >> 1) + (pair0 + pl)] = __float2bfloat16_rn(t);
+            } else if (type == kStOproj || type == kStDown) {
+                float* out = p.x;
+                {
+                    const float x0 = __ldcg(out + (size_t)m * n_rows + ra);
+                    const float y0 = x0 + va;
+                    out[(size_t)m * n_rows + ra] = y0;
+                    s_loc[m][0] = fmaf(x0, y0, s_loc[m][0]);
+                    s_loc[m][1] = fmaf(x0, x0, s_loc[m][1]);
+                    s_loc[m][2] = fmaf(y0, y0, s_loc[m][2]);
+                }
+                if (has_b) {
+                    const float x1 = __ldcg(out + (size_t)m * n_rows + rb);
+                    const float y1 = x1 + vb;
+                    out[(size_t)m * n_rows + rb] = y1;
+                    s_loc[m][0] = fmaf(x1, y1, s_loc[m][0]);
+                    s_loc[m][1] = fmaf(x1, x1, s_loc[m][1]);
+                    s_loc[m][2] = fmaf(y1, y1, s_loc[m][2]);
+                }
+            } else if (type == kStQkv) {
+                const int pos = p.pos0 + m;
+                const int half = p.head_dim >> 1;
+                if (ra < p.d_model + p.kv_dim) {  // q or k: rotate the pair (j, j + head_dim/2) by pos * theta_j
+                    const int j = ra % p.head_dim;
+                    const float c = p.rope_cos[(size_t)pos * half + j], s = p.rope_sin[(size_t)pos * half + j];
+                    const float r0 = va * c - vb * s;
+                    const float r1 = vb * c + va * s;
+                    va = r0;
+                    vb = r1;
+                }
+                const __nv_bfloat16 ha = __float2bfloat16_rn(va), hb = __float2bfloat16_rn(vb);
+                if (ra < p.d_model) {
+                    p.q[(size_t)m * p.d_model + ra] = ha;
+                    p.q[(size_t)m * p.d_model + rb] = hb;
+                } else if (ra < p.d_model + p.kv_dim) {
+                    st.k_cache[(size_t)pos * p.kv_dim + (ra - p.d_model)] = ha;
+                    st.k_cache[(size_t)pos * p.kv_dim + (rb - p.d_model)] = hb;
+                } else {
+                    st.v_cache[(size_t)pos * p.kv_dim + (ra - p.d_model - p.kv_dim)] = ha;
+                    st.v_cache[(size_t)pos * p.kv_dim + (rb - p.d_model - p.kv_dim)] = hb;
+                }
+            } else {  // LM head
+                if (p.logits_out) {
+                    p.logits_out[(size_t)m * n_rows + ra] = va;
+                    if (has_b) p.logits_out[(size_t)m * n_rows + rb] = vb;
+                }
+                if (va > best_v[m]) {
+                    best_v[m] = va;
+                    best_i[m] = ra;
+                }
+                if (has_b && vb > best_v[m]) {
+                    best_v[m] = vb;
+                    best_i[m] = rb;
+                }
+            }
+        }
+    }
+
+    if (type == kStOproj || type == kStDown) {
+        // cosine similarity of the hidden state before and after this sublayer: warp-shuffle partial dot and
+        // norm products, one block-level finish, per-CTA partials combined by the last CTA to arrive
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                const float v = warp_sum(s_loc[m][j]);
+                if (lane == 0) red[warp * (kMaxRows * 4) + m * 4 + j] = v;
+            }
+        consumers_sync();
+        if (tid < M * 3) {
+            const int m = tid / 3, j = tid - m * 3;
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < kPassConsumerWarps; ++w) tot += red[w * (kMaxRows * 4) + m * 4 + j];
+            p.partials[((size_t)blockIdx.x * kMaxRows + m) * 4 + j] = tot;
+        }
+        if (last_cta_consumers(p.fin_counter, sm.flag)) {
+            if (tid < M) {
+                double sxy = 0, sxx = 0, syy = 0;
+                for (unsigned b = 0; b < gridDim.x; ++b) {
+                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
+                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1);
+                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 2);
+                }
+                const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
+                st.cos_out[tid] = (float)c;
+                red[tid] = (float)c;
+            }
+            consumers_sync();
+            if (tid == 0) {
+                if (p.acc_sim && st.sumcos) {
+                    double acc = *st.sumcos;
+                    for (int m = 0; m < M; ++m) acc += (double)red[m];
+                    *st.sumcos = acc;
+                }
+                *p.fin_counter = 0u;
+            }
+        }
+    } else if (type == kStLmHead) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            float v = best_v[m];
+            int i = best_i[m];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+                if (ov > v || (ov == v && oi < i)) {
+                    v = ov;
+                    i = oi;
+                }
+            }
+            if (lane == 0) {
+                red[warp * (kMaxRows * 4) + m * 4 + 0] = v;
+                red[warp * (kMaxRows * 4) + m * 4 + 1] = __int_as_float(i);
+            }
+        }
+        consumers_sync();
+        if (tid < M) {
+            float v = -INFINITY;
+            int i = INT_MAX;
+            for (int w = 0; w < kPassConsumerWarps; ++w) {
+                const float ov = red[w * (kMaxRows * 4) + tid * 4 + 0];
+                const int oi = __float_as_int(red[w * (kMaxRows * 4) + tid * 4 + 1]);
+                if (ov > v || (ov == v && oi < i)) {
+                    v = ov;
+                    i = oi;
+                }
+            }
+            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 0] = v;
+            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 1] = __int_as_float(i);
+        }
+        if (last_cta_consumers(p.fin_counter, sm.flag)) {
+            int* g = reinterpret_cast<int*>(red);
+            if (tid < M) {
+                float v = -INFINITY;
+                int i = INT_MAX;
+                for (unsigned b = 0; b < gridDim.x; ++b) {
+                    const float ov = __ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
+                    const int oi = __float_as_int(__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1));
+                    if (ov > v || (ov == v && oi < i)) {
+                        v = ov;
+                        i = oi;
+                    }
+                }
+                if (i == INT_MAX) i = 0;
+                p.argmax_out[tid] = i;
+                g[tid] = i;
+            }
+            consumers_sync();
+            if (tid == 0) {
+                if (p.accept_out && p.row_tokens) {
+                    // greedy verification (Section 1): drafted token j+1 is accepted while it equals M's argmax of row j
+                    int a = 0;
+                    while (a < M - 1 && p.row_tokens[a + 1] == g[a]) ++a;
+                    p.accept_out[0] = a;
+                    for (int j = 0; j < a; ++j) p.accept_out[1 + j] = p.row_tokens[j + 1];
+                    p.accept_out[1 + a] = g[a];
+                }
+                *p.fin_counter = 0u;
+            }
+        }
+    }
+}
+
+// ============================================================================================ attention stage
+// Byte offset of (key row r of the 128-key tile, 16-byte chunk c of the head) inside the tile's ring slots.
+struct TileAddr {
+    int nhb, row_bytes, swz;
+    __device__ __forceinline__ void locate(int r, int c, int& slot_in_tile, int& off) const {
+        const int rg = r >> 5, rr = r & 31;
+        const int hb = (nhb > 1) ? (c >> 3) : 0;
+        const int cc = (nhb > 1) ? (c & 7) : c;
+        slot_in_tile = rg * nhb + hb;
+        off = rr * row_bytes + ((swz ? (cc ^ (rr & 7)) : cc) << 4);
+    }
+};
+
+template <int M>
+__device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int hd = p.head_dim;
+    const int nhb = hd > 64 ? hd / 64 : 1;
+    const int box_cols = hd > 64 ? 64 : hd;
+    const int tile_slots = 4 * nhb;
+    int n_chunks;
+    const int n_local = attn_local_items(p, M, n_chunks);
+    const uint32_t gi0 = gi;
+    gi += (uint32_t)(n_local * 2 * tile_slots);
+    const int grp = warp >> 2;
+    if (grp >= p.attn_groups) return;
+
+    volatile int* err = p.err;
+    const int gt = tid & 127, glane = gt & 31, gwarp = gt >> 5;
+    const int bar_id = 2 + grp;
+    const int group = p.n_heads / p.n_kv_heads;
+    const int vec_per_row = hd / 8;
+    TileAddr ta{nhb, box_cols * 2, (box_cols * 2 == 128) ? 1 : 0};
+
+    // per-group scratch in region A
+    const size_t scratch_bytes = ((size_t)M * hd * 4 + (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16 + 15) & ~(size_t)15;
+    unsigned char* base = sm.reg_a + (size_t)grp * scratch_bytes;
+    float* qs = reinterpret_cast<float*>(base);   // [M][hd]
+    float* Ps = qs + M * hd;                       // [M][128]
+    float* red = Ps + M * kAttnChunk;              // [4][kMaxRows]
+    int* flag = reinterpret_cast<int*>(red + 4 * kMaxRows);
+
+    for (int j = grp; j < n_local; j += p.attn_groups) {
+        const int idx = blockIdx.x + j * gridDim.x;
+        const int kvh = idx / n_chunks, chunk = idx - kvh * n_chunks;
+        const int key0 = chunk * kAttnChunk;
+        const int last_pos = p.pos0 + M - 1;
+        const int n_valid = min(kAttnChunk, last_pos + 1 - key0);
+        const uint32_t gk = gi0 + (uint32_t)(j * 2 * tile_slots), gv = gk + tile_slots;
+        auto slot_ptr = [&](uint32_t g) -> unsigned char* { return sm.ring + (size_t)(g % p.ns) * kSlotBytes; };
+
+        // ---- K tile: wait for the boxes, then overwrite the rows this pass has just written (the producer may
+        //      have copied the tile before the QKV stage of this pass stored them)
+        for (int t = 0; t < tile_slots; ++t) mbar_wait(&sm.full[(gk + t) % p.ns], ((gk + t) / p.ns) & 1, err, kErrFullWait);
+        const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
+        const int n_fresh = fresh1 - fresh0 + 1;
+        if (n_fresh > 0) {
+            for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
+                const int fr = i / vec_per_row, c = i - fr * vec_per_row;
+                const int r = fresh0 + fr - key0;
+                int sit, off;
+                ta.locate(r, c, sit, off);
+                *reinterpret_cast<uint4*>(slot_ptr(gk + sit) + off) =
+                    __ldcg(reinterpret_cast<const uint4*>(st.k_cache + (size_t)(fresh0 + fr) * p.kv_dim + (size_t)kvh * hd + c * 8));
+            }
+        }
+        for (int g = 0; g < group; ++g) {
+            const int head = kvh * group + g;
+            bar_sync(bar_id, 128);  // patched tile visible; previous head's Ps / qs consumed
+            for (int i = gt; i < M * hd; i += 128) {
+                const int m = i / hd, e = i - m * hd;
+                qs[i] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)head * hd + e) << 16);
+            }
+            bar_sync(bar_id, 128);
+
+            // ---- scores: thread t owns key key0 + t
+            float sc[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) sc[m] = 0.f;
+            for (int c = 0; c < vec_per_row; ++c) {
+                int sit, off;
+                ta.locate(gt, c, sit, off);
+                const uint4 kv = *reinterpret_cast<const uint4*>(slot_ptr(gk + sit) + off);
+                const float kf[8] = {bf_lo(kv.x), bf_hi(kv.x), bf_lo(kv.y), bf_hi(kv.y),
+                                     bf_lo(kv.z), bf_hi(kv.z), bf_lo(kv.w), bf_hi(kv.w)};
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    const float4 q0 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8);
+                    const float4 q1 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8 + 4);
+                    float a = sc[m];
+                    a = fmaf(q0.x, kf[0], a);
+                    a = fmaf(q0.y, kf[1], a);
+                    a = fmaf(q0.z, kf[2], a);
+                    a = fmaf(q0.w, kf[3], a);
+                    a = fmaf(q1.x, kf[4], a);
+                    a = fmaf(q1.y, kf[5], a);
+                    a = fmaf(q1.z, kf[6], a);
+                    a = fmaf(q1.w, kf[7], a);
+                    sc[m] = a;
+                }
+            }
+            // ---- chunk-local softmax statistics; the row at position pos0+m sees keys <= pos0+m
+            const int key = key0 + gt;
+            float cmax[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const bool ok = key <= p.pos0 + m;
+                sc[m] = ok ? sc[m] * p.attn_scale : -INFINITY;
+                const float v = warp_max(sc[m]);
+                if (glane == 0) red[gwarp * kMaxRows + m] = v;
+            }
+            bar_sync(bar_id, 128);
+            if (g == group - 1) {  // K tile no longer needed: hand its slots back to the producer
+                if (gt == 0) {
+                    fence_proxy_async_smem();
+                    for (int t = 0; t < tile_slots; ++t) mbar_arrive(&sm.empty[(gk + t) % p.ns]);
+                }
+            }
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+                cmax[m] = fmaxf(fmaxf(red[0 * kMaxRows + m], red[1 * kMaxRows + m]),
+                                fmaxf(red[2 * kMaxRows + m], red[3 * kMaxRows + m]));
+            bar_sync(bar_id, 128);
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                const float pe = (sc[m] == -INFINITY) ? 0.f : expf(sc[m] - cmax[m]);
+                Ps[m * kAttnChunk + gt] = pe;
+                const float v = warp_sum(pe);
+                if (glane == 0) red[gwarp * kMaxRows + m] = v;
+            }
+            if (g == 0) {  // V tile: wait and patch once per item
+                for (int t = 0; t < tile_slots; ++t) mbar_wait(&sm.full[(gv + t) % p.ns], ((gv + t) / p.ns) & 1, err, kErrFullWait);
+                if (n_fresh > 0) {
+                    for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
+                        const int fr = i / vec_per_row, c = i - fr * vec_per_row;
+                        const int r = fresh0 + fr - key0;
+                        int sit, off;
+                        ta.locate(r, c, sit, off);
+                        *reinterpret_cast<uint4*>(slot_ptr(gv + sit) + off) =
+                            __ldcg(reinterpret_cast<const uint4*>(st.v_cache + (size_t)(fresh0 + fr) * p.kv_dim + (size_t)kvh * hd + c * 8));
+                    }
+                }
+            }
+            bar_sync(bar_id, 128);
+            if (gt < M) {
+                const float l = ((red[0 * kMaxRows + gt] + red[1 * kMaxRows + gt]) + red[2 * kMaxRows + gt]) + red[3 * kMaxRows + gt];
+                p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + gt) * 2 + 1] = l;
+            }
+            if (gt == 0) {
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+                    p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + m) * 2 + 0] = cmax[m];
+            }
+            // ---- P V: thread e owns output dimension e
+            for (int e = gt; e < hd; e += 128) {
+                float acc[M];
+#pragma unroll
+                for (int m = 0; m < M; ++m) acc[m] = 0.f;
+                const int c = e >> 3, sub = (e & 7) * 2;
+                for (int jj = 0; jj < n_valid; ++jj) {
+                    int sit, off;
+                    ta.locate(jj, c, sit, off);
+                    const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(slot_ptr(gv + sit) + off + sub));
+#pragma unroll
+                    for (int m = 0; m < M; ++m) acc[m] = fmaf(Ps[m * kAttnChunk + jj], v, acc[m]);
+                }
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+                    p.part_acc[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + m) * hd + e] = acc[m];
+            }
+        }
+        // ---- release the V tile; the last group to finish this kv head merges its chunks in order
+        __threadfence();
+        bar_sync(bar_id, 128);
+        if (gt == 0) {
+            fence_proxy_async_smem();
+            for (int t = 0; t < tile_slots; ++t) mbar_arrive(&sm.empty[(gv + t) % p.ns]);
+            const unsigned tk = atomicAdd(p.attn_counters + kvh, 1u);
+            *flag = (tk == (unsigned)n_chunks - 1) ? 1 : 0;
+        }
+        bar_sync(bar_id, 128);
+        if (*flag) {
+            __threadfence();
+            if (gt == 0) p.attn_counters[kvh] = 0u;
+            for (int g = 0; g < group; ++g) {
+                const int head = kvh * group + g;
+                for (int e = gt; e < hd; e += 128) {
+#pragma unroll
+                    for (int m = 0; m < M; ++m) {
+                        const int nc = (p.pos0 + m) / kAttnChunk + 1;
+                        float mx = -INFINITY, l = 0.f, acc = 0.f;
+                        for (int c = 0; c < nc; ++c) {
+                            const size_t b = ((size_t)head * p.chunk_stride + c) * kMaxRows + m;
+                            const float cm = __ldcg(p.part_ml + b * 2 + 0);
+                            const float cl = __ldcg(p.part_ml + b * 2 + 1);
+                            const float pa = __ldcg(p.part_acc + b * hd + e);
+                            const float mn = fmaxf(mx, cm);
+                            const float s_old = expf(mx - mn), s_new = expf(cm - mn);
+                            acc = acc * s_old + pa * s_new;
+                            l = l * s_old + cl * s_new;
+                            mx = mn;
+                        }
+                        p.a[(size_t)m * p.d_model + (size_t)head * hd + e] = __float2bfloat16_rn(acc / l);
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ============================================================================================ the kernel
+template <int M>
+__global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_constant__ PassParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    PassSmem sm;
+    sm.ring = base;
+    sm.full = reinterpret_cast<uint64_t*>(base + p.off_bars);
+    sm.empty = sm.full + p.ns;
+    sm.red = reinterpret_cast<float*>(base + p.off_misc);
+    sm.flag = reinterpret_cast<int*>(sm.red + kPassConsumerWarps * kMaxRows * 4);
+    sm.psum = reinterpret_cast<float*>(base + p.off_psum);
+    sm.reg_a = base + p.off_reg_a;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.ns; ++i) {
+            mbar_init(&sm.full[i], 1);
+            mbar_init(&sm.empty[i], 1);
+        }
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (threadIdx.x >= kPassConsumers) {
+        if (threadIdx.x == kPassConsumers) pass_producer<M>(p, sm);
+        return;
+    }
+
+    uint32_t gi = 0;
+    for (int s = 0; s < p.n_stages; ++s) {
+        if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);
+        const StageDesc st = p.stages[s];
+        if (st.type == kStEmbed) {
+            const int d = p.d_model;
+            for (int i = blockIdx.x * kPassConsumers + threadIdx.x; i < M * d; i += gridDim.x * kPassConsumers) {
+                const int m = i / d, e = i - m * d;
+                int t = __ldcg(p.tokens + m);
+                t = min(max(t, 0), p.vocab - 1);
+                p.x[i] = __bfloat162float(p.embed[(size_t)t * d + e]);
+            }
+        } else if (st.type == kStAttn) {
+            attn_stage<M>(p, st, sm, gi);
+        } else {
+            gemv_stage<M>(p, st, sm, gi);
+        }
+        grid_arrive(p);
+    }
+}
+
+}  // namespace asd

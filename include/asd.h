@@ -45,7 +45,7 @@ typedef enum {
 } asd_status;
 
 /* Shape of the decoder. Requirements: n_heads * head_dim == d_model; n_heads % n_kv_heads == 0;
- * head_dim % 8 == 0 and head_dim <= 256; d_model % 8 == 0; d_ffn % 8 == 0; 0 <= max_draft <= 8. */
+ * head_dim in {16, 32, 64, 128, 256}; d_model % 8 == 0; d_ffn % 8 == 0; 0 <= max_draft <= 8. */
 typedef struct {
     int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
     int32_t max_seq;   /* capacity of the KV cache in positions */
@@ -110,7 +110,7 @@ int asd_create(const asd_config* cfg, void* dev_workspace, size_t bytes, void* c
 int asd_destroy(asd_ctx* ctx);
 const char* asd_last_error(asd_ctx* ctx);
 
-/* Copy the weights into the workspace (gate and up rows are interleaved on the way). Blocking. */
+/* Copy the weights into the workspace, repacked into the order in which the pass kernel streams them. Blocking. */
 int asd_load_weights_host(asd_ctx* ctx, const asd_host_weights* w);
 /* Same tensors from a flat little-endian file: the twelve arrays of asd_host_weights in declaration order,
  * without header or padding. Errors: IO when the file is missing or short. */
@@ -158,9 +158,15 @@ int asd_generate_device(asd_ctx* ctx, const int32_t* dev_prompt, int32_t n_promp
 /* Per-row results of the last pass of M rows: cosines [L][M] (NaN where the sublayer was skipped),
  * argmax [M]. *M receives the row count. Any output may be NULL. */
 int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_mlp);
-/* Logits [M][vocab] of the last pass; only recorded while asd_set_debug(ctx, 1) is in effect. */
+/* Logits [M][vocab] of the last pass; only recorded while bit 0 of asd_set_debug's flags is set. */
 int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
-int asd_set_debug(asd_ctx* ctx, int32_t record_logits);
+/* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline. */
+int asd_set_debug(asd_ctx* ctx, int32_t flags);
+/* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][6][n_ctas]. Entries 0-3 are device
+ * timestamps in ns of every CTA: 0 = stage entered, 1 = inputs of the stage ready (previous stage finished on
+ * all CTAs), 2 = weight streaming done, 3 = stage left. Entries 4 and 5 are SM cycles that the CTA's first
+ * consumer warp spent waiting for ring slots and working on them. Call first with ns_out = NULL for the sizes. */
+int asd_get_last_trace(asd_ctx* ctx, int32_t* n_stages, int32_t* n_ctas, int64_t* ns_out);
 /* K and V rows (bf16 patterns, n_kv_heads*head_dim each) of one layer (0-based) at one position. */
 int asd_get_kv(asd_ctx* ctx, int32_t layer, int32_t pos, uint16_t* k, uint16_t* v);
 int asd_get_positions(asd_ctx* ctx, int32_t* n_committed, int32_t* draft_cursor);

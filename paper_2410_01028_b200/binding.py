@@ -50,7 +50,7 @@ EXPORTS = (
     "asd_workspace_bytes", "asd_create", "asd_destroy", "asd_last_error", "asd_load_weights_host",
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
-    "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_kv", "asd_get_positions", "asd_get_stats",
+    "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
     "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg",
 )
 
@@ -207,8 +207,17 @@ class Decoder:
         self._check(lib().asd_get_positions(self._ctx, ctypes.byref(a), ctypes.byref(b)), "asd_get_positions")
         return a.value, b.value
 
-    def set_debug(self, record_logits=True):
-        self._check(lib().asd_set_debug(self._ctx, ctypes.c_int32(1 if record_logits else 0)), "asd_set_debug")
+    def set_debug(self, record_logits=True, trace=False):
+        flags = (1 if record_logits else 0) | (2 if trace else 0)
+        self._check(lib().asd_set_debug(self._ctx, ctypes.c_int32(flags)), "asd_set_debug")
+
+    def get_last_trace(self):
+        """Per-stage device timeline of the last pass: int64 array [n_stages, 6, n_ctas] (see asd_get_last_trace)."""
+        ns, nc = ctypes.c_int32(), ctypes.c_int32()
+        self._check(lib().asd_get_last_trace(self._ctx, ctypes.byref(ns), ctypes.byref(nc), None), "asd_get_last_trace")
+        out = np.zeros((ns.value, 6, nc.value), np.int64)
+        self._check(lib().asd_get_last_trace(self._ctx, ctypes.byref(ns), ctypes.byref(nc), _vp(out)), "asd_get_last_trace")
+        return out
 
     # -- passes
     def prefill(self, tokens) -> int:

@@ -122,7 +122,7 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
     const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
     const size_t psum = ((size_t)np_max * 2 * M * 4 + 15) & ~(size_t)15;
-    const size_t misc = ((size_t)16 * kMaxRows * 4 * 4 + 32 + 15) & ~(size_t)15;
+    const size_t misc = ((size_t)16 * kMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16 + 15) & ~(size_t)15;
     const size_t xs = (size_t)M * pass_wseg(M) * kSeg * 2;
     const size_t reg_a = (std::max(xs, 2 * attn_scratch) + 15) & ~(size_t)15;
@@ -147,7 +147,7 @@ struct Layout {
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
     size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
     size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits;
-    size_t stage_tab, tmaps, sync_words;
+    size_t stage_tab, tmaps, sync_words, trace;
     int max_stages;
     size_t total;
     int chunk_stride;
@@ -166,6 +166,9 @@ static bool check_config(const asd_config& c) {
     return true;
 }
 
+// bytes of a matrix in the packed layout of the pass kernel: (pairs of rows) x (segments of 1024 inputs) x 4 KB
+static size_t packed_bytes(size_t n_rows, size_t n_in) { return ((n_rows + 1) / 2) * ((n_in + kSeg - 1) / kSeg) * (size_t)kSlotBytes; }
+
 static Layout make_layout(const asd_config& c) {
     Layout L{};
     const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = (size_t)c.n_kv_heads * c.head_dim, S = c.max_seq;
@@ -176,7 +179,7 @@ static Layout make_layout(const asd_config& c) {
         return at;
     };
     L.embed = take(V * d * 2);
-    L.lm_head = take(V * d * 2);
+    L.lm_head = take(packed_bytes(V, d));
     L.final_norm = take(d * 2);
     {
         size_t lo = 0;
@@ -186,11 +189,11 @@ static Layout make_layout(const asd_config& c) {
             return at;
         };
         L.l_attn_norm = ltake(d * 2);
-        L.l_wqkv = ltake((d + 2 * kvd) * d * 2);
-        L.l_wo = ltake(d * d * 2);
+        L.l_wqkv = ltake(packed_bytes(d + 2 * kvd, d));
+        L.l_wo = ltake(packed_bytes(d, d));
         L.l_mlp_norm = ltake(d * 2);
-        L.l_wgu = ltake(2 * f * d * 2);
-        L.l_wd = ltake(d * f * 2);
+        L.l_wgu = ltake(packed_bytes(2 * f, d));
+        L.l_wd = ltake(packed_bytes(d, f));
         L.layer_stride = lo;
     }
     L.layers = take(L.layer_stride * c.n_layers);
@@ -221,6 +224,7 @@ static Layout make_layout(const asd_config& c) {
     L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
     L.sync_words = take(256);
+    L.trace = take((size_t)L.max_stages * 6 * kMaxGemvGrid * 8);
     L.total = o;
     return L;
 }
@@ -242,7 +246,8 @@ struct asd_ctx {
     std::vector<uint8_t> skip_attn, skip_mlp;
     int64_t n_sim_rows = 0;
     int last_M = 0;
-    bool debug_logits = false, last_has_logits = false;
+    bool debug_logits = false, last_has_logits = false, trace = false;
+    int last_n_stages = 0;
     asd_stats stats{};
     int32_t* pinned = nullptr;  // small host staging buffer
     uint32_t bar_base = 0;      // value of the grid-barrier counter at the start of the next pass
@@ -356,7 +361,7 @@ static int build_stage_tables(asd_ctx* x) {
             if (!(which && x->skip_attn[l])) {
                 StageDesc q{};
                 q.type = kStQkv, q.layer = l, q.n_rows = d + 2 * kvd, q.n_in = d;
-                q.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wqkv);
+                q.W = lw + ly.l_wqkv;
                 q.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_attn_norm);
                 q.k_cache = kc, q.v_cache = vc;
                 t[n++] = q;
@@ -367,7 +372,7 @@ static int build_stage_tables(asd_ctx* x) {
                 t[n++] = a;
                 StageDesc o{};
                 o.type = kStOproj, o.layer = l, o.n_rows = d, o.n_in = d;
-                o.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wo);
+                o.W = lw + ly.l_wo;
                 o.cos_out = cosv + (size_t)(0 * L + l) * kMaxRows;
                 o.sumcos = x->at<double>(ly.sumcos) + l;
                 t[n++] = o;
@@ -375,12 +380,12 @@ static int build_stage_tables(asd_ctx* x) {
             if (!(which && x->skip_mlp[l])) {
                 StageDesc g{};
                 g.type = kStGateUp, g.layer = l, g.n_rows = 2 * f, g.n_in = d;
-                g.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wgu);
+                g.W = lw + ly.l_wgu;
                 g.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_mlp_norm);
                 t[n++] = g;
                 StageDesc w{};
                 w.type = kStDown, w.layer = l, w.n_rows = d, w.n_in = f;
-                w.W = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_wd);
+                w.W = lw + ly.l_wd;
                 w.cos_out = cosv + (size_t)(1 * L + l) * kMaxRows;
                 w.sumcos = x->at<double>(ly.sumcos) + L + l;
                 t[n++] = w;
@@ -388,7 +393,7 @@ static int build_stage_tables(asd_ctx* x) {
         }
         StageDesc h{};
         h.type = kStLmHead, h.layer = L, h.n_rows = c.vocab, h.n_in = d;
-        h.W = x->at<__nv_bfloat16>(ly.lm_head);
+        h.W = x->ws + ly.lm_head;
         h.gain = x->at<__nv_bfloat16>(ly.final_norm);
         t[n++] = h;
         (which ? x->n_stages_draft : x->n_stages_full) = n;
@@ -436,7 +441,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.partials = x->at<float>(ly.partials);
     p.fin_counter = words + 0;
     p.grid_bar = words + 16;
-    p.err = reinterpret_cast<int*>(x->at<int>(ly.accept) + 15);
+    p.err = reinterpret_cast<int*>(words + 32);
     p.bar_base = x->bar_base;
     const int table = use_mask ? 1 : 0;
     p.stages = x->at<StageDesc>(ly.stage_tab) + (size_t)table * ly.max_stages;
@@ -447,7 +452,10 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
     p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
     p.acc_sim = acc_sim ? 1 : 0;
+    p.trace = x->trace ? x->at<long long>(ly.trace) : nullptr;
+    x->last_n_stages = p.n_stages;
     p.ns = pl.ns, p.attn_groups = pl.attn_groups;
+    p.ns_magic = (unsigned)((1ull << 32) / (unsigned)pl.ns + 1);
     p.off_bars = pl.off_bars, p.off_misc = pl.off_misc, p.off_psum = pl.off_psum, p.off_reg_a = pl.off_reg_a;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));
@@ -468,19 +476,22 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     return ASD_OK;
 }
 
-// the bounded waits of the pass kernel report through a device word; 0 = no error
-static int check_device_error(asd_ctx* x, int word) {
-    if (word == 0) return ASD_OK;
+// the bounded waits of the pass kernel report through eight device words; word 0 = 0 means no error
+static int check_device_error(asd_ctx* x, const int32_t* w) {
+    if (w[0] == 0) return ASD_OK;
     static const char* names[] = {"", "a ring slot was never filled", "a ring slot was never released", "the grid barrier never completed"};
-    return fail(x, ASD_ERR_DEVICE_TIMEOUT, std::string("pass kernel gave up waiting: ") + (word >= 1 && word <= 3 ? names[word] : "unknown"));
+    char buf[256];
+    snprintf(buf, sizeof buf, "pass kernel gave up waiting: %s (stage %d, item %d, slot %d, CTA %d, thread %d, tag %d, parity %d)",
+             (w[0] >= 1 && w[0] <= 3) ? names[w[0]] : "unknown", w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+    return fail(x, ASD_ERR_DEVICE_TIMEOUT, buf);
 }
 
-// copy n ints from the device and the pass kernel's error word to the pinned buffer, wait, and check the word
+// copy n ints from the device and the pass kernel's error words to the pinned buffer, wait, and check them
 static int read_back(asd_ctx* x, const int* dev_src, int n) {
     if (n > 0) ASD_CUDA(x, cudaMemcpyAsync(x->pinned, dev_src, (size_t)n * 4, cudaMemcpyDeviceToHost, x->stream));
-    ASD_CUDA(x, cudaMemcpyAsync(x->pinned + 32, x->at<int>(x->lay.accept) + 15, 4, cudaMemcpyDeviceToHost, x->stream));
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned + 32, x->at<unsigned>(x->lay.sync_words) + 32, 32, cudaMemcpyDeviceToHost, x->stream));
     ASD_CUDA(x, cudaStreamSynchronize(x->stream));
-    return check_device_error(x, x->pinned[32]);
+    return check_device_error(x, x->pinned + 32);
 }
 
 // ---------------------------------------------------------------- Algorithm 1
@@ -574,27 +585,73 @@ extern "C" int asd_destroy(asd_ctx* x) {
 
 extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : "null context"; }
 
+// Repack one matrix into the pass kernel's layout and copy it to the device. The logical matrix has n_rows
+// rows of n_in inputs; row(r) returns the host pointer of logical row r. CTA b of a G-CTA grid owns pairs
+// [b*P/G, (b+1)*P/G); its slab is segment-major (for seg: for pair: 2 x 2 KB), ragged ends zero padded.
+template <class RowFn, class PairFn>
+static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, PairFn pair_rows_of,
+                         std::vector<unsigned char>& staging) {
+    const size_t n_pairs = (n_rows + 1) / 2, n_seg = (n_in + kSeg - 1) / kSeg;
+    const size_t total = n_pairs * n_seg * kSlotBytes;
+    const int G = x->dev->num_sms;
+    staging.assign(total, 0);
+#pragma omp parallel for schedule(static)
+    for (int b = 0; b < G; ++b) {
+        const size_t pair0 = (size_t)b * n_pairs / G, pair1 = (size_t)(b + 1) * n_pairs / G, np = pair1 - pair0;
+        unsigned char* slab = staging.data() + pair0 * n_seg * kSlotBytes;
+        for (size_t sg = 0; sg < n_seg; ++sg) {
+            const size_t k0 = sg * kSeg, len = std::min<size_t>(kSeg, n_in - k0);
+            for (size_t pl = 0; pl < np; ++pl) {
+                size_t ra, rb;
+                pair_rows_of(pair0 + pl, ra, rb);
+                unsigned char* item = slab + (sg * np + pl) * kSlotBytes;
+                memcpy(item, row(ra) + k0, len * 2);
+                if (rb < n_rows) memcpy(item + kSlotBytes / 2, row(rb) + k0, len * 2);
+            }
+        }
+    }
+    ASD_CUDA(x, cudaMemcpyAsync(dev_dst, staging.data(), total, cudaMemcpyHostToDevice, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));  // staging is reused by the next matrix
+    return ASD_OK;
+}
+
 static int upload_weights(asd_ctx* x, const asd_host_weights& w) {
     const asd_config& c = x->c;
     const Layout& ly = x->lay;
-    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = x->kv_dim;
+    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, kvd = x->kv_dim, hd = c.head_dim, half = hd / 2;
     cudaStream_t s = x->stream;
+    std::vector<unsigned char> staging;
+    auto plain_pair = [](size_t pr, size_t& ra, size_t& rb) { ra = 2 * pr, rb = 2 * pr + 1; };
+    int rc;
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.embed, w.embed, V * d * 2, cudaMemcpyHostToDevice, s));
-    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.lm_head, w.lm_head, V * d * 2, cudaMemcpyHostToDevice, s));
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.final_norm, w.final_norm, d * 2, cudaMemcpyHostToDevice, s));
+    if ((rc = upload_packed(x, x->ws + ly.lm_head, V, d, [&](size_t r) { return w.lm_head + r * d; }, plain_pair, staging))) return rc;
     for (int l = 0; l < c.n_layers; ++l) {
         unsigned char* lw = x->layer(l);
         ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_attn_norm, w.attn_norm + (size_t)l * d, d * 2, cudaMemcpyHostToDevice, s));
-        unsigned char* qkv = lw + ly.l_wqkv;
-        ASD_CUDA(x, cudaMemcpyAsync(qkv, w.wq + (size_t)l * d * d, d * d * 2, cudaMemcpyHostToDevice, s));
-        ASD_CUDA(x, cudaMemcpyAsync(qkv + d * d * 2, w.wk + (size_t)l * kvd * d, kvd * d * 2, cudaMemcpyHostToDevice, s));
-        ASD_CUDA(x, cudaMemcpyAsync(qkv + (d + kvd) * d * 2, w.wv + (size_t)l * kvd * d, kvd * d * 2, cudaMemcpyHostToDevice, s));
-        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_wo, w.wo + (size_t)l * d * d, d * d * 2, cudaMemcpyHostToDevice, s));
         ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_mlp_norm, w.mlp_norm + (size_t)l * d, d * 2, cudaMemcpyHostToDevice, s));
-        // gate row i -> row 2i, up row i -> row 2i+1, so that one warp holds both operands of SwiGLU
-        ASD_CUDA(x, cudaMemcpy2DAsync(lw + ly.l_wgu, 2 * d * 2, w.wg + (size_t)l * f * d, d * 2, d * 2, f, cudaMemcpyHostToDevice, s));
-        ASD_CUDA(x, cudaMemcpy2DAsync(lw + ly.l_wgu + d * 2, 2 * d * 2, w.wu + (size_t)l * f * d, d * 2, d * 2, f, cudaMemcpyHostToDevice, s));
-        ASD_CUDA(x, cudaMemcpyAsync(lw + ly.l_wd, w.wd + (size_t)l * d * f, d * f * 2, cudaMemcpyHostToDevice, s));
+        // fused [q rows; k rows; v rows]; a pair is the two rotary partners (j, j + head_dim/2) of one head
+        const uint16_t *wq = w.wq + (size_t)l * d * d, *wk = w.wk + (size_t)l * kvd * d, *wv = w.wv + (size_t)l * kvd * d;
+        auto qkv_row = [&](size_t r) { return r < d ? wq + r * d : (r < d + kvd ? wk + (r - d) * d : wv + (r - d - kvd) * d); };
+        auto qkv_pair = [&](size_t pr, size_t& ra, size_t& rb) {
+            const size_t nq = d / 2, nk = kvd / 2;
+            size_t base, pp;
+            if (pr < nq) base = 0, pp = pr;
+            else if (pr < nq + nk) base = d, pp = pr - nq;
+            else base = d + kvd, pp = pr - nq - nk;
+            ra = base + (pp / half) * hd + pp % half;
+            rb = ra + half;
+        };
+        if ((rc = upload_packed(x, lw + ly.l_wqkv, d + 2 * kvd, d, qkv_row, qkv_pair, staging))) return rc;
+        const uint16_t* wo = w.wo + (size_t)l * d * d;
+        if ((rc = upload_packed(x, lw + ly.l_wo, d, d, [&](size_t r) { return wo + r * d; }, plain_pair, staging))) return rc;
+        // gate_i and up_i form a pair, so that one warp holds both operands of SwiGLU
+        const uint16_t *wg = w.wg + (size_t)l * f * d, *wu = w.wu + (size_t)l * f * d;
+        if ((rc = upload_packed(x, lw + ly.l_wgu, 2 * f, d, [&](size_t r) { return (r & 1) ? wu + (r / 2) * d : wg + (r / 2) * d; },
+                                plain_pair, staging)))
+            return rc;
+        const uint16_t* wd = w.wd + (size_t)l * d * f;
+        if ((rc = upload_packed(x, lw + ly.l_wd, d, f, [&](size_t r) { return wd + r * f; }, plain_pair, staging))) return rc;
     }
     ASD_CUDA(x, cudaStreamSynchronize(s));
     x->have_weights = true;
@@ -642,7 +699,7 @@ extern "C" int asd_reset(asd_ctx* x) {
     x->spans.clear();
     x->events_used = 0;
     ASD_CUDA(x, cudaMemsetAsync(x->ws + x->lay.sumcos, 0, (size_t)2 * std::max(x->c.n_layers, 1) * 8, x->stream));
-    ASD_CUDA(x, cudaMemsetAsync(x->at<int>(x->lay.accept), 0, 64 * 4, x->stream));
+    ASD_CUDA(x, cudaMemsetAsync(x->at<unsigned>(x->lay.sync_words) + 32, 0, 32, x->stream));
     return build_stage_tables(x);
 }
 
@@ -941,9 +998,22 @@ extern "C" int asd_get_last_cosines(asd_ctx* x, int32_t* M, float* cos_attn, flo
     return ASD_OK;
 }
 
-extern "C" int asd_set_debug(asd_ctx* x, int32_t record_logits) {
+extern "C" int asd_set_debug(asd_ctx* x, int32_t flags) {
     if (!x) return ASD_ERR_ARG;
-    x->debug_logits = record_logits != 0;
+    x->debug_logits = (flags & 1) != 0;
+    x->trace = (flags & 2) != 0;
+    return ASD_OK;
+}
+
+extern "C" int asd_get_last_trace(asd_ctx* x, int32_t* n_stages, int32_t* n_ctas, int64_t* ns_out) {
+    if (!x) return ASD_ERR_ARG;
+    if (!x->trace || x->last_n_stages == 0) return fail(x, ASD_ERR_STATE, "no pass has run with tracing on (asd_set_debug bit 1)");
+    if (n_stages) *n_stages = x->last_n_stages;
+    if (n_ctas) *n_ctas = x->dev->num_sms;
+    if (ns_out) {
+        ASD_CUDA(x, cudaMemcpyAsync(ns_out, x->ws + x->lay.trace, (size_t)x->last_n_stages * 6 * x->dev->num_sms * 8, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    }
     return ASD_OK;
 }
 

@@ -332,16 +332,26 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvParams 
             p.partials[((size_t)blockIdx.x * kMaxRows + m) * 4 + j] = tot;
         }
         if (last_cta_arrives(p.counter, flag)) {
-            if (tid < M) {
+            // one warp per activation row: lanes add the per-CTA partials b = lane, lane+32, ... in order, then an
+            // xor butterfly in double precision (fixed order, independent of the row count)
+            if (warp < M) {
                 double sxy = 0, sxx = 0, syy = 0;
-                for (unsigned b = 0; b < gridDim.x; ++b) {
-                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
-                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1);
-                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 2);
+                for (unsigned b = lane; b < gridDim.x; b += 32) {
+                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 0);
+                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 1);
+                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 2);
                 }
-                const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
-                p.cos_out[tid] = (float)c;
-                red[tid] = (float)c;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    sxy += __shfl_xor_sync(0xffffffffu, sxy, o);
+                    sxx += __shfl_xor_sync(0xffffffffu, sxx, o);
+                    syy += __shfl_xor_sync(0xffffffffu, syy, o);
+                }
+                if (lane == 0) {
+                    const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
+                    p.cos_out[warp] = (float)c;
+                    red[warp] = (float)c;
+                }
             }
             __syncthreads();
             if (tid == 0) {

@@ -4,16 +4,24 @@
 // HBM idle at every boundary (launch latency, RMSNorm prologue, drain). Weights, however, never depend on
 // activations. So here one CTA per SM stays resident for the whole pass (cooperative launch) and is split in
 // two roles:
-//   * a producer thread walks this CTA's share of EVERY stage's weights (and of the old part of the KV cache)
+//   * a producer warp walks this CTA's share of EVERY stage's weights (and of the old part of the KV cache)
 //     in order and keeps a shared-memory ring of 4 KB slots full with TMA copies (cp.async.bulk, and
 //     cp.async.bulk.tensor with 128-byte swizzle for K/V boxes). It never waits for activations, so HBM keeps
-//     streaming across stage boundaries, grid barriers and prologues;
+//     streaming across stage boundaries, grid barriers and prologues. Weights are stored in HBM in exactly
+//     the order the ring consumes them (see "packed weights" below), so a CTA's slab of a stage is one
+//     contiguous byte range;
 //   * 15 consumer warps wait for the previous stage of all CTAs (a grid barrier on a monotonically increasing
 //     counter, bounded spin), stage the activations in shared memory (RMSNorm fused), multiply the ring slots
 //     with packed fp32 FMAs, and run the epilogue: RoPE + KV append, SwiGLU, residual add + cosine
 //     similarity (summand of C_l, Section 3.2), LM-head argmax + greedy acceptance (Section 1).
 // Sublayers in the skip mask (the draft model D, Algorithm 1) simply do not appear in the stage table: no
 // weights are streamed and no K/V is touched for them.
+//
+// Packed weights: a matrix [n_rows, n_in] is cut into PAIRS of rows (the two rotary partners of a q/k head,
+// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 1024 inputs. One ring item = one pair x one
+// segment = 2 x 2 KB = one 4 KB slot (a ragged last segment is zero padded). CTA b owns pairs
+// [b*P/G, (b+1)*P/G); its slab is stored segment-major: for seg: for pair: item. Consecutive ring items thus
+// belong to different pairs, i.e. to different consumer warps, and are consumed as soon as they land.
 //
 // Reduction order is fixed and independent of the row count M: per (weight row, activation row) a lane adds
 // the even and the odd elements of its 16-byte chunks of a 1024-element segment in order, the two halves are
@@ -32,7 +40,6 @@ namespace asd {
 constexpr int kPassConsumerWarps = 15;
 constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
-constexpr int kWsegMax = 4;                         // at most 4 segments of the reduction dimension per activation window
 constexpr int kXsBudget = 40960;                    // bytes of shared memory for the activation window / attention scratch
 
 enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead };
@@ -40,7 +47,7 @@ enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDo
 struct StageDesc {
     int type, layer;
     int n_rows, n_in;
-    const __nv_bfloat16* W;
+    const unsigned char* W;             // packed weights of this stage (4 KB items, see above)
     const __nv_bfloat16* gain;
     __nv_bfloat16 *k_cache, *v_cache;   // this layer's cache [max_seq, kv_dim]
     const CUtensorMap *tm_k, *tm_v;     // tensor maps over the same
@@ -72,15 +79,18 @@ struct PassParams {
     int* accept_out;
     float* logits_out;
     int acc_sim;
+    long long* trace;  // optional [n_stages][6][gridDim.x] device timestamps (ns) and cycle counts, or null
     // shared-memory plan (bytes from the 1024-aligned base)
     int ns;            // ring slots
+    unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
     int attn_groups;   // 1 or 2 groups of 4 warps work on attention items
     int off_bars, off_misc, off_psum, off_reg_a;
 };
 
+// segments of the reduction dimension whose activations (M rows, bf16) fit the shared-memory window
 __host__ __device__ inline int pass_wseg(int M) {
-    int w = kXsBudget / (M * 2048);
-    return w < 1 ? 1 : (w > kWsegMax ? kWsegMax : w);
+    const int w = kXsBudget / (M * 2048);
+    return w < 1 ? 1 : w;
 }
 
 struct PassSmem {
@@ -88,6 +98,7 @@ struct PassSmem {
     uint64_t *full, *empty;
     float* red;   // [16][kMaxRows*4]
     int* flag;    // [8]
+    volatile unsigned* consumed;  // [64] generations of each ring slot that consumers have finished with
     float* psum;
     unsigned char* reg_a;
 };
@@ -129,18 +140,74 @@ __device__ __forceinline__ int attn_local_items(const PassParams& p, int M, int&
     return ((int)blockIdx.x < total) ? (total - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 }
 
+// ============================================================================================ ring protocol
+// mbarrier waits are by phase PARITY, which is only unambiguous when the waiter is at most one phase away from
+// the barrier. Consumer warps and producer lanes skip through the ring (each takes every n-th item), so a
+// waiter can reach generation g of a slot while generation g-1 has not even landed. Every wait therefore
+// first checks a plain per-slot counter of consumed generations (monotonic, no aliasing) and only then the
+// barrier, which by then is at most one phase away.
+__device__ __forceinline__ void ring_locate(const PassParams& p, uint32_t g, int& slot, uint32_t& gen) {
+    gen = fast_div(g, p.ns_magic);
+    slot = (int)(g - gen * (uint32_t)p.ns);
+}
+
+__device__ __forceinline__ bool ring_spin_consumed(const PassParams& p, const PassSmem& sm, int slot, uint32_t gen, int code,
+                                                   int stage, uint32_t g, int tag) {
+    if (sm.consumed[slot] >= gen) return true;
+    volatile int* err = p.err;
+    const long long t0 = clock64();
+    for (unsigned spin = 1;; ++spin) {
+        if (sm.consumed[slot] >= gen) return true;
+        if ((spin & 255u) != 0) continue;
+        if (*err != kErrNone) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            if (atomicCAS(p.err, kErrNone, code) == kErrNone) {
+                p.err[1] = stage, p.err[2] = (int)g, p.err[3] = slot, p.err[4] = blockIdx.x, p.err[5] = threadIdx.x;
+                p.err[6] = tag, p.err[7] = -1;
+            }
+            return false;
+        }
+    }
+}
+
+// consumer: wait until ring item g has landed; returns the slot
+__device__ __forceinline__ int ring_wait_full(const PassParams& p, const PassSmem& sm, uint32_t g, int stage, int tag) {
+    int slot;
+    uint32_t gen;
+    ring_locate(p, g, slot, gen);
+    if (gen > 0 && !ring_spin_consumed(p, sm, slot, gen, kErrFullWait, stage, g, tag)) return slot;
+    mbar_wait(&sm.full[slot], gen & 1, p.err, kErrFullWait, stage, g, slot, tag);
+    return slot;
+}
+// consumer: one thread, after all readers of the slot are done (warp or group barrier before the call)
+__device__ __forceinline__ void ring_release(const PassParams& p, const PassSmem& sm, uint32_t g) {
+    int slot;
+    uint32_t gen;
+    ring_locate(p, g, slot, gen);
+    __threadfence_block();  // the readers' shared-memory loads are ordered before the slot is handed back
+    sm.consumed[slot] = gen + 1;
+    mbar_arrive(&sm.empty[slot]);
+}
+// producer: wait until the slot of ring item g may be overwritten; returns the slot
+__device__ __forceinline__ int ring_acquire(const PassParams& p, const PassSmem& sm, uint32_t g, int stage, int tag) {
+    int slot;
+    uint32_t gen;
+    ring_locate(p, g, slot, gen);
+    if (gen > 0) {
+        if (!ring_spin_consumed(p, sm, slot, gen, kErrEmptyWait, stage, g, tag)) return slot;
+        mbar_wait(&sm.empty[slot], (gen - 1) & 1, p.err, kErrEmptyWait, stage, g, slot, tag);
+    }
+    return slot;
+}
+
 // ============================================================================================ producer
+// The whole producer warp feeds the ring: lane l takes ring items l, l+32, ... of each stage.
 template <int M>
 __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
+    const int lane = threadIdx.x & 31;
     volatile int* err = p.err;
-    uint32_t gi = 0;
-    const int ns = p.ns;
-    auto acquire = [&](uint32_t g) -> int {   // wait until the slot of ring item g may be overwritten
-        const int slot = g % ns;
-        const uint32_t gen = g / ns;
-        if (gen > 0) mbar_wait(&sm.empty[slot], (gen - 1) & 1, err, kErrEmptyWait);
-        return slot;
-    };
+    uint32_t gi = 0, issued[2] = {0, 0};
+    int n_issued = 0;
     for (int s = 0; s < p.n_stages; ++s) {
         const StageDesc st = p.stages[s];
         if (st.type == kStEmbed) continue;
@@ -150,60 +217,61 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
             const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
             const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
             const uint32_t box_bytes = 32u * box_cols * 2u;
-            for (int j = 0; j < n_local; ++j) {
-                const int idx = blockIdx.x + j * gridDim.x;
-                const int kvh = idx / n_chunks, chunk = idx - kvh * n_chunks;
-                for (int which = 0; which < 2; ++which) {
-                    const CUtensorMap* tm = which ? st.tm_v : st.tm_k;
-                    for (int rg = 0; rg < 4; ++rg)
-                        for (int hb = 0; hb < nhb; ++hb) {
-                            const int slot = acquire(gi);
-                            mbar_expect_tx(&sm.full[slot], box_bytes);
-                            tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, tm, kvh * p.head_dim + hb * 64,
-                                        chunk * kAttnChunk + rg * 32, &sm.full[slot]);
-                            ++gi;
-                        }
-                }
+            const int tile_slots = 4 * nhb;
+            const int n_items = n_local * 2 * tile_slots;
+            for (int idx = lane; idx < n_items; idx += 32) {
+                const int j = idx / (2 * tile_slots), r = idx - j * 2 * tile_slots;
+                const int which = r / tile_slots, t = r - which * tile_slots;
+                const int rg = t / nhb, hb = t - rg * nhb;
+                const int item = blockIdx.x + j * gridDim.x;
+                const int kvh = item / n_chunks, chunk = item - kvh * n_chunks;
+                const uint32_t g = gi + (uint32_t)idx;
+                const int slot = ring_acquire(p, sm, g, s, M);
+                mbar_expect_tx(&sm.full[slot], box_bytes);
+                tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, which ? st.tm_v : st.tm_k, kvh * p.head_dim + hb * 64,
+                            chunk * kAttnChunk + rg * 32, &sm.full[slot]);
+                issued[1] = issued[0], issued[0] = g, ++n_issued;
             }
+            gi += (uint32_t)n_items;
             continue;
         }
-        // GEMV stage: windows of segments, pairs inside a window, segments of a pair consecutively
+        // GEMV stage: this CTA's slab is contiguous and already in ring order
         int pair0, np;
         cta_pairs(st.n_rows, pair0, np);
         const int n_seg = (st.n_in + kSeg - 1) / kSeg;
-        const int wseg = pass_wseg(M);
-        for (int w0 = 0; w0 < n_seg; w0 += wseg) {
-            const int ws = min(wseg, n_seg - w0);
-            for (int pl = 0; pl < np; ++pl) {
-                int ra, rb;
-                stage_pair_rows(st.type, p, pair0 + pl, ra, rb);
-                rb = min(rb, st.n_rows - 1);
-                for (int sg = w0; sg < w0 + ws; ++sg) {
-                    const int k0 = sg * kSeg;
-                    const uint32_t bytes = (uint32_t)min(kSeg, st.n_in - k0) * 2u;
-                    const int slot = acquire(gi);
-                    unsigned char* dst = sm.ring + (size_t)slot * kSlotBytes;
-                    mbar_expect_tx(&sm.full[slot], 2u * bytes);
-                    tma_load_1d(dst, st.W + (size_t)ra * st.n_in + k0, bytes, &sm.full[slot]);
-                    tma_load_1d(dst + kSlotBytes / 2, st.W + (size_t)rb * st.n_in + k0, bytes, &sm.full[slot]);
-                    ++gi;
-                }
-            }
+        const int n_items = np * n_seg;
+        const unsigned char* slab = st.W + (size_t)pair0 * n_seg * kSlotBytes;
+        for (int idx = lane; idx < n_items; idx += 32) {
+            const uint32_t g = gi + (uint32_t)idx;
+            const int slot = ring_acquire(p, sm, g, s, M);
+            mbar_expect_tx(&sm.full[slot], kSlotBytes);
+            tma_load_1d(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)idx * kSlotBytes, kSlotBytes, &sm.full[slot]);
+            issued[1] = issued[0], issued[0] = g, ++n_issued;
         }
+        gi += (uint32_t)n_items;
     }
-    // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let them land
-    // (bounded) before the CTA exits.
+    // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let this lane's
+    // last two copies land (bounded) before the CTA exits (the ring holds at most two items of a lane).
     if (*err != kErrNone) {
-        const uint32_t n_wait = gi < (uint32_t)ns ? gi : (uint32_t)ns;
-        for (uint32_t k = 0; k < n_wait; ++k) {
-            const uint32_t g = gi - 1 - k;
-            const int slot = g % ns;
-            const uint32_t par = (g / ns) & 1;
+        for (int k = 0; k < 2 && k < n_issued; ++k) {
+            int slot;
+            uint32_t gen;
+            ring_locate(p, issued[k], slot, gen);
             const long long t0 = clock64();
-            while (!mbar_try_wait(&sm.full[slot], par) && clock64() - t0 < 20000000LL) {
+            while (!mbar_try_wait(&sm.full[slot], gen & 1) && clock64() - t0 < 20000000LL) {
             }
         }
     }
+}
+
+__device__ __forceinline__ long long global_ns() {
+    long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// per-stage timeline of every CTA (debugging aid): 0 = stage entered, 1 = inputs ready, 2 = streaming done, 3 = stage left
+__device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k) {
+    if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 6 + k) * gridDim.x + blockIdx.x] = global_ns();
 }
 
 // ============================================================================================ grid barrier
@@ -223,7 +291,10 @@ __device__ __forceinline__ void grid_wait(const PassParams& p, unsigned target) 
         while ((int)(ld_acquire_gpu(p.grid_bar) - target) < 0) {
             if (*err != kErrNone) break;
             if (clock64() - t0 > kWaitCycles) {
-                atomicCAS(p.err, kErrNone, kErrGridWait);
+                if (atomicCAS(p.err, kErrNone, kErrGridWait) == kErrNone) {
+                    p.err[1] = (int)((target - p.bar_base) / gridDim.x), p.err[2] = (int)ld_acquire_gpu(p.grid_bar);
+                    p.err[3] = (int)target, p.err[4] = blockIdx.x;
+                }
                 break;
             }
         }
@@ -247,7 +318,7 @@ __device__ __forceinline__ bool last_cta_consumers(unsigned* counter, int* flag_
 
 // ============================================================================================ GEMV stage
 template <int M>
-__device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi) {
+__device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int type = st.type;
     const bool norm = (type == kStQkv || type == kStGateUp || type == kStLmHead);
@@ -260,7 +331,6 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
     float* red = sm.red;
     float* psum = sm.psum;
-    volatile int* err = p.err;
 
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
@@ -292,6 +362,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     }
     for (int i = tid; i < np * 2 * M; i += kPassConsumers) psum[i] = 0.f;
 
+    long long cyc_wait = 0, cyc_work = 0;  // when tracing: cycles this warp spent waiting for slots / working on them
     // ---- stream the slab window by window
     for (int w0 = 0; w0 < n_seg; w0 += wseg) {
         const int ws = min(wseg, n_seg - w0);
@@ -323,19 +394,16 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         }
         consumers_sync();
 
-        for (int pl = warp; pl < np; pl += kPassConsumerWarps) {
-            float sa[M], sb[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) {
-                sa[m] = psum[(pl * 2 + 0) * M + m];
-                sb[m] = psum[(pl * 2 + 1) * M + m];
-            }
-            for (int sg = 0; sg < ws; ++sg) {
-                const uint32_t g = gi + (uint32_t)(np * w0 + pl * ws + sg);
-                const int slot = g % p.ns;
-                mbar_wait(&sm.full[slot], (g / p.ns) & 1, err, kErrFullWait);
+        // ring order is segment-major: consecutive items belong to different pairs, i.e. to different warps
+        for (int sg = 0; sg < ws; ++sg) {
+            const int seg = w0 + sg;
+            const int seglen = min(kSeg, n_in - seg * kSeg);
+            for (int pl = warp; pl < np; pl += kPassConsumerWarps) {
+                const uint32_t g = gi + (uint32_t)(seg * np + pl);
+                const long long tw0 = p.trace ? clock64() : 0;
+                const int slot = ring_wait_full(p, sm, g, stage, M * 1000 + seg);
+                const long long tw1 = p.trace ? clock64() : 0;
                 const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes;
-                const int seglen = min(kSeg, n_in - (w0 + sg) * kSeg);
                 unsigned long long acc_a[M], acc_b[M];
 #pragma unroll
                 for (int m = 0; m < M; ++m) acc_a[m] = acc_b[m] = 0ull;
@@ -363,27 +431,37 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.empty[slot]);
+                if (lane == 0) ring_release(p, sm, g);
+                float va[M], vb[M];
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
                     float e, o;
                     unpack2(acc_a[m], e, o);
-                    sa[m] += warp_sum(e + o);
+                    va[m] = warp_sum(e + o);
                     unpack2(acc_b[m], e, o);
-                    sb[m] += warp_sum(e + o);
+                    vb[m] = warp_sum(e + o);
                 }
-            }
-            if (lane == 0) {
+                if (lane == 0) {  // segments of a pair are added in ascending order, always by this warp
 #pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    psum[(pl * 2 + 0) * M + m] = sa[m];
-                    psum[(pl * 2 + 1) * M + m] = sb[m];
+                    for (int m = 0; m < M; ++m) {
+                        psum[(pl * 2 + 0) * M + m] += va[m];
+                        psum[(pl * 2 + 1) * M + m] += vb[m];
+                    }
+                }
+                if (p.trace) {
+                    cyc_wait += tw1 - tw0;
+                    cyc_work += clock64() - tw1;
                 }
             }
         }
     }
     gi += (uint32_t)(np * n_seg);
     consumers_sync();
+    trace_mark(p, stage, 2);
+    if (p.trace && tid == 0) {
+        p.trace[((size_t)stage * 6 + 4) * gridDim.x + blockIdx.x] = cyc_wait;
+        p.trace[((size_t)stage * 6 + 5) * gridDim.x + blockIdx.x] = cyc_work;
+    }
 
     // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
     float s_loc[M][3];
@@ -481,16 +559,26 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             p.partials[((size_t)blockIdx.x * kMaxRows + m) * 4 + j] = tot;
         }
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
-            if (tid < M) {
+            // one warp per activation row: lanes add the per-CTA partials b = lane, lane+32, ... in order, then an
+            // xor butterfly in double precision (fixed order, independent of the row count)
+            if (warp < M) {
                 double sxy = 0, sxx = 0, syy = 0;
-                for (unsigned b = 0; b < gridDim.x; ++b) {
-                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
-                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1);
-                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 2);
+                for (unsigned b = lane; b < gridDim.x; b += 32) {
+                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 0);
+                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 1);
+                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 2);
                 }
-                const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
-                st.cos_out[tid] = (float)c;
-                red[tid] = (float)c;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    sxy += __shfl_xor_sync(0xffffffffu, sxy, o);
+                    sxx += __shfl_xor_sync(0xffffffffu, sxx, o);
+                    syy += __shfl_xor_sync(0xffffffffu, syy, o);
+                }
+                if (lane == 0) {
+                    const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
+                    st.cos_out[warp] = (float)c;
+                    red[warp] = (float)c;
+                }
             }
             consumers_sync();
             if (tid == 0) {
@@ -538,20 +626,31 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         }
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
             int* g = reinterpret_cast<int*>(red);
-            if (tid < M) {
+            if (warp < M) {  // one warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index
                 float v = -INFINITY;
                 int i = INT_MAX;
-                for (unsigned b = 0; b < gridDim.x; ++b) {
-                    const float ov = __ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
-                    const int oi = __float_as_int(__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1));
+                for (unsigned b = lane; b < gridDim.x; b += 32) {
+                    const float ov = __ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 0);
+                    const int oi = __float_as_int(__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 1));
                     if (ov > v || (ov == v && oi < i)) {
                         v = ov;
                         i = oi;
                     }
                 }
-                if (i == INT_MAX) i = 0;
-                p.argmax_out[tid] = i;
-                g[tid] = i;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+                    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+                    if (ov > v || (ov == v && oi < i)) {
+                        v = ov;
+                        i = oi;
+                    }
+                }
+                if (lane == 0) {
+                    if (i == INT_MAX) i = 0;
+                    p.argmax_out[warp] = i;
+                    g[warp] = i;
+                }
             }
             consumers_sync();
             if (tid == 0) {
@@ -583,7 +682,7 @@ struct TileAddr {
 };
 
 template <int M>
-__device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi) {
+__device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, warp = tid >> 5;
     const int hd = p.head_dim;
     const int nhb = hd > 64 ? hd / 64 : 1;
@@ -596,7 +695,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     const int grp = warp >> 2;
     if (grp >= p.attn_groups) return;
 
-    volatile int* err = p.err;
+    
     const int gt = tid & 127, glane = gt & 31, gwarp = gt >> 5;
     const int bar_id = 2 + grp;
     const int group = p.n_heads / p.n_kv_heads;
@@ -618,11 +717,16 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         const int last_pos = p.pos0 + M - 1;
         const int n_valid = min(kAttnChunk, last_pos + 1 - key0);
         const uint32_t gk = gi0 + (uint32_t)(j * 2 * tile_slots), gv = gk + tile_slots;
-        auto slot_ptr = [&](uint32_t g) -> unsigned char* { return sm.ring + (size_t)(g % p.ns) * kSlotBytes; };
+        auto slot_ptr = [&](uint32_t g) -> unsigned char* {
+            int slot;
+            uint32_t gen;
+            ring_locate(p, g, slot, gen);
+            return sm.ring + (size_t)slot * kSlotBytes;
+        };
 
         // ---- K tile: wait for the boxes, then overwrite the rows this pass has just written (the producer may
         //      have copied the tile before the QKV stage of this pass stored them)
-        for (int t = 0; t < tile_slots; ++t) mbar_wait(&sm.full[(gk + t) % p.ns], ((gk + t) / p.ns) & 1, err, kErrFullWait);
+        for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
         const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
         const int n_fresh = fresh1 - fresh0 + 1;
         if (n_fresh > 0) {
@@ -684,7 +788,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             if (g == group - 1) {  // K tile no longer needed: hand its slots back to the producer
                 if (gt == 0) {
                     fence_proxy_async_smem();
-                    for (int t = 0; t < tile_slots; ++t) mbar_arrive(&sm.empty[(gk + t) % p.ns]);
+                    for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gk + t);
                 }
             }
 #pragma unroll
@@ -700,7 +804,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                 if (glane == 0) red[gwarp * kMaxRows + m] = v;
             }
             if (g == 0) {  // V tile: wait and patch once per item
-                for (int t = 0; t < tile_slots; ++t) mbar_wait(&sm.full[(gv + t) % p.ns], ((gv + t) / p.ns) & 1, err, kErrFullWait);
+                for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gv + t, stage, M * 1000 + 500 + j);
                 if (n_fresh > 0) {
                     for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
                         const int fr = i / vec_per_row, c = i - fr * vec_per_row;
@@ -745,7 +849,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         bar_sync(bar_id, 128);
         if (gt == 0) {
             fence_proxy_async_smem();
-            for (int t = 0; t < tile_slots; ++t) mbar_arrive(&sm.empty[(gv + t) % p.ns]);
+            for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
             const unsigned tk = atomicAdd(p.attn_counters + kvh, 1u);
             *flag = (tk == (unsigned)n_chunks - 1) ? 1 : 0;
         }
@@ -789,7 +893,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     sm.full = reinterpret_cast<uint64_t*>(base + p.off_bars);
     sm.empty = sm.full + p.ns;
     sm.red = reinterpret_cast<float*>(base + p.off_misc);
-    sm.flag = reinterpret_cast<int*>(sm.red + kPassConsumerWarps * kMaxRows * 4);
+    sm.flag = reinterpret_cast<int*>(sm.red + 16 * kMaxRows * 4);
+    sm.consumed = reinterpret_cast<volatile unsigned*>(sm.flag + 8);
     sm.psum = reinterpret_cast<float*>(base + p.off_psum);
     sm.reg_a = base + p.off_reg_a;
 
@@ -797,19 +902,22 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
         for (int i = 0; i < p.ns; ++i) {
             mbar_init(&sm.full[i], 1);
             mbar_init(&sm.empty[i], 1);
+            sm.consumed[i] = 0u;
         }
         mbar_fence_init();
     }
     __syncthreads();
 
     if (threadIdx.x >= kPassConsumers) {
-        if (threadIdx.x == kPassConsumers) pass_producer<M>(p, sm);
+        pass_producer<M>(p, sm);
         return;
     }
 
     uint32_t gi = 0;
     for (int s = 0; s < p.n_stages; ++s) {
+        trace_mark(p, s, 0);
         if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);
+        trace_mark(p, s, 1);
         const StageDesc st = p.stages[s];
         if (st.type == kStEmbed) {
             const int d = p.d_model;
@@ -820,10 +928,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
                 p.x[i] = __bfloat162float(p.embed[(size_t)t * d + e]);
             }
         } else if (st.type == kStAttn) {
-            attn_stage<M>(p, st, sm, gi);
+            attn_stage<M>(p, st, sm, gi, s);
         } else {
-            gemv_stage<M>(p, st, sm, gi);
+            gemv_stage<M>(p, st, sm, gi, s);
         }
+        trace_mark(p, s, 3);
         grid_arrive(p);
     }
 }

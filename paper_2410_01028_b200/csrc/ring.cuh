@@ -45,14 +45,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Wait for a phase of an mbarrier. Returns false when the wait was abandoned (error word set).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err, int code) {
+// The first wait to give up also records where it was: err[1..7] = stage, ring item, slot, CTA, thread, tag, parity.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err, int code, int stage = -1,
+                                          unsigned item = 0, int slot = -1, int tag = 0) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (true) {
+    for (unsigned spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 255u) != 0) continue;  // the error word lives in global memory: look at it only now and then
         if (*err != kErrNone) return false;
         if (clock64() - t0 > kWaitCycles) {
-            atomicCAS(const_cast<int*>(err), kErrNone, code);
+            if (atomicCAS(const_cast<int*>(err), kErrNone, code) == kErrNone) {
+                err[1] = stage, err[2] = (int)item, err[3] = slot, err[4] = blockIdx.x, err[5] = threadIdx.x, err[6] = tag;
+                err[7] = (int)parity;
+            }
             return false;
         }
     }
@@ -100,6 +106,9 @@ __device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsign
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+// exact g / d for 0 <= g < 2^22 and 1 <= d <= 64, with magic = 2^32 / d + 1 (computed on the host)
+__device__ __forceinline__ uint32_t fast_div(uint32_t g, uint32_t magic) { return __umulhi(g, magic); }
+
 // a packed bf16 pair (element k in the low half, k+1 in the high half) widened to a packed fp32 pair
 __device__ __forceinline__ unsigned long long bf2_to_f2(uint32_t u) {
     return pack2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));

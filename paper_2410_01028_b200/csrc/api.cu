@@ -147,7 +147,7 @@ struct Layout {
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
     size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
     size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits;
-    size_t stage_tab, tmaps, sync_words, trace;
+    size_t stage_tab, tmaps, sync_words, trace, resid_tab;
     int max_stages;
     size_t total;
     int chunk_stride;
@@ -209,7 +209,7 @@ static Layout make_layout(const asd_config& c) {
     L.chunk_stride = (int)((S + kAttnChunk - 1) / kAttnChunk);
     L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * c.head_dim * 4);
     L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * 2 * 4);
-    L.partials = take((size_t)kMaxGemvGrid * kMaxRows * 4 * 4);
+    L.partials = take((size_t)(2 * c.n_layers + 1) * kMaxGemvGrid * kMaxRows * 4 * 4);
     L.counters = take((size_t)(c.n_kv_heads + 64) * 4);
     L.cosv = take((size_t)2 * std::max(c.n_layers, 1) * kMaxRows * 4);
     L.sumcos = take((size_t)2 * std::max(c.n_layers, 1) * 8);
@@ -220,10 +220,11 @@ static Layout make_layout(const asd_config& c) {
     L.argmax = take(64 * 4);
     L.accept = take(64 * 4);
     L.logits = take((size_t)kMaxRows * V * 4);
-    L.max_stages = 5 * c.n_layers + 2;
+    L.max_stages = 5 * c.n_layers + 3;
     L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
     L.sync_words = take(256);
+    L.resid_tab = take((size_t)2 * (2 * std::max(c.n_layers, 1)) * sizeof(ResidOut));
     L.trace = take((size_t)L.max_stages * 6 * kMaxGemvGrid * 8);
     L.total = o;
     return L;
@@ -251,7 +252,7 @@ struct asd_ctx {
     asd_stats stats{};
     int32_t* pinned = nullptr;  // small host staging buffer
     uint32_t bar_base = 0;      // value of the grid-barrier counter at the start of the next pass
-    int n_stages_full = 0, n_stages_draft = 0;
+    int n_stages_full = 0, n_stages_draft = 0, n_resid_full = 0, n_resid_draft = 0;
     std::vector<cudaEvent_t> events;
     size_t events_used = 0;
     struct Span { int kind; size_t e0, e1; };
@@ -349,9 +350,12 @@ static int build_stage_tables(asd_ctx* x) {
     float* cosv = x->at<float>(ly.cosv);
     const CUtensorMap* maps = x->at<CUtensorMap>(ly.tmaps);
     std::vector<StageDesc> tab((size_t)2 * ly.max_stages);
+    const int max_resid = 2 * std::max(L, 1);
+    std::vector<ResidOut> resid((size_t)2 * max_resid);
     for (int which = 0; which < 2; ++which) {
         StageDesc* t = tab.data() + (size_t)which * ly.max_stages;
-        int n = 0;
+        int n = 0, nr = 0;
+        ResidOut* ro = resid.data() + (size_t)which * max_resid;
         t[n] = StageDesc{};
         t[n++].type = kStEmbed;
         for (int l = 0; l < L; ++l) {
@@ -373,8 +377,8 @@ static int build_stage_tables(asd_ctx* x) {
                 StageDesc o{};
                 o.type = kStOproj, o.layer = l, o.n_rows = d, o.n_in = d;
                 o.W = lw + ly.l_wo;
-                o.cos_out = cosv + (size_t)(0 * L + l) * kMaxRows;
-                o.sumcos = x->at<double>(ly.sumcos) + l;
+                o.resid_slot = nr;
+                ro[nr++] = ResidOut{cosv + (size_t)(0 * L + l) * kMaxRows, x->at<double>(ly.sumcos) + l};
                 t[n++] = o;
             }
             if (!(which && x->skip_mlp[l])) {
@@ -386,19 +390,24 @@ static int build_stage_tables(asd_ctx* x) {
                 StageDesc w{};
                 w.type = kStDown, w.layer = l, w.n_rows = d, w.n_in = f;
                 w.W = lw + ly.l_wd;
-                w.cos_out = cosv + (size_t)(1 * L + l) * kMaxRows;
-                w.sumcos = x->at<double>(ly.sumcos) + L + l;
+                w.resid_slot = nr;
+                ro[nr++] = ResidOut{cosv + (size_t)(1 * L + l) * kMaxRows, x->at<double>(ly.sumcos) + L + l};
                 t[n++] = w;
             }
         }
+        StageDesc fin{};  // turns the residual stages' partial sums into cosine similarities
+        fin.type = kStFinish, fin.layer = L;
+        t[n++] = fin;
         StageDesc h{};
         h.type = kStLmHead, h.layer = L, h.n_rows = c.vocab, h.n_in = d;
         h.W = x->ws + ly.lm_head;
         h.gain = x->at<__nv_bfloat16>(ly.final_norm);
         t[n++] = h;
         (which ? x->n_stages_draft : x->n_stages_full) = n;
+        (which ? x->n_resid_draft : x->n_resid_full) = nr;
     }
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.stage_tab, tab.data(), tab.size() * sizeof(StageDesc), cudaMemcpyHostToDevice, x->stream));
+    ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.resid_tab, resid.data(), resid.size() * sizeof(ResidOut), cudaMemcpyHostToDevice, x->stream));
     return ASD_OK;
 }
 
@@ -439,6 +448,8 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.attn_counters = x->at<unsigned>(ly.counters) + 64;
     p.chunk_stride = ly.chunk_stride;
     p.partials = x->at<float>(ly.partials);
+    p.resid = x->at<ResidOut>(ly.resid_tab) + (size_t)(use_mask ? 1 : 0) * (2 * std::max(L, 1));
+    p.n_resid = use_mask ? x->n_resid_draft : x->n_resid_full;
     p.fin_counter = words + 0;
     p.grid_bar = words + 16;
     p.err = reinterpret_cast<int*>(words + 32);

@@ -42,7 +42,7 @@ constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
 constexpr int kXsBudget = 40960;                    // bytes of shared memory for the activation window / attention scratch
 
-enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead };
+enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead, kStFinish };
 
 struct StageDesc {
     int type, layer;
@@ -51,8 +51,13 @@ struct StageDesc {
     const __nv_bfloat16* gain;
     __nv_bfloat16 *k_cache, *v_cache;   // this layer's cache [max_seq, kv_dim]
     const CUtensorMap *tm_k, *tm_v;     // tensor maps over the same
-    float* cos_out;                     // [kMaxRows] cosine of this sublayer, per row
-    double* sumcos;                     // running sum over prompt rows
+    int resid_slot;                     // residual stages: which block of per-CTA partial sums they write
+};
+
+// where the cosine similarity of one residual stage goes (filled in by the finish stage of the pass)
+struct ResidOut {
+    float* cos_out;  // [kMaxRows] cosine of this sublayer, per row
+    double* sumcos;  // running sum over prompt rows
 };
 
 struct PassParams {
@@ -67,7 +72,9 @@ struct PassParams {
     float *part_acc, *part_ml;
     unsigned* attn_counters;
     int chunk_stride;
-    float* partials;
+    float* partials;        // [n_resid + 1][gridDim.x][kMaxRows][4] per-CTA partial sums (last block: LM head)
+    const ResidOut* resid;  // [n_resid] outputs of the residual stages of this pass, in stage order
+    int n_resid;
     unsigned* fin_counter;
     unsigned* grid_bar;
     unsigned bar_base;
@@ -210,7 +217,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     int n_issued = 0;
     for (int s = 0; s < p.n_stages; ++s) {
         const StageDesc st = p.stages[s];
-        if (st.type == kStEmbed) continue;
+        if (st.type == kStEmbed || st.type == kStFinish) continue;
         if (st.type == kStAttn) {
             int n_chunks;
             const int n_local = attn_local_items(p, M, n_chunks);
@@ -272,6 +279,18 @@ __device__ __forceinline__ long long global_ns() {
 // per-stage timeline of every CTA (debugging aid): 0 = stage entered, 1 = inputs ready, 2 = streaming done, 3 = stage left
 __device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k) {
     if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 6 + k) * gridDim.x + blockIdx.x] = global_ns();
+}
+
+// Sum a and b over the warp with 5 shuffles instead of 10: after the first exchange the lower half-warp carries
+// a and the upper half-warp carries b. Each value goes through exactly the additions of a plain xor butterfly
+// (16, 8, 4, 2, 1), so the result is bit-identical to it. a's total is valid in lanes 0..15, b's in lanes 16..31.
+__device__ __forceinline__ float warp_sum_pair(float a, float b, int lane) {
+    const bool upper = (lane & 16) != 0;
+    const float keep = upper ? b : a, give = upper ? a : b;
+    float v = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
 }
 
 // ============================================================================================ grid barrier
@@ -432,21 +451,18 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 }
                 __syncwarp();
                 if (lane == 0) ring_release(p, sm, g);
-                float va[M], vb[M];
+                float vab[M];
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
-                    float e, o;
-                    unpack2(acc_a[m], e, o);
-                    va[m] = warp_sum(e + o);
-                    unpack2(acc_b[m], e, o);
-                    vb[m] = warp_sum(e + o);
+                    float ea, oa, eb, ob;
+                    unpack2(acc_a[m], ea, oa);
+                    unpack2(acc_b[m], eb, ob);
+                    vab[m] = warp_sum_pair(ea + oa, eb + ob, lane);
                 }
-                if (lane == 0) {  // segments of a pair are added in ascending order, always by this warp
+                if ((lane & 15) == 0) {  // lane 0 holds row a, lane 16 row b; segments are added in ascending order
+                    const int r = lane >> 4;
 #pragma unroll
-                    for (int m = 0; m < M; ++m) {
-                        psum[(pl * 2 + 0) * M + m] += va[m];
-                        psum[(pl * 2 + 1) * M + m] += vb[m];
-                    }
+                    for (int m = 0; m < M; ++m) psum[(pl * 2 + r) * M + m] += vab[m];
                 }
                 if (p.trace) {
                     cyc_wait += tw1 - tw0;
@@ -542,7 +558,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     if (type == kStOproj || type == kStDown) {
         // cosine similarity of the hidden state before and after this sublayer: warp-shuffle partial dot and
-        // norm products, one block-level finish, per-CTA partials combined by the last CTA to arrive
+        // norm products, one block-level finish; the per-CTA partials are combined by the finish stage of the pass
 #pragma unroll
         for (int m = 0; m < M; ++m)
 #pragma unroll
@@ -556,39 +572,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             float tot = 0.f;
 #pragma unroll
             for (int w = 0; w < kPassConsumerWarps; ++w) tot += red[w * (kMaxRows * 4) + m * 4 + j];
-            p.partials[((size_t)blockIdx.x * kMaxRows + m) * 4 + j] = tot;
-        }
-        if (last_cta_consumers(p.fin_counter, sm.flag)) {
-            // one warp per activation row: lanes add the per-CTA partials b = lane, lane+32, ... in order, then an
-            // xor butterfly in double precision (fixed order, independent of the row count)
-            if (warp < M) {
-                double sxy = 0, sxx = 0, syy = 0;
-                for (unsigned b = lane; b < gridDim.x; b += 32) {
-                    sxy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 0);
-                    sxx += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 1);
-                    syy += (double)__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 2);
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    sxy += __shfl_xor_sync(0xffffffffu, sxy, o);
-                    sxx += __shfl_xor_sync(0xffffffffu, sxx, o);
-                    syy += __shfl_xor_sync(0xffffffffu, syy, o);
-                }
-                if (lane == 0) {
-                    const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
-                    st.cos_out[warp] = (float)c;
-                    red[warp] = (float)c;
-                }
-            }
-            consumers_sync();
-            if (tid == 0) {
-                if (p.acc_sim && st.sumcos) {
-                    double acc = *st.sumcos;
-                    for (int m = 0; m < M; ++m) acc += (double)red[m];
-                    *st.sumcos = acc;
-                }
-                *p.fin_counter = 0u;
-            }
+            p.partials[(((size_t)st.resid_slot * gridDim.x + blockIdx.x) * kMaxRows + m) * 4 + j] = tot;
         }
     } else if (type == kStLmHead) {
 #pragma unroll
@@ -621,17 +605,19 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     i = oi;
                 }
             }
-            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 0] = v;
-            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 1] = __int_as_float(i);
+            float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kMaxRows * 4;
+            lmp[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 0] = v;
+            lmp[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 1] = __int_as_float(i);
         }
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
             int* g = reinterpret_cast<int*>(red);
             if (warp < M) {  // one warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index
                 float v = -INFINITY;
                 int i = INT_MAX;
+                const float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kMaxRows * 4;
                 for (unsigned b = lane; b < gridDim.x; b += 32) {
-                    const float ov = __ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 0);
-                    const int oi = __float_as_int(__ldcg(p.partials + ((size_t)b * kMaxRows + warp) * 4 + 1));
+                    const float ov = __ldcg(lmp + ((size_t)b * kMaxRows + warp) * 4 + 0);
+                    const int oi = __float_as_int(__ldcg(lmp + ((size_t)b * kMaxRows + warp) * 4 + 1));
                     if (ov > v || (ov == v && oi < i)) {
                         v = ov;
                         i = oi;
@@ -665,6 +651,45 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 *p.fin_counter = 0u;
             }
         }
+    }
+}
+
+// ============================================================================================ finish stage
+// Cosine similarities of all residual stages of the pass (summand of C_l, Section 3.2). Residual stage r is
+// finished by CTA r mod gridDim.x: one warp per activation row adds the per-CTA partials b = lane, lane+32, ...
+// in order, then an xor butterfly, all in double precision (fixed order, independent of the row count).
+template <int M>
+__device__ void finish_stage(const PassParams& p, const PassSmem& sm) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int r = blockIdx.x; r < p.n_resid; r += gridDim.x) {
+        const float* part = p.partials + (size_t)r * gridDim.x * kMaxRows * 4;
+        const ResidOut out = p.resid[r];
+        if (warp < M) {
+            double sxy = 0, sxx = 0, syy = 0;
+            for (unsigned b = lane; b < gridDim.x; b += 32) {
+                sxy += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 0);
+                sxx += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 1);
+                syy += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 2);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                sxy += __shfl_xor_sync(0xffffffffu, sxy, o);
+                sxx += __shfl_xor_sync(0xffffffffu, sxx, o);
+                syy += __shfl_xor_sync(0xffffffffu, syy, o);
+            }
+            if (lane == 0) {
+                const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
+                out.cos_out[warp] = (float)c;
+                sm.red[warp] = (float)c;
+            }
+        }
+        consumers_sync();
+        if (tid == 0 && p.acc_sim && out.sumcos) {  // rows are added in order: chunked prefill equals one-shot prefill
+            double acc = *out.sumcos;
+            for (int m = 0; m < M; ++m) acc += (double)sm.red[m];
+            *out.sumcos = acc;
+        }
+        consumers_sync();
     }
 }
 
@@ -864,16 +889,26 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                     for (int m = 0; m < M; ++m) {
                         const int nc = (p.pos0 + m) / kAttnChunk + 1;
                         float mx = -INFINITY, l = 0.f, acc = 0.f;
-                        for (int c = 0; c < nc; ++c) {
-                            const size_t b = ((size_t)head * p.chunk_stride + c) * kMaxRows + m;
-                            const float cm = __ldcg(p.part_ml + b * 2 + 0);
-                            const float cl = __ldcg(p.part_ml + b * 2 + 1);
-                            const float pa = __ldcg(p.part_acc + b * hd + e);
-                            const float mn = fmaxf(mx, cm);
-                            const float s_old = expf(mx - mn), s_new = expf(cm - mn);
-                            acc = acc * s_old + pa * s_new;
-                            l = l * s_old + cl * s_new;
-                            mx = mn;
+                        for (int c0 = 0; c0 < nc; c0 += 8) {  // loads of a batch are independent; the merge stays in chunk order
+                            float cm[8], cl[8], pa[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const int c = min(c0 + i, nc - 1);
+                                const size_t b = ((size_t)head * p.chunk_stride + c) * kMaxRows + m;
+                                cm[i] = __ldcg(p.part_ml + b * 2 + 0);
+                                cl[i] = __ldcg(p.part_ml + b * 2 + 1);
+                                pa[i] = __ldcg(p.part_acc + b * hd + e);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (c0 + i < nc) {
+                                    const float mn = fmaxf(mx, cm[i]);
+                                    const float s_old = expf(mx - mn), s_new = expf(cm[i] - mn);
+                                    acc = acc * s_old + pa[i] * s_new;
+                                    l = l * s_old + cl[i] * s_new;
+                                    mx = mn;
+                                }
+                            }
                         }
                         p.a[(size_t)m * p.d_model + (size_t)head * hd + e] = __float2bfloat16_rn(acc / l);
                     }
@@ -927,6 +962,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
                 t = min(max(t, 0), p.vocab - 1);
                 p.x[i] = __bfloat162float(p.embed[(size_t)t * d + e]);
             }
+        } else if (st.type == kStFinish) {
+            finish_stage<M>(p, sm);
         } else if (st.type == kStAttn) {
             attn_stage<M>(p, st, sm, gi, s);
         } else {

@@ -215,6 +215,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     volatile int* err = p.err;
     uint32_t gi = 0, issued[2] = {0, 0};
     int n_issued = 0;
+    const uint64_t pol_stream = make_policy_evict_first();  // weights are read once per pass: do not let them age in L2
     for (int s = 0; s < p.n_stages; ++s) {
         const StageDesc st = p.stages[s];
         if (st.type == kStEmbed || st.type == kStFinish) continue;
@@ -252,7 +253,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
             const uint32_t g = gi + (uint32_t)idx;
             const int slot = ring_acquire(p, sm, g, s, M);
             mbar_expect_tx(&sm.full[slot], kSlotBytes);
-            tma_load_1d(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)idx * kSlotBytes, kSlotBytes, &sm.full[slot]);
+            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)idx * kSlotBytes, kSlotBytes, &sm.full[slot], pol_stream);
             issued[1] = issued[0], issued[0] = g, ++n_issued;
         }
         gi += (uint32_t)n_items;
@@ -949,6 +950,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     }
 
     uint32_t gi = 0;
+    if (p.trace && threadIdx.x == 0) {  // which SM runs this CTA (entry 4 of the embedding stage, which streams nothing)
+        unsigned smid;
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        p.trace[((size_t)0 * 6 + 4) * gridDim.x + blockIdx.x] = smid;
+    }
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);
         if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);

@@ -14,7 +14,7 @@
 
 namespace asd {
 
-constexpr int kPrefillRows = 8;  // prompt rows per pass of the chunked prefill
+constexpr int kPrefillRows = kPassMaxRows;  // prompt rows per pass of the chunked prefill
 constexpr size_t kAlign = 256;
 constexpr int kMaxGemvGrid = 1024;
 
@@ -55,6 +55,7 @@ static cudaError_t launch_pass(int M, const PassParams& p, int grid, size_t smem
         case 7: return launch_pass_m7(p, grid, smem, s);
         case 8: return launch_pass_m8(p, grid, smem, s);
         case 9: return launch_pass_m9(p, grid, smem, s);
+        case 16: return launch_pass_m16(p, grid, smem, s);
     }
     return cudaErrorInvalidValue;
 }
@@ -84,6 +85,7 @@ static cudaError_t device_info(DeviceInfo** out) {
         if ((e = configure_m7(d.max_smem)) != cudaSuccess) return e;
         if ((e = configure_m8(d.max_smem)) != cudaSuccess) return e;
         if ((e = configure_m9(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_m16(d.max_smem)) != cudaSuccess) return e;
         d.ready = true;
     }
     *out = &d;
@@ -122,9 +124,9 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
     const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
     const size_t psum = ((size_t)np_max * 2 * M * 4 + 15) & ~(size_t)15;
-    const size_t misc = ((size_t)16 * kMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
-    const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16 + 15) & ~(size_t)15;
-    const size_t xs = (size_t)M * pass_wseg(M) * kSeg * 2;
+    const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
+    const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
+    const size_t xs = (size_t)M * ((size_t)pass_wseg(M) * kSegK + kXsPad) * 2;
     const size_t reg_a = (std::max(xs, 2 * attn_scratch) + 15) & ~(size_t)15;
     const long long avail = (long long)dv.max_smem - 1024 - (long long)(psum + misc + reg_a) - 2 * 64 * 8;
     int ns = (int)std::min<long long>(64, avail / kSlotBytes);
@@ -166,8 +168,8 @@ static bool check_config(const asd_config& c) {
     return true;
 }
 
-// bytes of a matrix in the packed layout of the pass kernel: (pairs of rows) x (segments of 1024 inputs) x 4 KB
-static size_t packed_bytes(size_t n_rows, size_t n_in) { return ((n_rows + 1) / 2) * ((n_in + kSeg - 1) / kSeg) * (size_t)kSlotBytes; }
+// bytes of a matrix in the packed layout of the pass kernel: (pairs of rows) x (segments of 256 inputs) x 1 KB
+static size_t packed_bytes(size_t n_rows, size_t n_in) { return ((n_rows + 1) / 2) * ((n_in + kSegK - 1) / kSegK) * (size_t)1024; }
 
 static Layout make_layout(const asd_config& c) {
     Layout L{};
@@ -202,16 +204,16 @@ static Layout make_layout(const asd_config& c) {
     L.kv_layer_stride = align_up(S * kvd * 2);
     L.kcache = take(L.kv_layer_stride * c.n_layers);
     L.vcache = take(L.kv_layer_stride * c.n_layers);
-    L.x = take(kMaxRows * d * 4);
-    L.q = take(kMaxRows * d * 2);
-    L.a = take(kMaxRows * d * 2);
-    L.t = take(kMaxRows * f * 2);
+    L.x = take(kPassMaxRows * d * 4);
+    L.q = take(kPassMaxRows * d * 2);
+    L.a = take(kPassMaxRows * d * 2);
+    L.t = take(kPassMaxRows * f * 2);
     L.chunk_stride = (int)((S + kAttnChunk - 1) / kAttnChunk);
-    L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * c.head_dim * 4);
-    L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kMaxRows * 2 * 4);
-    L.partials = take((size_t)(2 * c.n_layers + 1) * kMaxGemvGrid * kMaxRows * 4 * 4);
+    L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * c.head_dim * 4);
+    L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * 2 * 4);
+    L.partials = take((size_t)(2 * c.n_layers + 1) * kMaxGemvGrid * kPassMaxRows * 4 * 4);
     L.counters = take((size_t)(c.n_kv_heads + 64) * 4);
-    L.cosv = take((size_t)2 * std::max(c.n_layers, 1) * kMaxRows * 4);
+    L.cosv = take((size_t)2 * std::max(c.n_layers, 1) * kPassMaxRows * 4);
     L.sumcos = take((size_t)2 * std::max(c.n_layers, 1) * 8);
     L.tok_in = take(64 * 4);
     L.draft_toks = take(64 * 4);
@@ -219,7 +221,7 @@ static Layout make_layout(const asd_config& c) {
     L.prompt_toks = take((S + 16) * 4);
     L.argmax = take(64 * 4);
     L.accept = take(64 * 4);
-    L.logits = take((size_t)kMaxRows * V * 4);
+    L.logits = take((size_t)kPassMaxRows * V * 4);
     L.max_stages = 5 * c.n_layers + 3;
     L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
@@ -378,7 +380,7 @@ static int build_stage_tables(asd_ctx* x) {
                 o.type = kStOproj, o.layer = l, o.n_rows = d, o.n_in = d;
                 o.W = lw + ly.l_wo;
                 o.resid_slot = nr;
-                ro[nr++] = ResidOut{cosv + (size_t)(0 * L + l) * kMaxRows, x->at<double>(ly.sumcos) + l};
+                ro[nr++] = ResidOut{cosv + (size_t)(0 * L + l) * kPassMaxRows, x->at<double>(ly.sumcos) + l};
                 t[n++] = o;
             }
             if (!(which && x->skip_mlp[l])) {
@@ -391,7 +393,7 @@ static int build_stage_tables(asd_ctx* x) {
                 w.type = kStDown, w.layer = l, w.n_rows = d, w.n_in = f;
                 w.W = lw + ly.l_wd;
                 w.resid_slot = nr;
-                ro[nr++] = ResidOut{cosv + (size_t)(1 * L + l) * kMaxRows, x->at<double>(ly.sumcos) + L + l};
+                ro[nr++] = ResidOut{cosv + (size_t)(1 * L + l) * kPassMaxRows, x->at<double>(ly.sumcos) + L + l};
                 t[n++] = w;
             }
         }
@@ -420,13 +422,13 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     const Layout& ly = x->lay;
     const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
     cudaStream_t s = x->stream;
-    if (M < 1 || M > kMaxRows) return fail(x, ASD_ERR_ARG, "row count out of range");
+    if (M < 1 || (M > kMaxRows && M != kPassMaxRows)) return fail(x, ASD_ERR_ARG, "row count out of range");
     if ((long long)pos0 + M > c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "pass would exceed max_seq positions");
     PassPlan pl;
     if (!plan_pass(*x->dev, c, M, &pl)) return fail(x, ASD_ERR_ARG, "decoder shape does not fit the pass kernel's shared-memory plan");
 
     float* cosv = x->at<float>(ly.cosv);
-    ASD_CUDA(x, cudaMemsetAsync(cosv, 0xFF, (size_t)2 * std::max(L, 1) * kMaxRows * 4, s));  // NaN = skipped
+    ASD_CUDA(x, cudaMemsetAsync(cosv, 0xFF, (size_t)2 * std::max(L, 1) * kPassMaxRows * 4, s));  // NaN = skipped
 
     unsigned* words = x->at<unsigned>(ly.sync_words);
     PassParams p{};
@@ -549,7 +551,7 @@ extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t byt
     if (e != cudaSuccess) return bail(e);
     {
         PassPlan pl;
-        if (!plan_pass(*x->dev, *cfg, kMaxRows, &pl) || !plan_pass(*x->dev, *cfg, 1, &pl)) {
+        if (!plan_pass(*x->dev, *cfg, kPassMaxRows, &pl) || !plan_pass(*x->dev, *cfg, 1, &pl)) {
             delete x;
             return ASD_ERR_ARG;
         }
@@ -598,26 +600,38 @@ extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : 
 
 // Repack one matrix into the pass kernel's layout and copy it to the device. The logical matrix has n_rows
 // rows of n_in inputs; row(r) returns the host pointer of logical row r. CTA b of a G-CTA grid owns pairs
-// [b*P/G, (b+1)*P/G); its slab is segment-major (for seg: for pair: 2 x 2 KB), ragged ends zero padded.
+// [b*P/G, (b+1)*P/G) in octets of four pairs (the last may be smaller); its slab is segment-major (for each
+// segment of 256 inputs: for each octet), and an item of R rows is 8 column blocks of 32 inputs, each block
+// R rows x 64 bytes. Inputs past n_in are zero.
 template <class RowFn, class PairFn>
 static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, PairFn pair_rows_of,
                          std::vector<unsigned char>& staging) {
-    const size_t n_pairs = (n_rows + 1) / 2, n_seg = (n_in + kSeg - 1) / kSeg;
-    const size_t total = n_pairs * n_seg * kSlotBytes;
+    const size_t n_pairs = (n_rows + 1) / 2, n_seg = (n_in + kSegK - 1) / kSegK;
+    const size_t total = n_pairs * n_seg * 1024;
     const int G = x->dev->num_sms;
     staging.assign(total, 0);
 #pragma omp parallel for schedule(static)
     for (int b = 0; b < G; ++b) {
         const size_t pair0 = (size_t)b * n_pairs / G, pair1 = (size_t)(b + 1) * n_pairs / G, np = pair1 - pair0;
-        unsigned char* slab = staging.data() + pair0 * n_seg * kSlotBytes;
+        unsigned char* slab = staging.data() + pair0 * n_seg * 1024;
         for (size_t sg = 0; sg < n_seg; ++sg) {
-            const size_t k0 = sg * kSeg, len = std::min<size_t>(kSeg, n_in - k0);
-            for (size_t pl = 0; pl < np; ++pl) {
-                size_t ra, rb;
-                pair_rows_of(pair0 + pl, ra, rb);
-                unsigned char* item = slab + (sg * np + pl) * kSlotBytes;
-                memcpy(item, row(ra) + k0, len * 2);
-                if (rb < n_rows) memcpy(item + kSlotBytes / 2, row(rb) + k0, len * 2);
+            for (size_t o = 0; o * 4 < np; ++o) {
+                const size_t pairs = std::min<size_t>(4, np - 4 * o), R = 2 * pairs;
+                unsigned char* item = slab + sg * np * 1024 + o * kSlotBytes;
+                for (size_t pq = 0; pq < pairs; ++pq) {
+                    size_t rr[2];
+                    pair_rows_of(pair0 + 4 * o + pq, rr[0], rr[1]);
+                    for (int h = 0; h < 2; ++h) {
+                        if (rr[h] >= n_rows) continue;
+                        const uint16_t* src = row(rr[h]);
+                        const size_t g = 2 * pq + h;
+                        for (size_t j = 0; j < 8; ++j) {
+                            const size_t k = sg * kSegK + j * 32;
+                            if (k >= n_in) break;
+                            memcpy(item + j * (R * 64) + g * 64, src + k, std::min<size_t>(32, n_in - k) * 2);
+                        }
+                    }
+                }
             }
         }
     }
@@ -723,8 +737,10 @@ static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int3
     int rc = new_event(x, &e0);
     if (rc) return rc;
     int last_rows = 0;
-    for (int c0 = 0; c0 < n; c0 += kPrefillRows) {
-        const int M = std::min(kPrefillRows, n - c0);
+    for (int c0 = 0, M = 0; c0 < n; c0 += M) {
+        // row counts the pass kernel is built for: 16, or 1..9
+        const int left = n - c0;
+        M = left >= kPrefillRows ? kPrefillRows : (left > kMaxRows ? 8 : left);
         const bool last = c0 + M >= n;
         rc = run_pass(x, M, x->n_committed + c0, dev_tokens + c0, false, true, last, nullptr, false, nullptr);
         if (rc) return rc;
@@ -899,7 +915,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
     const bool need_host_token = gp->eos_id >= 0;
     rc = prefill_device(x, dev_prompt, n_prompt, need_host_token ? &first : nullptr, false);
     if (rc) return rc;
-    const int last_rows = (n_prompt - 1) % kPrefillRows + 1;
+    const int last_rows = x->last_M;  // rows of the last prefill pass
     ASD_CUDA(x, cudaMemcpyAsync(dev_out, x->at<int>(x->lay.argmax) + (last_rows - 1), 4, cudaMemcpyDeviceToDevice, s));
     int produced = 1;
     bool stop = need_host_token && first == gp->eos_id;
@@ -998,13 +1014,13 @@ extern "C" int asd_get_last_cosines(asd_ctx* x, int32_t* M, float* cos_attn, flo
     if (x->last_M == 0) return fail(x, ASD_ERR_STATE, "no pass has run");
     const int L = x->c.n_layers, m = x->last_M;
     if (M) *M = m;
-    std::vector<float> h((size_t)2 * std::max(L, 1) * kMaxRows);
+    std::vector<float> h((size_t)2 * std::max(L, 1) * kPassMaxRows);
     ASD_CUDA(x, cudaMemcpyAsync(h.data(), x->ws + x->lay.cosv, h.size() * 4, cudaMemcpyDeviceToHost, x->stream));
     ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     for (int l = 0; l < L; ++l)
         for (int r = 0; r < m; ++r) {
-            if (cos_attn) cos_attn[(size_t)l * m + r] = h[((size_t)0 * L + l) * kMaxRows + r];
-            if (cos_mlp) cos_mlp[(size_t)l * m + r] = h[((size_t)1 * L + l) * kMaxRows + r];
+            if (cos_attn) cos_attn[(size_t)l * m + r] = h[((size_t)0 * L + l) * kPassMaxRows + r];
+            if (cos_mlp) cos_mlp[(size_t)l * m + r] = h[((size_t)1 * L + l) * kPassMaxRows + r];
         }
     return ASD_OK;
 }

@@ -6,7 +6,8 @@
 
 namespace asd {
 
-constexpr int kMaxRows = 9;        // rows per pass: max draft length 8, plus the last accepted token
+constexpr int kMaxRows = 9;        // rows of the stand-alone fused GEMV: max draft length 8, plus the last accepted token
+constexpr int kPassMaxRows = 16;   // rows of one pass of the persistent kernel (prefill feeds the prompt 16 rows at a time)
 constexpr int kGemvThreads = 512;  // 16 warps per CTA, one CTA per SM
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kSeg = 1024;         // elements of the reduction dimension per warp work item
@@ -55,6 +56,8 @@ ASD_DECLARE_LAUNCHERS(6)
 ASD_DECLARE_LAUNCHERS(7)
 ASD_DECLARE_LAUNCHERS(8)
 ASD_DECLARE_LAUNCHERS(9)
+cudaError_t launch_pass_m16(const PassParams& p, int grid, size_t smem, cudaStream_t s);
+cudaError_t configure_m16(int max_smem);
 
 size_t gemv_smem_bytes(int M, int n_rows, int n_in, int grid, bool x_in_smem);
 

@@ -1,4 +1,5 @@
-// Instantiations of the row-count-templated kernels; compiled once per ASD_M in 1..9.
+// Instantiations of the row-count-templated kernels; compiled once per ASD_M in 1..9 (both kernels) and 16 (pass
+// kernel only: the row count of a prefill pass).
 #include "gemv.cuh"
 #include "pass.cuh"
 
@@ -11,6 +12,7 @@ namespace asd {
 #define ASD_CAT2(a, b) a##b
 #define ASD_CAT(a, b) ASD_CAT2(a, b)
 
+#if ASD_M <= 9
 template <int EPI, bool NORM>
 static cudaError_t launch_one(const GemvParams& p, int grid, size_t smem, cudaStream_t s) {
     gemv_kernel<ASD_M, EPI, NORM><<<grid, kGemvThreads, smem, s>>>(p);
@@ -25,6 +27,7 @@ cudaError_t ASD_CAT(launch_gemv_m, ASD_M)(int epi, bool norm, const GemvParams& 
     }
     return cudaErrorInvalidValue;
 }
+#endif
 
 cudaError_t ASD_CAT(launch_pass_m, ASD_M)(const PassParams& p, int grid, size_t smem, cudaStream_t s) {
     void* args[] = {const_cast<PassParams*>(&p)};
@@ -38,12 +41,14 @@ cudaError_t ASD_CAT(configure_m, ASD_M)(int max_smem) {
 #define ASD_SET(k)                                                                              \
     e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);         \
     if (e != cudaSuccess) return e;
+#if ASD_M <= 9
     ASD_SET((gemv_kernel<ASD_M, kEpiPlain, true>))
     ASD_SET((gemv_kernel<ASD_M, kEpiPlain, false>))
     ASD_SET((gemv_kernel<ASD_M, kEpiSwiglu, true>))
     ASD_SET((gemv_kernel<ASD_M, kEpiSwiglu, false>))
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, true>))
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, false>))
+#endif
     ASD_SET((pass_kernel<ASD_M>))
 #undef ASD_SET
     return cudaSuccess;

@@ -12,23 +12,29 @@
 //     contiguous byte range;
 //   * 15 consumer warps wait for the previous stage of all CTAs (a grid barrier on a monotonically increasing
 //     counter, bounded spin), stage the activations in shared memory (RMSNorm fused), multiply the ring slots
-//     with packed fp32 FMAs, and run the epilogue: RoPE + KV append, SwiGLU, residual add + cosine
+//     on the tensor cores, and run the epilogue: RoPE + KV append, SwiGLU, residual add + cosine
 //     similarity (summand of C_l, Section 3.2), LM-head argmax + greedy acceptance (Section 1).
 // Sublayers in the skip mask (the draft model D, Algorithm 1) simply do not appear in the stage table: no
 // weights are streamed and no K/V is touched for them.
 //
 // Packed weights: a matrix [n_rows, n_in] is cut into PAIRS of rows (the two rotary partners of a q/k head,
-// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 1024 inputs. One ring item = one pair x one
-// segment = 2 x 2 KB = one 4 KB slot (a ragged last segment is zero padded). CTA b owns pairs
-// [b*P/G, (b+1)*P/G); its slab is stored segment-major: for seg: for pair: item. Consecutive ring items thus
-// belong to different pairs, i.e. to different consumer warps, and are consumed as soon as they land.
+// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 256 inputs. CTA b owns pairs [b*P/G, (b+1)*P/G)
+// and groups them into OCTETS of four pairs (the last octet may hold fewer). One ring item = one octet x one
+// segment = up to 8 rows x 512 bytes = one 4 KB slot, stored as 8 column blocks of 32 inputs. The CTA's slab is
+// segment-major (for seg: for octet), so consecutive ring items belong to different consumer warps and are
+// consumed as soon as they land, and no byte of padding crosses HBM for shapes whose input size is a multiple
+// of 256.
 //
-// Reduction order is fixed and independent of the row count M: per (weight row, activation row) a lane adds
-// the even and the odd elements of its 16-byte chunks of a 1024-element segment in order, the two halves are
-// added, lanes are combined by an xor butterfly, segments are added in ascending order. Attention chunks are
-// aligned to absolute positions and merged in order. Row m of a (k+1)-row verify pass is therefore
-// bit-identical to a 1-row decode pass at the same position, so speculative output equals autoregressive
-// output bit for bit.
+// The products run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate): the activation rows are the
+// 16-row A operand, the 8 weight rows of an item the B operand, so one step serves any row count up to 16 and
+// the arithmetic of a row does not depend on how many rows share the pass. tcgen05 is not used here on
+// purpose: its smallest tile (64 weight rows) does not fit a 148-way row split that leaves ~28 rows of the
+// d x d matrices to a CTA, and its A operand would need the activations padded to 64+ rows in shared memory.
+//
+// Reduction order is fixed and independent of the row count M: an item's 16 steps alternate between two
+// accumulators that are added at the end, segments are added in ascending order. Attention chunks are aligned
+// to absolute positions and merged in order. Row m of a (k+1)-row verify pass is therefore bit-identical to
+// a 1-row decode pass at the same position, so speculative output equals autoregressive output bit for bit.
 #pragma once
 #include <limits.h>
 
@@ -56,7 +62,7 @@ struct StageDesc {
 
 // where the cosine similarity of one residual stage goes (filled in by the finish stage of the pass)
 struct ResidOut {
-    float* cos_out;  // [kMaxRows] cosine of this sublayer, per row
+    float* cos_out;  // [kPassMaxRows] cosine of this sublayer, per row
     double* sumcos;  // running sum over prompt rows
 };
 
@@ -72,7 +78,7 @@ struct PassParams {
     float *part_acc, *part_ml;
     unsigned* attn_counters;
     int chunk_stride;
-    float* partials;        // [n_resid + 1][gridDim.x][kMaxRows][4] per-CTA partial sums (last block: LM head)
+    float* partials;        // [n_resid + 1][gridDim.x][kPassMaxRows][4] per-CTA partial sums (last block: LM head)
     const ResidOut* resid;  // [n_resid] outputs of the residual stages of this pass, in stage order
     int n_resid;
     unsigned* fin_counter;
@@ -94,16 +100,28 @@ struct PassParams {
     int off_bars, off_misc, off_psum, off_reg_a;
 };
 
-// segments of the reduction dimension whose activations (M rows, bf16) fit the shared-memory window
+constexpr int kSegK = 256;     // inputs per ring item
+constexpr int kOctRows = 8;    // weight rows per ring item (four pairs): the N of one m16n8k16 tensor-core step
+constexpr int kXsPad = 32;     // bf16 elements of padding per activation row (64 bytes: conflict-free 16-byte reads)
+
+// 256-input segments whose activations (M rows, bf16, padded rows) fit the shared-memory window
 __host__ __device__ inline int pass_wseg(int M) {
-    const int w = kXsBudget / (M * 2048);
+    const int w = (kXsBudget / M - kXsPad * 2) / (kSegK * 2);
     return w < 1 ? 1 : w;
+}
+
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col): one warp-wide tensor-core step
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 struct PassSmem {
     unsigned char* ring;
     uint64_t *full, *empty;
-    float* red;   // [16][kMaxRows*4]
+    float* red;   // [16][kPassMaxRows*4]
     int* flag;    // [8]
     volatile unsigned* consumed;  // [64] generations of each ring slot that consumers have finished with
     float* psum;
@@ -243,17 +261,21 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
             gi += (uint32_t)n_items;
             continue;
         }
-        // GEMV stage: this CTA's slab is contiguous and already in ring order
+        // GEMV stage: this CTA's slab is contiguous and already in ring order (segment-major, octets inside)
         int pair0, np;
         cta_pairs(st.n_rows, pair0, np);
-        const int n_seg = (st.n_in + kSeg - 1) / kSeg;
-        const int n_items = np * n_seg;
-        const unsigned char* slab = st.W + (size_t)pair0 * n_seg * kSlotBytes;
+        const int n_seg = (st.n_in + kSegK - 1) / kSegK;
+        const int n_oct = (np + 3) >> 2;
+        const int n_items = n_oct * n_seg;
+        const unsigned char* slab = st.W + (size_t)pair0 * n_seg * 1024;
         for (int idx = lane; idx < n_items; idx += 32) {
+            const int seg = idx / n_oct, o = idx - seg * n_oct;
+            const uint32_t bytes = (uint32_t)min(4, np - 4 * o) * 1024u;  // pairs of this octet x 2 rows x 512 bytes
             const uint32_t g = gi + (uint32_t)idx;
             const int slot = ring_acquire(p, sm, g, s, M);
-            mbar_expect_tx(&sm.full[slot], kSlotBytes);
-            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)idx * kSlotBytes, kSlotBytes, &sm.full[slot], pol_stream);
+            mbar_expect_tx(&sm.full[slot], bytes);
+            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)seg * np * 1024 + (size_t)o * kSlotBytes, bytes,
+                             &sm.full[slot], pol_stream);
             issued[1] = issued[0], issued[0] = g, ++n_issued;
         }
         gi += (uint32_t)n_items;
@@ -280,18 +302,6 @@ __device__ __forceinline__ long long global_ns() {
 // per-stage timeline of every CTA (debugging aid): 0 = stage entered, 1 = inputs ready, 2 = streaming done, 3 = stage left
 __device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k) {
     if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 6 + k) * gridDim.x + blockIdx.x] = global_ns();
-}
-
-// Sum a and b over the warp with 5 shuffles instead of 10: after the first exchange the lower half-warp carries
-// a and the upper half-warp carries b. Each value goes through exactly the additions of a plain xor butterfly
-// (16, 8, 4, 2, 1), so the result is bit-identical to it. a's total is valid in lanes 0..15, b's in lanes 16..31.
-__device__ __forceinline__ float warp_sum_pair(float a, float b, int lane) {
-    const bool upper = (lane & 16) != 0;
-    const float keep = upper ? b : a, give = upper ? a : b;
-    float v = keep + __shfl_xor_sync(0xffffffffu, give, 16);
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
 }
 
 // ============================================================================================ grid barrier
@@ -345,9 +355,10 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     const int n_in = st.n_in, n_rows = st.n_rows;
     int pair0, np;
     cta_pairs(n_rows, pair0, np);
-    const int n_seg = (n_in + kSeg - 1) / kSeg;
+    const int n_seg = (n_in + kSegK - 1) / kSegK;
+    const int n_oct = (np + 3) >> 2;
     const int wseg = pass_wseg(M);
-    const int xstride = wseg * kSeg;
+    const int xstride = wseg * kSegK + kXsPad;  // bf16 elements per activation row in the window
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
     float* red = sm.red;
     float* psum = sm.psum;
@@ -369,14 +380,14 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 s = fmaf(v.w, v.w, s);
             }
             s = warp_sum(s);
-            if (lane == 0) red[warp * (kMaxRows * 4) + m] = s;
+            if (lane == 0) red[warp * (kPassMaxRows * 4) + m] = s;
         }
         consumers_sync();
 #pragma unroll
         for (int m = 0; m < M; ++m) {
             float s = 0.f;
 #pragma unroll
-            for (int w = 0; w < kPassConsumerWarps; ++w) s += red[w * (kMaxRows * 4) + m];
+            for (int w = 0; w < kPassConsumerWarps; ++w) s += red[w * (kPassMaxRows * 4) + m];
             inv[m] = 1.0f / sqrtf(s / (float)n_in + p.eps);
         }
     }
@@ -384,86 +395,87 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     long long cyc_wait = 0, cyc_work = 0;  // when tracing: cycles this warp spent waiting for slots / working on them
     // ---- stream the slab window by window
+    const int g8 = lane >> 2, q4 = lane & 3;  // tensor-core fragment coordinates of this lane
     for (int w0 = 0; w0 < n_seg; w0 += wseg) {
         const int ws = min(wseg, n_seg - w0);
-        const int k0 = w0 * kSeg;
-        const int klen = min(n_in - k0, ws * kSeg);
+        const int k0 = w0 * kSegK;
+        const int wlen = ws * kSegK;  // inputs in this window, including the zero padding past n_in
         consumers_sync();  // previous window fully consumed; psum zeroed; red free
         if (norm) {
-            for (int i = tid * 4; i < klen; i += kPassConsumers * 4) {
-                const uint2 gv = *reinterpret_cast<const uint2*>(st.gain + k0 + i);
+            for (int i = tid * 4; i < wlen; i += kPassConsumers * 4) {
+                const bool in = k0 + i < n_in;
+                uint2 gv = make_uint2(0u, 0u);
+                if (in) gv = *reinterpret_cast<const uint2*>(st.gain + k0 + i);
                 const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + k0 + i));
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv[m] * g0, v.y * inv[m] * g1);
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv[m] * g2, v.w * inv[m] * g3);
-                    uint2 o;
-                    o.x = *reinterpret_cast<uint32_t*>(&lo);
-                    o.y = *reinterpret_cast<uint32_t*>(&hi);
+                    uint2 o = make_uint2(0u, 0u);
+                    if (in) {
+                        const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + k0 + i));
+                        __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv[m] * g0, v.y * inv[m] * g1);
+                        __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv[m] * g2, v.w * inv[m] * g3);
+                        o.x = *reinterpret_cast<uint32_t*>(&lo);
+                        o.y = *reinterpret_cast<uint32_t*>(&hi);
+                    }
                     *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
                 }
             }
         } else {
-            for (int i = tid * 8; i < klen; i += kPassConsumers * 8) {
+            for (int i = tid * 8; i < wlen; i += kPassConsumers * 8) {
+                const bool in = k0 + i < n_in;
 #pragma unroll
-                for (int m = 0; m < M; ++m)
-                    *reinterpret_cast<uint4*>(xs + (size_t)m * xstride + i) =
-                        __ldcg(reinterpret_cast<const uint4*>(xb + (size_t)m * n_in + k0 + i));
+                for (int m = 0; m < M; ++m) {
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (in) v = __ldcg(reinterpret_cast<const uint4*>(xb + (size_t)m * n_in + k0 + i));
+                    *reinterpret_cast<uint4*>(xs + (size_t)m * xstride + i) = v;
+                }
             }
         }
         consumers_sync();
 
-        // ring order is segment-major: consecutive items belong to different pairs, i.e. to different warps
+        // Ring order is segment-major: consecutive items are different octets, i.e. different warps. One item is
+        // 8 weight rows x 256 inputs, stored as 8 column blocks of 32 inputs ([block][row][64 bytes]); lane
+        // (g8, q4) owns inputs 32*block + 8*q4 .. +7 of row g8. Two m16n8k16 steps per block: the activations are
+        // the 16-row A operand (rows >= M repeat row M-1 and are ignored), the weights the 8-column B operand.
+        const __nv_bfloat16* xlo = xs + (size_t)min(g8, M - 1) * xstride + q4 * 8;
+        const __nv_bfloat16* xhi = xs + (size_t)min(g8 + 8, M - 1) * xstride + q4 * 8;
         for (int sg = 0; sg < ws; ++sg) {
             const int seg = w0 + sg;
-            const int seglen = min(kSeg, n_in - seg * kSeg);
-            for (int pl = warp; pl < np; pl += kPassConsumerWarps) {
-                const uint32_t g = gi + (uint32_t)(seg * np + pl);
+            for (int o = warp; o < n_oct; o += kPassConsumerWarps) {
+                const uint32_t g = gi + (uint32_t)(seg * n_oct + o);
+                const int rows = 2 * min(4, np - 4 * o);
                 const long long tw0 = p.trace ? clock64() : 0;
                 const int slot = ring_wait_full(p, sm, g, stage, M * 1000 + seg);
                 const long long tw1 = p.trace ? clock64() : 0;
-                const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes;
-                unsigned long long acc_a[M], acc_b[M];
+                const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes + g8 * 64 + q4 * 16;
+                const int blk = rows * 64;
+                uint4 wv[8];
 #pragma unroll
-                for (int m = 0; m < M; ++m) acc_a[m] = acc_b[m] = 0ull;
+                for (int j = 0; j < 8; ++j)
+                    wv[j] = (g8 < rows) ? *reinterpret_cast<const uint4*>(sl + j * blk) : make_uint4(0u, 0u, 0u, 0u);
+                float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int kk = i * 256 + lane * 8;
-                    if (kk < seglen) {
-                        const uint4 wa = *reinterpret_cast<const uint4*>(sl + kk * 2);
-                        const uint4 wb = *reinterpret_cast<const uint4*>(sl + kSlotBytes / 2 + kk * 2);
-                        const unsigned long long a0 = bf2_to_f2(wa.x), a1 = bf2_to_f2(wa.y), a2 = bf2_to_f2(wa.z), a3 = bf2_to_f2(wa.w);
-                        const unsigned long long b0 = bf2_to_f2(wb.x), b1 = bf2_to_f2(wb.y), b2 = bf2_to_f2(wb.z), b3 = bf2_to_f2(wb.w);
-#pragma unroll
-                        for (int m = 0; m < M; ++m) {
-                            const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)m * xstride + sg * kSeg + kk);
-                            const unsigned long long x0 = bf2_to_f2(xv.x), x1 = bf2_to_f2(xv.y), x2 = bf2_to_f2(xv.z), x3 = bf2_to_f2(xv.w);
-                            acc_a[m] = ffma2(a0, x0, acc_a[m]);
-                            acc_a[m] = ffma2(a1, x1, acc_a[m]);
-                            acc_a[m] = ffma2(a2, x2, acc_a[m]);
-                            acc_a[m] = ffma2(a3, x3, acc_a[m]);
-                            acc_b[m] = ffma2(b0, x0, acc_b[m]);
-                            acc_b[m] = ffma2(b1, x1, acc_b[m]);
-                            acc_b[m] = ffma2(b2, x2, acc_b[m]);
-                            acc_b[m] = ffma2(b3, x3, acc_b[m]);
-                        }
-                    }
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 al = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + j * 32);
+                    uint4 ah = make_uint4(0u, 0u, 0u, 0u);
+                    if (M > 8) ah = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + j * 32);
+                    mma_bf16_16816(c0, al.x, ah.x, al.y, ah.y, wv[j].x, wv[j].y);
+                    mma_bf16_16816(c1, al.z, ah.z, al.w, ah.w, wv[j].z, wv[j].w);
                 }
                 __syncwarp();
                 if (lane == 0) ring_release(p, sm, g);
-                float vab[M];
-#pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    float ea, oa, eb, ob;
-                    unpack2(acc_a[m], ea, oa);
-                    unpack2(acc_b[m], eb, ob);
-                    vab[m] = warp_sum_pair(ea + oa, eb + ob, lane);
-                }
-                if ((lane & 15) == 0) {  // lane 0 holds row a, lane 16 row b; segments are added in ascending order
-                    const int r = lane >> 4;
-#pragma unroll
-                    for (int m = 0; m < M; ++m) psum[(pl * 2 + r) * M + m] += vab[m];
+                // c[0], c[1]: activation row g8, weight rows 2*q4, 2*q4+1 of the octet (= pair 4*o + q4); c[2], c[3]: row g8 + 8.
+                // Segments of a pair are added in ascending order, always by this lane.
+                const int pl = 4 * o + q4;
+                if (pl < np) {
+                    if (g8 < M) {
+                        psum[(pl * 2 + 0) * M + g8] += c0[0] + c1[0];
+                        psum[(pl * 2 + 1) * M + g8] += c0[1] + c1[1];
+                    }
+                    if (M > 8 && g8 + 8 < M) {
+                        psum[(pl * 2 + 0) * M + g8 + 8] += c0[2] + c1[2];
+                        psum[(pl * 2 + 1) * M + g8 + 8] += c0[3] + c1[3];
+                    }
                 }
                 if (p.trace) {
                     cyc_wait += tw1 - tw0;
@@ -472,7 +484,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             }
         }
     }
-    gi += (uint32_t)(np * n_seg);
+    gi += (uint32_t)(n_oct * n_seg);
     consumers_sync();
     trace_mark(p, stage, 2);
     if (p.trace && tid == 0) {
@@ -565,15 +577,15 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 #pragma unroll
             for (int j = 0; j < 3; ++j) {
                 const float v = warp_sum(s_loc[m][j]);
-                if (lane == 0) red[warp * (kMaxRows * 4) + m * 4 + j] = v;
+                if (lane == 0) red[warp * (kPassMaxRows * 4) + m * 4 + j] = v;
             }
         consumers_sync();
         if (tid < M * 3) {
             const int m = tid / 3, j = tid - m * 3;
             float tot = 0.f;
 #pragma unroll
-            for (int w = 0; w < kPassConsumerWarps; ++w) tot += red[w * (kMaxRows * 4) + m * 4 + j];
-            p.partials[(((size_t)st.resid_slot * gridDim.x + blockIdx.x) * kMaxRows + m) * 4 + j] = tot;
+            for (int w = 0; w < kPassConsumerWarps; ++w) tot += red[w * (kPassMaxRows * 4) + m * 4 + j];
+            p.partials[(((size_t)st.resid_slot * gridDim.x + blockIdx.x) * kPassMaxRows + m) * 4 + j] = tot;
         }
     } else if (type == kStLmHead) {
 #pragma unroll
@@ -590,8 +602,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 }
             }
             if (lane == 0) {
-                red[warp * (kMaxRows * 4) + m * 4 + 0] = v;
-                red[warp * (kMaxRows * 4) + m * 4 + 1] = __int_as_float(i);
+                red[warp * (kPassMaxRows * 4) + m * 4 + 0] = v;
+                red[warp * (kPassMaxRows * 4) + m * 4 + 1] = __int_as_float(i);
             }
         }
         consumers_sync();
@@ -599,26 +611,26 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             float v = -INFINITY;
             int i = INT_MAX;
             for (int w = 0; w < kPassConsumerWarps; ++w) {
-                const float ov = red[w * (kMaxRows * 4) + tid * 4 + 0];
-                const int oi = __float_as_int(red[w * (kMaxRows * 4) + tid * 4 + 1]);
+                const float ov = red[w * (kPassMaxRows * 4) + tid * 4 + 0];
+                const int oi = __float_as_int(red[w * (kPassMaxRows * 4) + tid * 4 + 1]);
                 if (ov > v || (ov == v && oi < i)) {
                     v = ov;
                     i = oi;
                 }
             }
-            float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kMaxRows * 4;
-            lmp[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 0] = v;
-            lmp[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 1] = __int_as_float(i);
+            float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kPassMaxRows * 4;
+            lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 0] = v;
+            lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 1] = __int_as_float(i);
         }
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
             int* g = reinterpret_cast<int*>(red);
-            if (warp < M) {  // one warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index
+            for (int m = warp; m < M; m += kPassConsumerWarps) {  // a warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index
                 float v = -INFINITY;
                 int i = INT_MAX;
-                const float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kMaxRows * 4;
+                const float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kPassMaxRows * 4;
                 for (unsigned b = lane; b < gridDim.x; b += 32) {
-                    const float ov = __ldcg(lmp + ((size_t)b * kMaxRows + warp) * 4 + 0);
-                    const int oi = __float_as_int(__ldcg(lmp + ((size_t)b * kMaxRows + warp) * 4 + 1));
+                    const float ov = __ldcg(lmp + ((size_t)b * kPassMaxRows + m) * 4 + 0);
+                    const int oi = __float_as_int(__ldcg(lmp + ((size_t)b * kPassMaxRows + m) * 4 + 1));
                     if (ov > v || (ov == v && oi < i)) {
                         v = ov;
                         i = oi;
@@ -635,8 +647,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 }
                 if (lane == 0) {
                     if (i == INT_MAX) i = 0;
-                    p.argmax_out[warp] = i;
-                    g[warp] = i;
+                    p.argmax_out[m] = i;
+                    g[m] = i;
                 }
             }
             consumers_sync();
@@ -663,14 +675,14 @@ template <int M>
 __device__ void finish_stage(const PassParams& p, const PassSmem& sm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int r = blockIdx.x; r < p.n_resid; r += gridDim.x) {
-        const float* part = p.partials + (size_t)r * gridDim.x * kMaxRows * 4;
+        const float* part = p.partials + (size_t)r * gridDim.x * kPassMaxRows * 4;
         const ResidOut out = p.resid[r];
-        if (warp < M) {
+        for (int m = warp; m < M; m += kPassConsumerWarps) {
             double sxy = 0, sxx = 0, syy = 0;
             for (unsigned b = lane; b < gridDim.x; b += 32) {
-                sxy += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 0);
-                sxx += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 1);
-                syy += (double)__ldcg(part + ((size_t)b * kMaxRows + warp) * 4 + 2);
+                sxy += (double)__ldcg(part + ((size_t)b * kPassMaxRows + m) * 4 + 0);
+                sxx += (double)__ldcg(part + ((size_t)b * kPassMaxRows + m) * 4 + 1);
+                syy += (double)__ldcg(part + ((size_t)b * kPassMaxRows + m) * 4 + 2);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -680,8 +692,8 @@ __device__ void finish_stage(const PassParams& p, const PassSmem& sm) {
             }
             if (lane == 0) {
                 const double c = sxy / fmax(sqrt(sxx) * sqrt(syy), 1e-30);
-                out.cos_out[warp] = (float)c;
-                sm.red[warp] = (float)c;
+                out.cos_out[m] = (float)c;
+                sm.red[m] = (float)c;
             }
         }
         consumers_sync();
@@ -729,12 +741,12 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     TileAddr ta{nhb, box_cols * 2, (box_cols * 2 == 128) ? 1 : 0};
 
     // per-group scratch in region A
-    const size_t scratch_bytes = ((size_t)M * hd * 4 + (size_t)M * kAttnChunk * 4 + 4 * kMaxRows * 4 + 16 + 15) & ~(size_t)15;
+    const size_t scratch_bytes = ((size_t)M * hd * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     unsigned char* base = sm.reg_a + (size_t)grp * scratch_bytes;
     float* qs = reinterpret_cast<float*>(base);   // [M][hd]
     float* Ps = qs + M * hd;                       // [M][128]
-    float* red = Ps + M * kAttnChunk;              // [4][kMaxRows]
-    int* flag = reinterpret_cast<int*>(red + 4 * kMaxRows);
+    float* red = Ps + M * kAttnChunk;              // [4][kPassMaxRows]
+    int* flag = reinterpret_cast<int*>(red + 4 * kPassMaxRows);
 
     for (int j = grp; j < n_local; j += p.attn_groups) {
         const int idx = blockIdx.x + j * gridDim.x;
@@ -808,7 +820,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                 const bool ok = key <= p.pos0 + m;
                 sc[m] = ok ? sc[m] * p.attn_scale : -INFINITY;
                 const float v = warp_max(sc[m]);
-                if (glane == 0) red[gwarp * kMaxRows + m] = v;
+                if (glane == 0) red[gwarp * kPassMaxRows + m] = v;
             }
             bar_sync(bar_id, 128);
             if (g == group - 1) {  // K tile no longer needed: hand its slots back to the producer
@@ -819,15 +831,15 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
 #pragma unroll
             for (int m = 0; m < M; ++m)
-                cmax[m] = fmaxf(fmaxf(red[0 * kMaxRows + m], red[1 * kMaxRows + m]),
-                                fmaxf(red[2 * kMaxRows + m], red[3 * kMaxRows + m]));
+                cmax[m] = fmaxf(fmaxf(red[0 * kPassMaxRows + m], red[1 * kPassMaxRows + m]),
+                                fmaxf(red[2 * kPassMaxRows + m], red[3 * kPassMaxRows + m]));
             bar_sync(bar_id, 128);
 #pragma unroll
             for (int m = 0; m < M; ++m) {
                 const float pe = (sc[m] == -INFINITY) ? 0.f : expf(sc[m] - cmax[m]);
                 Ps[m * kAttnChunk + gt] = pe;
                 const float v = warp_sum(pe);
-                if (glane == 0) red[gwarp * kMaxRows + m] = v;
+                if (glane == 0) red[gwarp * kPassMaxRows + m] = v;
             }
             if (g == 0) {  // V tile: wait and patch once per item
                 for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gv + t, stage, M * 1000 + 500 + j);
@@ -844,13 +856,13 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
             bar_sync(bar_id, 128);
             if (gt < M) {
-                const float l = ((red[0 * kMaxRows + gt] + red[1 * kMaxRows + gt]) + red[2 * kMaxRows + gt]) + red[3 * kMaxRows + gt];
-                p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + gt) * 2 + 1] = l;
+                const float l = ((red[0 * kPassMaxRows + gt] + red[1 * kPassMaxRows + gt]) + red[2 * kPassMaxRows + gt]) + red[3 * kPassMaxRows + gt];
+                p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + gt) * 2 + 1] = l;
             }
             if (gt == 0) {
 #pragma unroll
                 for (int m = 0; m < M; ++m)
-                    p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + m) * 2 + 0] = cmax[m];
+                    p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * 2 + 0] = cmax[m];
             }
             // ---- P V: thread e owns output dimension e
             for (int e = gt; e < hd; e += 128) {
@@ -867,7 +879,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                 }
 #pragma unroll
                 for (int m = 0; m < M; ++m)
-                    p.part_acc[(((size_t)head * p.chunk_stride + chunk) * kMaxRows + m) * hd + e] = acc[m];
+                    p.part_acc[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * hd + e] = acc[m];
             }
         }
         // ---- release the V tile; the last group to finish this kv head merges its chunks in order
@@ -895,7 +907,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 const int c = min(c0 + i, nc - 1);
-                                const size_t b = ((size_t)head * p.chunk_stride + c) * kMaxRows + m;
+                                const size_t b = ((size_t)head * p.chunk_stride + c) * kPassMaxRows + m;
                                 cm[i] = __ldcg(p.part_ml + b * 2 + 0);
                                 cl[i] = __ldcg(p.part_ml + b * 2 + 1);
                                 pa[i] = __ldcg(p.part_acc + b * hd + e);
@@ -929,7 +941,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     sm.full = reinterpret_cast<uint64_t*>(base + p.off_bars);
     sm.empty = sm.full + p.ns;
     sm.red = reinterpret_cast<float*>(base + p.off_misc);
-    sm.flag = reinterpret_cast<int*>(sm.red + 16 * kMaxRows * 4);
+    sm.flag = reinterpret_cast<int*>(sm.red + 16 * kPassMaxRows * 4);
     sm.consumed = reinterpret_cast<volatile unsigned*>(sm.flag + 8);
     sm.psum = reinterpret_cast<float*>(base + p.off_psum);
     sm.reg_a = base + p.off_reg_a;

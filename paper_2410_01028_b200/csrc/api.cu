@@ -123,7 +123,8 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const int kvd = c.n_kv_heads * c.head_dim;
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
     const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
-    const size_t psum = ((size_t)np_max * 2 * M * 4 + 15) & ~(size_t)15;
+    // per-pair partial sums; when a CTA has fewer than 8 octets up to 15 warps keep copies (at most 60 pairs in all)
+    const size_t psum = ((size_t)std::max<long long>(np_max, 64) * 2 * M * 4 + 15) & ~(size_t)15;
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M) * kSegK + kXsPad) * 2;
@@ -227,7 +228,7 @@ static Layout make_layout(const asd_config& c) {
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
     L.sync_words = take(256);
     L.resid_tab = take((size_t)2 * (2 * std::max(c.n_layers, 1)) * sizeof(ResidOut));
-    L.trace = take((size_t)L.max_stages * 6 * kMaxGemvGrid * 8);
+    L.trace = take((size_t)L.max_stages * 8 * kMaxGemvGrid * 8);
     L.total = o;
     return L;
 }
@@ -1038,7 +1039,7 @@ extern "C" int asd_get_last_trace(asd_ctx* x, int32_t* n_stages, int32_t* n_ctas
     if (n_stages) *n_stages = x->last_n_stages;
     if (n_ctas) *n_ctas = x->dev->num_sms;
     if (ns_out) {
-        ASD_CUDA(x, cudaMemcpyAsync(ns_out, x->ws + x->lay.trace, (size_t)x->last_n_stages * 6 * x->dev->num_sms * 8, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaMemcpyAsync(ns_out, x->ws + x->lay.trace, (size_t)x->last_n_stages * 8 * x->dev->num_sms * 8, cudaMemcpyDeviceToHost, x->stream));
         ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     }
     return ASD_OK;

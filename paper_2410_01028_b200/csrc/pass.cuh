@@ -92,7 +92,7 @@ struct PassParams {
     int* accept_out;
     float* logits_out;
     int acc_sim;
-    long long* trace;  // optional [n_stages][6][gridDim.x] device timestamps (ns) and cycle counts, or null
+    long long* trace;  // optional [n_stages][8][gridDim.x] device timestamps (ns) and cycle counts, or null
     // shared-memory plan (bytes from the 1024-aligned base)
     int ns;            // ring slots
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
@@ -301,7 +301,7 @@ __device__ __forceinline__ long long global_ns() {
 }
 // per-stage timeline of every CTA (debugging aid): 0 = stage entered, 1 = inputs ready, 2 = streaming done, 3 = stage left
 __device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k) {
-    if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 6 + k) * gridDim.x + blockIdx.x] = global_ns();
+    if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 8 + k) * gridDim.x + blockIdx.x] = global_ns();
 }
 
 // ============================================================================================ grid barrier
@@ -391,7 +391,13 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             inv[m] = 1.0f / sqrtf(s / (float)n_in + p.eps);
         }
     }
-    for (int i = tid; i < np * 2 * M; i += kPassConsumers) psum[i] = 0.f;
+    // Few octets (the d x d matrices leave ~28 rows to a CTA): several warps share an octet, warp set ks taking the
+    // segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are added
+    // in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
+    const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
+    const int copy_stride = np * 2 * M;
+    for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
+    trace_mark(p, stage, 6);
 
     long long cyc_wait = 0, cyc_work = 0;  // when tracing: cycles this warp spent waiting for slots / working on them
     // ---- stream the slab window by window
@@ -433,15 +439,21 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         }
         consumers_sync();
 
+        if (w0 == 0) trace_mark(p, stage, 7);
         // Ring order is segment-major: consecutive items are different octets, i.e. different warps. One item is
         // 8 weight rows x 256 inputs, stored as 8 column blocks of 32 inputs ([block][row][64 bytes]); lane
         // (g8, q4) owns inputs 32*block + 8*q4 .. +7 of row g8. Two m16n8k16 steps per block: the activations are
         // the 16-row A operand (rows >= M repeat row M-1 and are ignored), the weights the 8-column B operand.
         const __nv_bfloat16* xlo = xs + (size_t)min(g8, M - 1) * xstride + q4 * 8;
         const __nv_bfloat16* xhi = xs + (size_t)min(g8 + 8, M - 1) * xstride + q4 * 8;
+        const int ks = (S > 1) ? warp / n_oct : 0;                 // which copy of the partial sums this warp adds into
+        const int o_first = (S > 1) ? ((ks < S) ? warp - ks * n_oct : n_oct) : warp;
+        const int o_step = (S > 1) ? n_oct : kPassConsumerWarps;  // S > 1: exactly one octet per warp
+        float* psum_w = psum + (size_t)ks * copy_stride;
         for (int sg = 0; sg < ws; ++sg) {
             const int seg = w0 + sg;
-            for (int o = warp; o < n_oct; o += kPassConsumerWarps) {
+            if (S > 1 && seg % S != ks) continue;
+            for (int o = o_first; o < n_oct; o += o_step) {
                 const uint32_t g = gi + (uint32_t)(seg * n_oct + o);
                 const int rows = 2 * min(4, np - 4 * o);
                 const long long tw0 = p.trace ? clock64() : 0;
@@ -469,12 +481,12 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 const int pl = 4 * o + q4;
                 if (pl < np) {
                     if (g8 < M) {
-                        psum[(pl * 2 + 0) * M + g8] += c0[0] + c1[0];
-                        psum[(pl * 2 + 1) * M + g8] += c0[1] + c1[1];
+                        psum_w[(pl * 2 + 0) * M + g8] += c0[0] + c1[0];
+                        psum_w[(pl * 2 + 1) * M + g8] += c0[1] + c1[1];
                     }
                     if (M > 8 && g8 + 8 < M) {
-                        psum[(pl * 2 + 0) * M + g8 + 8] += c0[2] + c1[2];
-                        psum[(pl * 2 + 1) * M + g8 + 8] += c0[3] + c1[3];
+                        psum_w[(pl * 2 + 0) * M + g8 + 8] += c0[2] + c1[2];
+                        psum_w[(pl * 2 + 1) * M + g8 + 8] += c0[3] + c1[3];
                     }
                 }
                 if (p.trace) {
@@ -488,8 +500,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     consumers_sync();
     trace_mark(p, stage, 2);
     if (p.trace && tid == 0) {
-        p.trace[((size_t)stage * 6 + 4) * gridDim.x + blockIdx.x] = cyc_wait;
-        p.trace[((size_t)stage * 6 + 5) * gridDim.x + blockIdx.x] = cyc_work;
+        p.trace[((size_t)stage * 8 + 4) * gridDim.x + blockIdx.x] = cyc_wait;
+        p.trace[((size_t)stage * 8 + 5) * gridDim.x + blockIdx.x] = cyc_work;
     }
 
     // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
@@ -509,6 +521,10 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 #pragma unroll
         for (int m = 0; m < M; ++m) {
             float va = psum[(pl * 2 + 0) * M + m], vb = psum[(pl * 2 + 1) * M + m];
+            for (int k = 1; k < S; ++k) {
+                va += psum[(size_t)k * copy_stride + (pl * 2 + 0) * M + m];
+                vb += psum[(size_t)k * copy_stride + (pl * 2 + 1) * M + m];
+            }
             if (type == kStGateUp) {
                 const float t = va / (1.0f + expf(-va)) * vb;
                 p.t[(size_t)m * (n_rows >> 1) + (pair0 + pl)] = __float2bfloat16_rn(t);
@@ -965,7 +981,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     if (p.trace && threadIdx.x == 0) {  // which SM runs this CTA (entry 4 of the embedding stage, which streams nothing)
         unsigned smid;
         asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        p.trace[((size_t)0 * 6 + 4) * gridDim.x + blockIdx.x] = smid;
+        p.trace[((size_t)0 * 8 + 4) * gridDim.x + blockIdx.x] = smid;
     }
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);

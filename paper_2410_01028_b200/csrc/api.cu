@@ -131,7 +131,7 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const size_t reg_a = (std::max(xs, 2 * attn_scratch) + 15) & ~(size_t)15;
     const long long avail = (long long)dv.max_smem - 1024 - (long long)(psum + misc + reg_a) - 2 * 64 * 8;
     int ns = (int)std::min<long long>(64, avail / kSlotBytes);
-    const int tile_slots = 4 * std::max(1, c.head_dim / 64);
+    const int tile_slots = (kAttnChunk / kBoxKeys) * std::max(1, c.head_dim / 64);
     if (ns < 2 * tile_slots || ns < 8) return false;
     pl->ns = ns;
     pl->attn_groups = ns >= 4 * tile_slots ? 2 : 1;
@@ -169,8 +169,8 @@ static bool check_config(const asd_config& c) {
     return true;
 }
 
-// bytes of a matrix in the packed layout of the pass kernel: (pairs of rows) x (segments of 256 inputs) x 1 KB
-static size_t packed_bytes(size_t n_rows, size_t n_in) { return ((n_rows + 1) / 2) * ((n_in + kSegK - 1) / kSegK) * (size_t)1024; }
+// bytes of a matrix in the packed layout of the pass kernel: (pairs of rows) x (column blocks of 32 inputs) x 128 bytes
+static size_t packed_bytes(size_t n_rows, size_t n_in) { return ((n_rows + 1) / 2) * ((n_in + 31) / 32) * (size_t)128; }
 
 static Layout make_layout(const asd_config& c) {
     Layout L{};
@@ -313,7 +313,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// One 2-D tensor map per layer and per cache: [max_seq rows, kv_dim columns] bf16, boxes of 32 keys x (up to) 64
+// One 2-D tensor map per layer and per cache: [max_seq rows, kv_dim columns] bf16, boxes of 64 keys x (up to) 64
 // columns; 128-byte rows are stored with the 128-byte swizzle so that one thread per key reads its row without
 // shared-memory bank conflicts.
 static int make_tensor_maps(asd_ctx* x) {
@@ -328,7 +328,7 @@ static int make_tensor_maps(asd_ctx* x) {
     const int box_cols = c.head_dim > 64 ? 64 : c.head_dim;
     const cuuint64_t gdim[2] = {(cuuint64_t)x->kv_dim, (cuuint64_t)c.max_seq};
     const cuuint64_t gstride[1] = {(cuuint64_t)x->kv_dim * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)box_cols, 32u};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)kBoxKeys};
     const cuuint32_t estr[2] = {1u, 1u};
     const CUtensorMapSwizzle swz = (box_cols * 2 == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
     for (int l = 0; l < L; ++l)
@@ -602,23 +602,24 @@ extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : 
 // Repack one matrix into the pass kernel's layout and copy it to the device. The logical matrix has n_rows
 // rows of n_in inputs; row(r) returns the host pointer of logical row r. CTA b of a G-CTA grid owns pairs
 // [b*P/G, (b+1)*P/G) in octets of four pairs (the last may be smaller); its slab is segment-major (for each
-// segment of 256 inputs: for each octet), and an item of R rows is 8 column blocks of 32 inputs, each block
-// R rows x 64 bytes. Inputs past n_in are zero.
+// segment of 512 inputs: for each octet), and an item of R rows is a run of column blocks of 32 inputs, each
+// block R rows x 64 bytes (16 blocks, fewer in the last segment). Inputs past n_in are zero.
 template <class RowFn, class PairFn>
 static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, PairFn pair_rows_of,
                          std::vector<unsigned char>& staging) {
-    const size_t n_pairs = (n_rows + 1) / 2, n_seg = (n_in + kSegK - 1) / kSegK;
-    const size_t total = n_pairs * n_seg * 1024;
+    const size_t n_pairs = (n_rows + 1) / 2, row_blocks = (n_in + 31) / 32, n_seg = (n_in + kSegK - 1) / kSegK;
+    const size_t total = n_pairs * row_blocks * 128;
     const int G = x->dev->num_sms;
     staging.assign(total, 0);
 #pragma omp parallel for schedule(static)
     for (int b = 0; b < G; ++b) {
         const size_t pair0 = (size_t)b * n_pairs / G, pair1 = (size_t)(b + 1) * n_pairs / G, np = pair1 - pair0;
-        unsigned char* slab = staging.data() + pair0 * n_seg * 1024;
+        unsigned char* slab = staging.data() + pair0 * row_blocks * 128;
         for (size_t sg = 0; sg < n_seg; ++sg) {
+            const size_t nblk = std::min<size_t>(16, row_blocks - sg * 16);
             for (size_t o = 0; o * 4 < np; ++o) {
                 const size_t pairs = std::min<size_t>(4, np - 4 * o), R = 2 * pairs;
-                unsigned char* item = slab + sg * np * 1024 + o * kSlotBytes;
+                unsigned char* item = slab + sg * np * 2048 + o * nblk * 512;
                 for (size_t pq = 0; pq < pairs; ++pq) {
                     size_t rr[2];
                     pair_rows_of(pair0 + 4 * o + pq, rr[0], rr[1]);
@@ -626,9 +627,8 @@ static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size
                         if (rr[h] >= n_rows) continue;
                         const uint16_t* src = row(rr[h]);
                         const size_t g = 2 * pq + h;
-                        for (size_t j = 0; j < 8; ++j) {
+                        for (size_t j = 0; j < nblk; ++j) {
                             const size_t k = sg * kSegK + j * 32;
-                            if (k >= n_in) break;
                             memcpy(item + j * (R * 64) + g * 64, src + k, std::min<size_t>(32, n_in - k) * 2);
                         }
                     }

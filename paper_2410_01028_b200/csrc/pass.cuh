@@ -18,12 +18,12 @@
 // weights are streamed and no K/V is touched for them.
 //
 // Packed weights: a matrix [n_rows, n_in] is cut into PAIRS of rows (the two rotary partners of a q/k head,
-// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 256 inputs. CTA b owns pairs [b*P/G, (b+1)*P/G)
+// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 512 inputs. CTA b owns pairs [b*P/G, (b+1)*P/G)
 // and groups them into OCTETS of four pairs (the last octet may hold fewer). One ring item = one octet x one
-// segment = up to 8 rows x 512 bytes = one 4 KB slot, stored as 8 column blocks of 32 inputs. The CTA's slab is
+// segment of 512 inputs = up to 8 rows x 1 KB = one 8 KB slot, stored as up to 16 column blocks of 32 inputs
+// (rows x 64 bytes each; the last segment of a row simply has fewer blocks). The CTA's slab is
 // segment-major (for seg: for octet), so consecutive ring items belong to different consumer warps and are
-// consumed as soon as they land, and no byte of padding crosses HBM for shapes whose input size is a multiple
-// of 256.
+// consumed as soon as they land, and no padding crosses HBM for input sizes that are multiples of 32.
 //
 // The products run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate): the activation rows are the
 // 16-row A operand, the 8 weight rows of an item the B operand, so one step serves any row count up to 16 and
@@ -100,7 +100,8 @@ struct PassParams {
     int off_bars, off_misc, off_psum, off_reg_a;
 };
 
-constexpr int kSegK = 256;     // inputs per ring item
+constexpr int kSegK = 512;     // inputs per ring item (16 column blocks of 32; the last item of a row may hold fewer)
+constexpr int kBoxKeys = 64;   // keys per K/V box (one ring slot)
 constexpr int kOctRows = 8;    // weight rows per ring item (four pairs): the N of one m16n8k16 tensor-core step
 constexpr int kXsPad = 32;     // bf16 elements of padding per activation row (64 bytes: conflict-free 16-byte reads)
 
@@ -242,8 +243,8 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
             const int n_local = attn_local_items(p, M, n_chunks);
             const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
             const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
-            const uint32_t box_bytes = 32u * box_cols * 2u;
-            const int tile_slots = 4 * nhb;
+            const uint32_t box_bytes = (uint32_t)kBoxKeys * box_cols * 2u;
+            const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
             const int n_items = n_local * 2 * tile_slots;
             for (int idx = lane; idx < n_items; idx += 32) {
                 const int j = idx / (2 * tile_slots), r = idx - j * 2 * tile_slots;
@@ -255,7 +256,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 const int slot = ring_acquire(p, sm, g, s, M);
                 mbar_expect_tx(&sm.full[slot], box_bytes);
                 tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, which ? st.tm_v : st.tm_k, kvh * p.head_dim + hb * 64,
-                            chunk * kAttnChunk + rg * 32, &sm.full[slot]);
+                            chunk * kAttnChunk + rg * kBoxKeys, &sm.full[slot]);
                 issued[1] = issued[0], issued[0] = g, ++n_issued;
             }
             gi += (uint32_t)n_items;
@@ -267,14 +268,17 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
         const int n_seg = (st.n_in + kSegK - 1) / kSegK;
         const int n_oct = (np + 3) >> 2;
         const int n_items = n_oct * n_seg;
-        const unsigned char* slab = st.W + (size_t)pair0 * n_seg * 1024;
+        const int row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
+        const unsigned char* slab = st.W + (size_t)pair0 * row_blocks * 128;
         for (int idx = lane; idx < n_items; idx += 32) {
             const int seg = idx / n_oct, o = idx - seg * n_oct;
-            const uint32_t bytes = (uint32_t)min(4, np - 4 * o) * 1024u;  // pairs of this octet x 2 rows x 512 bytes
+            const int nblk = min(16, row_blocks - seg * 16);  // column blocks of this segment
+            const int rows = 2 * min(4, np - 4 * o);
+            const uint32_t bytes = (uint32_t)(nblk * rows * 64);
             const uint32_t g = gi + (uint32_t)idx;
             const int slot = ring_acquire(p, sm, g, s, M);
             mbar_expect_tx(&sm.full[slot], bytes);
-            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)seg * np * 1024 + (size_t)o * kSlotBytes, bytes,
+            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)seg * np * 2048 + (size_t)o * nblk * 512, bytes,
                              &sm.full[slot], pol_stream);
             issued[1] = issued[0], issued[0] = g, ++n_issued;
         }
@@ -441,7 +445,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
         if (w0 == 0) trace_mark(p, stage, 7);
         // Ring order is segment-major: consecutive items are different octets, i.e. different warps. One item is
-        // 8 weight rows x 256 inputs, stored as 8 column blocks of 32 inputs ([block][row][64 bytes]); lane
+        // up to 8 weight rows x 512 inputs, stored as column blocks of 32 inputs ([block][row][64 bytes]); lane
         // (g8, q4) owns inputs 32*block + 8*q4 .. +7 of row g8. Two m16n8k16 steps per block: the activations are
         // the 16-row A operand (rows >= M repeat row M-1 and are ignored), the weights the 8-column B operand.
         const __nv_bfloat16* xlo = xs + (size_t)min(g8, M - 1) * xstride + q4 * 8;
@@ -461,18 +465,25 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 const long long tw1 = p.trace ? clock64() : 0;
                 const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes + g8 * 64 + q4 * 16;
                 const int blk = rows * 64;
-                uint4 wv[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    wv[j] = (g8 < rows) ? *reinterpret_cast<const uint4*>(sl + j * blk) : make_uint4(0u, 0u, 0u, 0u);
+                const int nblk = min(16, ((n_in + 31) >> 5) - seg * 16);
                 float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint4 al = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + j * 32);
-                    uint4 ah = make_uint4(0u, 0u, 0u, 0u);
-                    if (M > 8) ah = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + j * 32);
-                    mma_bf16_16816(c0, al.x, ah.x, al.y, ah.y, wv[j].x, wv[j].y);
-                    mma_bf16_16816(c1, al.z, ah.z, al.w, ah.w, wv[j].z, wv[j].w);
+                for (int h = 0; h < 2; ++h) {  // two halves of 8 column blocks: weights of a half in registers, then 16 steps
+                    uint4 wv[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        wv[j] = (g8 < rows && h * 8 + j < nblk) ? *reinterpret_cast<const uint4*>(sl + (h * 8 + j) * blk)
+                                                                 : make_uint4(0u, 0u, 0u, 0u);
+                    if (h * 8 < nblk) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const uint4 al = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + (h * 8 + j) * 32);
+                            uint4 ah = make_uint4(0u, 0u, 0u, 0u);
+                            if (M > 8) ah = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + (h * 8 + j) * 32);
+                            mma_bf16_16816(c0, al.x, ah.x, al.y, ah.y, wv[j].x, wv[j].y);
+                            mma_bf16_16816(c1, al.z, ah.z, al.w, ah.w, wv[j].z, wv[j].w);
+                        }
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) ring_release(p, sm, g);
@@ -727,7 +738,7 @@ __device__ void finish_stage(const PassParams& p, const PassSmem& sm) {
 struct TileAddr {
     int nhb, row_bytes, swz;
     __device__ __forceinline__ void locate(int r, int c, int& slot_in_tile, int& off) const {
-        const int rg = r >> 5, rr = r & 31;
+        const int rg = r / kBoxKeys, rr = r % kBoxKeys;
         const int hb = (nhb > 1) ? (c >> 3) : 0;
         const int cc = (nhb > 1) ? (c & 7) : c;
         slot_in_tile = rg * nhb + hb;
@@ -741,7 +752,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     const int hd = p.head_dim;
     const int nhb = hd > 64 ? hd / 64 : 1;
     const int box_cols = hd > 64 ? 64 : hd;
-    const int tile_slots = 4 * nhb;
+    const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
     int n_chunks;
     const int n_local = attn_local_items(p, M, n_chunks);
     const uint32_t gi0 = gi;

@@ -10,7 +10,7 @@
 
 namespace asd {
 
-constexpr int kSlotBytes = 4096;             // one ring slot: two weight rows x 1024 bf16, or one 32-key K/V box
+constexpr int kSlotBytes = 8192;             // one ring slot: 8 weight rows x 512 bf16 inputs, or one 64-key K/V box
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
 
 enum DeviceError : int {

@@ -370,18 +370,38 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
 
-    // ---- RMSNorm statistics (same arithmetic for every row count)
+    // ---- RMSNorm statistics (same arithmetic for every row count). With one or two rows the hidden state read
+    //      here stays in registers for the window fill below (one L2 round trip less per stage).
+    constexpr bool kKeepX = (M <= 2);
+    const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
+    float4 xr[kKeepX ? M : 1][3];
     float inv[M];
     if (norm) {
 #pragma unroll
         for (int m = 0; m < M; ++m) {
             float s = 0.f;
-            for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
-                const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
-                s = fmaf(v.x, v.x, s);
-                s = fmaf(v.y, v.y, s);
-                s = fmaf(v.z, v.z, s);
-                s = fmaf(v.w, v.w, s);
+            if (keep) {
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const int i = (tid + c * kPassConsumers) * 4;
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i < n_in) v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
+                    xr[kKeepX ? m : 0][c] = v;
+                    if (i < n_in) {
+                        s = fmaf(v.x, v.x, s);
+                        s = fmaf(v.y, v.y, s);
+                        s = fmaf(v.z, v.z, s);
+                        s = fmaf(v.w, v.w, s);
+                    }
+                }
+            } else {
+                for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
+                    s = fmaf(v.x, v.x, s);
+                    s = fmaf(v.y, v.y, s);
+                    s = fmaf(v.z, v.z, s);
+                    s = fmaf(v.w, v.w, s);
+                }
             }
             s = warp_sum(s);
             if (lane == 0) red[warp * (kPassMaxRows * 4) + m] = s;
@@ -411,7 +431,32 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         const int k0 = w0 * kSegK;
         const int wlen = ws * kSegK;  // inputs in this window, including the zero padding past n_in
         consumers_sync();  // previous window fully consumed; psum zeroed; red free
-        if (norm) {
+        if (keep) {  // a single window (n_in <= 5760): normalise the rows held in registers
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const int i = (tid + c * kPassConsumers) * 4;
+                if (i < wlen) {
+                    const bool in = i < n_in;
+                    uint2 gv = make_uint2(0u, 0u);
+                    if (in) gv = *reinterpret_cast<const uint2*>(st.gain + i);
+                    const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
+#pragma unroll
+                    for (int m = 0; m < M; ++m) {
+                        uint2 o = make_uint2(0u, 0u);
+                        if (in) {
+                            const float4 v = xr[kKeepX ? m : 0][c];
+                            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv[m] * g0, v.y * inv[m] * g1);
+                            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv[m] * g2, v.w * inv[m] * g3);
+                            o.x = *reinterpret_cast<uint32_t*>(&lo);
+                            o.y = *reinterpret_cast<uint32_t*>(&hi);
+                        }
+                        *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                    }
+                }
+            }
+            for (int i = kPassConsumers * 12 + tid * 4; i < wlen; i += kPassConsumers * 4)  // zero padding past 5760
+                for (int m = 0; m < M; ++m) *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = make_uint2(0u, 0u);
+        } else if (norm) {
             for (int i = tid * 4; i < wlen; i += kPassConsumers * 4) {
                 const bool in = k0 + i < n_in;
                 uint2 gv = make_uint2(0u, 0u);
@@ -525,7 +570,29 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         best_v[m] = -INFINITY;
         best_i[m] = INT_MAX;
     }
-    for (int pl = tid; pl < np; pl += kPassConsumers) {
+    const bool resid = (type == kStOproj || type == kStDown);
+    if (resid) {
+        // residual add: one thread per weight row, the M loads of the old hidden state issued together
+        float* out = p.x;
+        for (int e = tid; e < np * 2; e += kPassConsumers) {
+            const int row = 2 * pair0 + e;
+            if (row >= n_rows) continue;
+            float xv[M];
+#pragma unroll
+            for (int m = 0; m < M; ++m) xv[m] = __ldcg(out + (size_t)m * n_rows + row);
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                float v = psum[e * M + m];
+                for (int k = 1; k < S; ++k) v += psum[(size_t)k * copy_stride + e * M + m];
+                const float y = xv[m] + v;
+                out[(size_t)m * n_rows + row] = y;
+                s_loc[m][0] = fmaf(xv[m], y, s_loc[m][0]);
+                s_loc[m][1] = fmaf(xv[m], xv[m], s_loc[m][1]);
+                s_loc[m][2] = fmaf(y, y, s_loc[m][2]);
+            }
+        }
+    }
+    for (int pl = resid ? np : tid; pl < np; pl += kPassConsumers) {
         int ra, rb;
         stage_pair_rows(type, p, pair0 + pl, ra, rb);
         const bool has_b = rb < n_rows;
@@ -539,24 +606,6 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             if (type == kStGateUp) {
                 const float t = va / (1.0f + expf(-va)) * vb;
                 p.t[(size_t)m * (n_rows >> 1) + (pair0 + pl)] = __float2bfloat16_rn(t);
-            } else if (type == kStOproj || type == kStDown) {
-                float* out = p.x;
-                {
-                    const float x0 = __ldcg(out + (size_t)m * n_rows + ra);
-                    const float y0 = x0 + va;
-                    out[(size_t)m * n_rows + ra] = y0;
-                    s_loc[m][0] = fmaf(x0, y0, s_loc[m][0]);
-                    s_loc[m][1] = fmaf(x0, x0, s_loc[m][1]);
-                    s_loc[m][2] = fmaf(y0, y0, s_loc[m][2]);
-                }
-                if (has_b) {
-                    const float x1 = __ldcg(out + (size_t)m * n_rows + rb);
-                    const float y1 = x1 + vb;
-                    out[(size_t)m * n_rows + rb] = y1;
-                    s_loc[m][0] = fmaf(x1, y1, s_loc[m][0]);
-                    s_loc[m][1] = fmaf(x1, x1, s_loc[m][1]);
-                    s_loc[m][2] = fmaf(y1, y1, s_loc[m][2]);
-                }
             } else if (type == kStQkv) {
                 const int pos = p.pos0 + m;
                 const int half = p.head_dim >> 1;

@@ -840,6 +840,14 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
 
         // ---- K tile: wait for the boxes, then overwrite the rows this pass has just written (the producer may
         //      have copied the tile before the QKV stage of this pass stored them)
+        constexpr int kQPerThread = (M * 256 + 127) / 128;  // head_dim <= 256
+        unsigned short qreg[kQPerThread];
+#pragma unroll
+        for (int u = 0; u < kQPerThread; ++u) {  // the first head's queries are requested before waiting for the tile
+            const int i = gt + u * 128;
+            const int m = i / hd, e = i - m * hd;
+            qreg[u] = (i < M * hd) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
+        }
         for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
         const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
         const int n_fresh = fresh1 - fresh0 + 1;
@@ -856,36 +864,49 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         for (int g = 0; g < group; ++g) {
             const int head = kvh * group + g;
             bar_sync(bar_id, 128);  // patched tile visible; previous head's Ps / qs consumed
-            for (int i = gt; i < M * hd; i += 128) {
-                const int m = i / hd, e = i - m * hd;
-                qs[i] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)head * hd + e) << 16);
+            if (g == 0) {
+#pragma unroll
+                for (int u = 0; u < kQPerThread; ++u)
+                    if (gt + u * 128 < M * hd) qs[gt + u * 128] = __uint_as_float((uint32_t)qreg[u] << 16);
+            } else {
+                for (int i = gt; i < M * hd; i += 128) {
+                    const int m = i / hd, e = i - m * hd;
+                    qs[i] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)head * hd + e) << 16);
+                }
             }
             bar_sync(bar_id, 128);
 
+            if (j == 0 && g == 0) trace_mark(p, stage, 2);  // attention timeline: 2 = inputs staged, 4 = softmax done, 5 = P V done, 6 = ticket taken, 7 = merged
             // ---- scores: thread t owns key key0 + t
             float sc[M];
 #pragma unroll
             for (int m = 0; m < M; ++m) sc[m] = 0.f;
-            for (int c = 0; c < vec_per_row; ++c) {
-                int sit, off;
-                ta.locate(gt, c, sit, off);
-                const uint4 kv = *reinterpret_cast<const uint4*>(slot_ptr(gk + sit) + off);
-                const float kf[8] = {bf_lo(kv.x), bf_hi(kv.x), bf_lo(kv.y), bf_hi(kv.y),
-                                     bf_lo(kv.z), bf_hi(kv.z), bf_lo(kv.w), bf_hi(kv.w)};
+            {
+                const int rg = gt / kBoxKeys, rr = gt % kBoxKeys;
+                const int chunks_per_box = box_cols / 8;
+                for (int hb = 0; hb < nhb; ++hb) {
+                    const unsigned char* krow = slot_ptr(gk + rg * nhb + hb) + rr * ta.row_bytes;
+                    for (int cc = 0; cc < chunks_per_box; ++cc) {
+                        const int c = hb * 8 + cc;
+                        const uint4 kv = *reinterpret_cast<const uint4*>(krow + ((ta.swz ? (cc ^ (rr & 7)) : cc) << 4));
+                        const float kf[8] = {bf_lo(kv.x), bf_hi(kv.x), bf_lo(kv.y), bf_hi(kv.y),
+                                             bf_lo(kv.z), bf_hi(kv.z), bf_lo(kv.w), bf_hi(kv.w)};
 #pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    const float4 q0 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8);
-                    const float4 q1 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8 + 4);
-                    float a = sc[m];
-                    a = fmaf(q0.x, kf[0], a);
-                    a = fmaf(q0.y, kf[1], a);
-                    a = fmaf(q0.z, kf[2], a);
-                    a = fmaf(q0.w, kf[3], a);
-                    a = fmaf(q1.x, kf[4], a);
-                    a = fmaf(q1.y, kf[5], a);
-                    a = fmaf(q1.z, kf[6], a);
-                    a = fmaf(q1.w, kf[7], a);
-                    sc[m] = a;
+                        for (int m = 0; m < M; ++m) {
+                            const float4 q0 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8);
+                            const float4 q1 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8 + 4);
+                            float a = sc[m];
+                            a = fmaf(q0.x, kf[0], a);
+                            a = fmaf(q0.y, kf[1], a);
+                            a = fmaf(q0.z, kf[2], a);
+                            a = fmaf(q0.w, kf[3], a);
+                            a = fmaf(q1.x, kf[4], a);
+                            a = fmaf(q1.y, kf[5], a);
+                            a = fmaf(q1.z, kf[6], a);
+                            a = fmaf(q1.w, kf[7], a);
+                            sc[m] = a;
+                        }
+                    }
                 }
             }
             // ---- chunk-local softmax statistics; the row at position pos0+m sees keys <= pos0+m
@@ -940,24 +961,32 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                 for (int m = 0; m < M; ++m)
                     p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * 2 + 0] = cmax[m];
             }
+            if (j == 0 && g == 0) trace_mark(p, stage, 4);
             // ---- P V: thread e owns output dimension e
             for (int e = gt; e < hd; e += 128) {
                 float acc[M];
 #pragma unroll
                 for (int m = 0; m < M; ++m) acc[m] = 0.f;
                 const int c = e >> 3, sub = (e & 7) * 2;
-                for (int jj = 0; jj < n_valid; ++jj) {
-                    int sit, off;
-                    ta.locate(jj, c, sit, off);
-                    const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(slot_ptr(gv + sit) + off + sub));
+                const int hb = (nhb > 1) ? (c >> 3) : 0, cc = (nhb > 1) ? (c & 7) : c;
+                for (int rg = 0; rg * kBoxKeys < n_valid; ++rg) {  // keys in ascending order, one box after the other
+                    const unsigned char* vbox = slot_ptr(gv + rg * nhb + hb) + sub;
+                    const int nk = min(kBoxKeys, n_valid - rg * kBoxKeys);
+                    const float* prow = Ps + rg * kBoxKeys;
+#pragma unroll 4
+                    for (int rr = 0; rr < nk; ++rr) {
+                        const float v = __bfloat162float(
+                            *reinterpret_cast<const __nv_bfloat16*>(vbox + rr * ta.row_bytes + ((ta.swz ? (cc ^ (rr & 7)) : cc) << 4)));
 #pragma unroll
-                    for (int m = 0; m < M; ++m) acc[m] = fmaf(Ps[m * kAttnChunk + jj], v, acc[m]);
+                        for (int m = 0; m < M; ++m) acc[m] = fmaf(prow[m * kAttnChunk + rr], v, acc[m]);
+                    }
                 }
 #pragma unroll
                 for (int m = 0; m < M; ++m)
                     p.part_acc[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * hd + e] = acc[m];
             }
         }
+        if (j == 0) trace_mark(p, stage, 5);
         // ---- release the V tile; the last group to finish this kv head merges its chunks in order
         __threadfence();
         bar_sync(bar_id, 128);
@@ -968,6 +997,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             *flag = (tk == (unsigned)n_chunks - 1) ? 1 : 0;
         }
         bar_sync(bar_id, 128);
+        if (j == 0) trace_mark(p, stage, 6);
         if (*flag) {
             __threadfence();
             if (gt == 0) p.attn_counters[kvh] = 0u;
@@ -1004,6 +1034,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                 }
             }
         }
+        if (j == 0) trace_mark(p, stage, 7);
     }
 }
 

@@ -128,13 +128,15 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M) * kSegK + kXsPad) * 2;
-    const size_t reg_a = (std::max(xs, 2 * attn_scratch) + 15) & ~(size_t)15;
+    // up to three groups of four warps work on attention items, as many as their scratch fits the window's bytes
+    const int groups_by_scratch = (int)std::max<size_t>(1, std::min<size_t>(3, (size_t)kXsBudget / attn_scratch));
+    const size_t reg_a = (std::max(xs, groups_by_scratch * attn_scratch) + 15) & ~(size_t)15;
     const long long avail = (long long)dv.max_smem - 1024 - (long long)(psum + misc + reg_a) - 2 * 64 * 8;
     int ns = (int)std::min<long long>(64, avail / kSlotBytes);
     const int tile_slots = (kAttnChunk / kBoxKeys) * std::max(1, c.head_dim / 64);
     if (ns < 2 * tile_slots || ns < 8) return false;
     pl->ns = ns;
-    pl->attn_groups = ns >= 4 * tile_slots ? 2 : 1;
+    pl->attn_groups = std::max(1, std::min(groups_by_scratch, ns / (2 * tile_slots)));
     pl->off_bars = ns * kSlotBytes;
     pl->off_misc = pl->off_bars + 2 * 64 * 8;
     pl->off_psum = pl->off_misc + (int)misc;

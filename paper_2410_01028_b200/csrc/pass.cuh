@@ -96,7 +96,7 @@ struct PassParams {
     // shared-memory plan (bytes from the 1024-aligned base)
     int ns;            // ring slots
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
-    int attn_groups;   // 1 or 2 groups of 4 warps work on attention items
+    int attn_groups;   // 1 to 3 groups of 4 warps work on attention items
     int off_bars, off_misc, off_psum, off_reg_a;
 };
 
@@ -160,10 +160,13 @@ __device__ __forceinline__ void cta_pairs(int n_rows, int& pair0, int& np) {
     np = pair1 - pair0;
 }
 
-__device__ __forceinline__ int attn_local_items(const PassParams& p, int M, int& n_chunks) {
+// Attention work items (kv head, 128-key chunk), head-major; CTA b takes the contiguous range
+// [b*T/G, (b+1)*T/G): mostly chunks of one head, so queries, tickets and DRAM pages are reused.
+__device__ __forceinline__ int attn_local_items(const PassParams& p, int M, int& n_chunks, int& first) {
     n_chunks = (p.pos0 + M - 1) / kAttnChunk + 1;
-    const int total = p.n_kv_heads * n_chunks;
-    return ((int)blockIdx.x < total) ? (total - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const long long total = (long long)p.n_kv_heads * n_chunks;
+    first = (int)((long long)blockIdx.x * total / gridDim.x);
+    return (int)((long long)(blockIdx.x + 1) * total / gridDim.x) - first;
 }
 
 // ============================================================================================ ring protocol
@@ -239,8 +242,8 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
         const StageDesc st = p.stages[s];
         if (st.type == kStEmbed || st.type == kStFinish) continue;
         if (st.type == kStAttn) {
-            int n_chunks;
-            const int n_local = attn_local_items(p, M, n_chunks);
+            int n_chunks, first;
+            const int n_local = attn_local_items(p, M, n_chunks, first);
             const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
             const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
             const uint32_t box_bytes = (uint32_t)kBoxKeys * box_cols * 2u;
@@ -250,7 +253,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 const int j = idx / (2 * tile_slots), r = idx - j * 2 * tile_slots;
                 const int which = r / tile_slots, t = r - which * tile_slots;
                 const int rg = t / nhb, hb = t - rg * nhb;
-                const int item = blockIdx.x + j * gridDim.x;
+                const int item = first + j;
                 const int kvh = item / n_chunks, chunk = item - kvh * n_chunks;
                 const uint32_t g = gi + (uint32_t)idx;
                 const int slot = ring_acquire(p, sm, g, s, M);
@@ -802,8 +805,8 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     const int nhb = hd > 64 ? hd / 64 : 1;
     const int box_cols = hd > 64 ? 64 : hd;
     const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
-    int n_chunks;
-    const int n_local = attn_local_items(p, M, n_chunks);
+    int n_chunks, first;
+    const int n_local = attn_local_items(p, M, n_chunks, first);
     const uint32_t gi0 = gi;
     gi += (uint32_t)(n_local * 2 * tile_slots);
     const int grp = warp >> 2;
@@ -824,8 +827,10 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     float* red = Ps + M * kAttnChunk;              // [4][kPassMaxRows]
     int* flag = reinterpret_cast<int*>(red + 4 * kPassMaxRows);
 
+    int q_head = -1;   // head whose queries are in qs
+    unsigned run_cnt = 0;  // chunks of the current head finished by this group and not yet reported
     for (int j = grp; j < n_local; j += p.attn_groups) {
-        const int idx = blockIdx.x + j * gridDim.x;
+        const int idx = first + j;
         const int kvh = idx / n_chunks, chunk = idx - kvh * n_chunks;
         const int key0 = chunk * kAttnChunk;
         const int last_pos = p.pos0 + M - 1;
@@ -846,7 +851,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         for (int u = 0; u < kQPerThread; ++u) {  // the first head's queries are requested before waiting for the tile
             const int i = gt + u * 128;
             const int m = i / hd, e = i - m * hd;
-            qreg[u] = (i < M * hd) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
+            qreg[u] = (i < M * hd && q_head != kvh * group) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
         }
         for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
         const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
@@ -865,15 +870,18 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             const int head = kvh * group + g;
             bar_sync(bar_id, 128);  // patched tile visible; previous head's Ps / qs consumed
             if (g == 0) {
+                if (q_head != head) {
 #pragma unroll
-                for (int u = 0; u < kQPerThread; ++u)
-                    if (gt + u * 128 < M * hd) qs[gt + u * 128] = __uint_as_float((uint32_t)qreg[u] << 16);
+                    for (int u = 0; u < kQPerThread; ++u)
+                        if (gt + u * 128 < M * hd) qs[gt + u * 128] = __uint_as_float((uint32_t)qreg[u] << 16);
+                }
             } else {
                 for (int i = gt; i < M * hd; i += 128) {
                     const int m = i / hd, e = i - m * hd;
                     qs[i] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)head * hd + e) << 16);
                 }
             }
+            q_head = head;
             bar_sync(bar_id, 128);
 
             if (j == 0 && g == 0) trace_mark(p, stage, 2);  // attention timeline: 2 = inputs staged, 4 = softmax done, 5 = P V done, 6 = ticket taken, 7 = merged
@@ -987,15 +995,24 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
         }
         if (j == 0) trace_mark(p, stage, 5);
-        // ---- release the V tile; the last group to finish this kv head merges its chunks in order
-        __threadfence();
+        // ---- release the V tile. Finished chunks are reported once per run of chunks of the same head; the group
+        //      whose report completes the head merges its chunks in order.
+        ++run_cnt;
+        const int jn = j + p.attn_groups;
+        const bool report = (jn >= n_local) || ((first + jn) / n_chunks != kvh);
+        if (report) __threadfence();
         bar_sync(bar_id, 128);
         if (gt == 0) {
             fence_proxy_async_smem();
             for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
-            const unsigned tk = atomicAdd(p.attn_counters + kvh, 1u);
-            *flag = (tk == (unsigned)n_chunks - 1) ? 1 : 0;
+            if (report) {
+                const unsigned tk = atomicAdd(p.attn_counters + kvh, run_cnt);
+                *flag = (tk + run_cnt == (unsigned)n_chunks) ? 1 : 0;
+            } else {
+                *flag = 0;
+            }
         }
+        if (report) run_cnt = 0;
         bar_sync(bar_id, 128);
         if (j == 0) trace_mark(p, stage, 6);
         if (*flag) {

@@ -155,6 +155,24 @@ int asd_generate(asd_ctx* ctx, const int32_t* prompt, int32_t n_prompt, const as
 int asd_generate_device(asd_ctx* ctx, const int32_t* dev_prompt, int32_t n_prompt, const asd_gen_params* p,
                         int32_t* dev_out, int32_t* n_out, asd_stats* stats);
 
+/* How asd_prefill (and the prefill inside asd_generate) processes the prompt, the first step of inference in
+ * Section 3.2. Either way it fills the KV cache, adds every prompt row's per-sublayer cosine similarity to the
+ * sums behind C_l and returns t_1.
+ *   ASD_PREFILL_ROWS  passes of up to 16 rows through the decode kernel: row r of the prompt is bit-identical to
+ *                     a one-row pass at the same position.
+ *   ASD_PREFILL_GEMM  all rows but the last as dense bf16 products on the tensor cores (fp32 accumulation, the
+ *                     same rounding points; the accumulation order differs, so results agree with
+ *                     ASD_PREFILL_ROWS to rounding, not bit for bit), then the last row as a one-row pass.
+ *                     Needs head_dim 64 or 128, else ASD_ERR_ARG.
+ *   ASD_PREFILL_AUTO  (default) ASD_PREFILL_GEMM for prompts of more than 32 tokens where the shape allows it,
+ *                     otherwise ASD_PREFILL_ROWS.
+ * After a prompt that took the dense path, asd_get_last_cosines / asd_get_last_logits describe the one-row
+ * pass of the last prompt token. */
+#define ASD_PREFILL_AUTO 0
+#define ASD_PREFILL_ROWS 1
+#define ASD_PREFILL_GEMM 2
+int asd_set_prefill_mode(asd_ctx* ctx, int32_t mode);
+
 /* Per-row results of the last pass of M rows: cosines [L][M] (NaN where the sublayer was skipped),
  * argmax [M]. *M receives the row count. Any output may be NULL. */
 int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_mlp);
@@ -173,6 +191,17 @@ int asd_get_last_trace(asd_ctx* ctx, int32_t* n_stages, int32_t* n_ctas, int64_t
 int asd_get_kv(asd_ctx* ctx, int32_t layer, int32_t pos, uint16_t* k, uint16_t* v);
 int asd_get_positions(asd_ctx* ctx, int32_t* n_committed, int32_t* draft_cursor);
 int asd_get_stats(asd_ctx* ctx, asd_stats* stats);
+
+/* ------------------------------------------------------------------------------------------------------
+ * The dense product of the prompt path on its own (kernel-level tests and micro-benchmarks; Section 3.2: the
+ * prompt goes through every sublayer of M at once):  C[M, N] = A[M, K] * W[N, K]^T.
+ * All pointers are DEVICE pointers, 16-byte aligned: A and W bf16 row-major (raw 16-bit patterns), K % 8 == 0;
+ * C float row-major [M, N]; dev_status 8 ints that the call clears on the stream and that stay 0 unless a
+ * bounded device-side wait expired (word 0 != 0: C is not valid). The kernel is enqueued on the stream; the
+ * call does not wait for it. Nothing is allocated. Returns ASD_ERR_ARG for bad arguments, ASD_ERR_CUDA when
+ * the tensor maps cannot be encoded or the launch fails. */
+int asd_gemm_bf16(void* cuda_stream, int32_t M, int32_t N, int32_t K, const uint16_t* A, const uint16_t* W, float* C,
+                  int32_t* dev_status);
 
 /* ------------------------------------------------------------------------------------------------------
  * The sublayer building block on its own (kernel-level tests and micro-benchmarks): one fused

@@ -4,6 +4,7 @@ Every step of the method runs in the CUDA library; this package only marshals ar
 PyTorch is used for device memory and the CUDA stream, nothing else.
 """
 from .binding import (  # noqa: F401
-    ADMG_ALL, EPI_PLAIN, EPI_RESIDUAL, EPI_SWIGLU, MODE_AR, MODE_SPEC, MODE_SPEC_MANUAL_MASK, USE_CS, USE_RULE1,
-    USE_RULE2, AsdError, Decoder, admg, fused_gemv, fused_gemv_scratch_bytes, fused_gemv_static, lib, workspace_bytes,
+    ADMG_ALL, EPI_PLAIN, EPI_RESIDUAL, EPI_SWIGLU, MODE_AR, MODE_SPEC, MODE_SPEC_MANUAL_MASK, PREFILL_AUTO, PREFILL_GEMM,
+    PREFILL_ROWS, USE_CS, USE_RULE1, USE_RULE2, AsdError, Decoder, admg, fused_gemv, fused_gemv_scratch_bytes, fused_gemv_static,
+    gemm_bf16, lib, workspace_bytes,
 )

@@ -11,6 +11,7 @@ from . import build as _build
 USE_CS, USE_RULE1, USE_RULE2, ADMG_ALL = 1, 2, 4, 7
 MODE_AR, MODE_SPEC, MODE_SPEC_MANUAL_MASK = 0, 1, 2
 EPI_PLAIN, EPI_SWIGLU, EPI_RESIDUAL = 0, 1, 2
+PREFILL_AUTO, PREFILL_ROWS, PREFILL_GEMM = 0, 1, 2
 OK, ERR_ARG, ERR_STATE, ERR_NOMEM, ERR_OVERFLOW, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_IO = 0, -1, -2, -3, -4, -5, -6, -7
 
 
@@ -51,7 +52,7 @@ EXPORTS = (
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
     "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
-    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg",
+    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_set_prefill_mode", "asd_gemm_bf16",
 )
 
 _lib = None
@@ -142,6 +143,20 @@ def fused_gemv_static(x, W, epilogue, out, gain=None, eps=1e-5, cos=None, stream
         raise AsdError(rc, "asd_fused_gemv_static")
 
 
+def gemm_bf16(A, W, C, status, stream=None):
+    """asd_gemm_bf16 on torch CUDA tensors: C[M, N] (float32) = A[M, K] (bfloat16) @ W[N, K]^T (bfloat16).
+    ``status`` is an int32 CUDA tensor of 8 elements; element 0 stays 0 unless a device-side wait expired."""
+    import torch
+    M, K = A.shape
+    N = W.shape[0]
+    assert W.shape[1] == K and tuple(C.shape) == (M, N) and status.numel() >= 8
+    st = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    rc = lib().asd_gemm_bf16(ctypes.c_void_p(st), ctypes.c_int32(M), ctypes.c_int32(N), ctypes.c_int32(K), _vp(A), _vp(W),
+                             _vp(C), _vp(status))
+    if rc:
+        raise AsdError(rc, "asd_gemm_bf16")
+
+
 class Decoder:
     """One decoding context. The workspace is a torch uint8 CUDA tensor; work runs on torch's current stream."""
 
@@ -210,6 +225,10 @@ class Decoder:
     def set_debug(self, record_logits=True, trace=False):
         flags = (1 if record_logits else 0) | (2 if trace else 0)
         self._check(lib().asd_set_debug(self._ctx, ctypes.c_int32(flags)), "asd_set_debug")
+
+    def set_prefill_mode(self, mode):
+        """PREFILL_AUTO (default), PREFILL_ROWS (row passes, bit-identical to one-row passes) or PREFILL_GEMM."""
+        self._check(lib().asd_set_prefill_mode(self._ctx, ctypes.c_int32(mode)), "asd_set_prefill_mode")
 
     def get_last_trace(self):
         """Per-stage device timeline of the last pass: int64 array [n_stages, 8, n_ctas] (see asd_get_last_trace)."""

@@ -11,6 +11,7 @@
 #include "../../include/asd.h"
 #include "common.cuh"
 #include "pass.cuh"
+#include "prefill.h"
 
 namespace asd {
 
@@ -86,6 +87,7 @@ static cudaError_t device_info(DeviceInfo** out) {
         if ((e = configure_m8(d.max_smem)) != cudaSuccess) return e;
         if ((e = configure_m9(d.max_smem)) != cudaSuccess) return e;
         if ((e = configure_m16(d.max_smem)) != cudaSuccess) return e;
+        if ((e = configure_prefill(d.max_smem)) != cudaSuccess) return e;
         d.ready = true;
     }
     *out = &d;
@@ -156,7 +158,17 @@ struct Layout {
     int max_stages;
     size_t total;
     int chunk_stride;
+    // dense prompt path: row-major copies of the sublayer matrices (one block per layer) and activations of a chunk
+    size_t rm_layers, rm_layer_stride, rm_wqkv, rm_wo, rm_wgu, rm_wd;
+    size_t pf_x, pf_xn, pf_q, pf_a, pf_t, pf_c, pf_cos;
+    int pf_rows;  // prompt rows per chunk of the dense path (0: shape not supported by it)
 };
+
+constexpr int kPrefillChunk = 2048;      // most prompt rows one chunk of the dense prompt path holds
+constexpr int kPrefillGemmMinRows = 32;  // shorter prompts take the row passes (default mode)
+
+// the dense prompt path needs whole 32-column groups inside a head (rotary epilogue) and a flash kernel for head_dim
+static bool dense_prefill_supported(const asd_config& c) { return c.n_layers > 0 && (c.head_dim == 64 || c.head_dim == 128); }
 
 static bool check_config(const asd_config& c) {
     if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.d_ffn <= 0 ||
@@ -231,6 +243,30 @@ static Layout make_layout(const asd_config& c) {
     L.sync_words = take(256);
     L.resid_tab = take((size_t)2 * (2 * std::max(c.n_layers, 1)) * sizeof(ResidOut));
     L.trace = take((size_t)L.max_stages * 8 * kMaxGemvGrid * 8);
+    L.pf_rows = 0;
+    if (dense_prefill_supported(c)) {
+        L.pf_rows = (int)std::min<size_t>(kPrefillChunk, (S + kGemmBM - 1) / kGemmBM * kGemmBM);
+        const size_t R = L.pf_rows;
+        size_t lo = 0;
+        auto ltake = [&](size_t bytes) {
+            size_t at = lo;
+            lo = align_up(lo + bytes);
+            return at;
+        };
+        L.rm_wqkv = ltake((d + 2 * kvd) * d * 2);
+        L.rm_wo = ltake(d * d * 2);
+        L.rm_wgu = ltake(2 * f * d * 2);
+        L.rm_wd = ltake(d * f * 2);
+        L.rm_layer_stride = lo;
+        L.rm_layers = take(L.rm_layer_stride * c.n_layers);
+        L.pf_x = take(R * d * 4);
+        L.pf_xn = take(R * d * 2);
+        L.pf_q = take(R * d * 2);
+        L.pf_a = take(R * d * 2);
+        L.pf_t = take(R * f * 2);
+        L.pf_c = take(R * d * 4);
+        L.pf_cos = take((size_t)2 * c.n_layers * R * 4);
+    }
     L.total = o;
     return L;
 }
@@ -254,6 +290,11 @@ struct asd_ctx {
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, trace = false;
     int last_n_stages = 0;
+    int prefill_mode = ASD_PREFILL_AUTO;
+    // tensor maps of the dense prompt path (host copies, passed to the kernels by value): activations with boxes of
+    // 64 x 128, and per layer the four matrices with boxes of 64 x 128 ([0..3]) and 64 x 256 ([4..7])
+    CUtensorMap tm_xn{}, tm_a{}, tm_t{};
+    std::vector<CUtensorMap> tm_w;
     asd_stats stats{};
     int32_t* pinned = nullptr;  // small host staging buffer
     uint32_t bar_base = 0;      // value of the grid-barrier counter at the start of the next pass
@@ -315,15 +356,32 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// bf16 matrix [rows, inner] row-major as a GEMM operand: boxes of 64 x box_rows elements, 128-byte swizzle, zeros
+// outside the matrix
+static bool encode_operand_map(EncodeTiledFn encode, CUtensorMap* m, void* base, size_t inner, size_t rows, uint32_t box_rows) {
+    const cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)inner * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kGemmBK, box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static EncodeTiledFn tensor_map_encoder() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+        return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
 // One 2-D tensor map per layer and per cache: [max_seq rows, kv_dim columns] bf16, boxes of 64 keys x (up to) 64
 // columns; 128-byte rows are stored with the 128-byte swizzle so that one thread per key reads its row without
 // shared-memory bank conflicts.
 static int make_tensor_maps(asd_ctx* x) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    ASD_CUDA(x, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-    if (!fn || qres != cudaDriverEntryPointSuccess) return fail(x, ASD_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
-    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return fail(x, ASD_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     const asd_config& c = x->c;
     const int L = c.n_layers;
     std::vector<CUtensorMap> maps((size_t)2 * std::max(L, 1));
@@ -343,6 +401,28 @@ static int make_tensor_maps(asd_ctx* x) {
         }
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + x->lay.tmaps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, x->stream));
     ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    if (x->lay.pf_rows > 0) {
+        // operands of the dense prompt path: bf16 [rows, inner] row-major, boxes of 64 inner elements (128 bytes, the
+        // swizzle span) x box_rows rows
+        const Layout& ly = x->lay;
+        const size_t d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, R = ly.pf_rows;
+        bool ok = encode_operand_map(encode, &x->tm_xn, x->ws + ly.pf_xn, d, R, kGemmBM) &&
+                  encode_operand_map(encode, &x->tm_a, x->ws + ly.pf_a, d, R, kGemmBM) &&
+                  encode_operand_map(encode, &x->tm_t, x->ws + ly.pf_t, f, R, kGemmBM);
+        x->tm_w.assign((size_t)8 * L, CUtensorMap{});
+        for (int l = 0; l < L && ok; ++l) {
+            unsigned char* rw = x->ws + ly.rm_layers + (size_t)l * ly.rm_layer_stride;
+            for (int v = 0; v < 2 && ok; ++v) {
+                const uint32_t bn = v ? 256u : 128u;
+                CUtensorMap* m = &x->tm_w[(size_t)l * 8 + v * 4];
+                ok = encode_operand_map(encode, m + 0, rw + ly.rm_wqkv, d, d + 2 * kvd, bn) &&
+                     encode_operand_map(encode, m + 1, rw + ly.rm_wo, d, d, bn) &&
+                     encode_operand_map(encode, m + 2, rw + ly.rm_wgu, d, 2 * f, bn) &&
+                     encode_operand_map(encode, m + 3, rw + ly.rm_wd, f, d, bn);
+            }
+        }
+        if (!ok) return fail(x, ASD_ERR_CUDA, "cuTensorMapEncodeTiled failed for an operand of the dense prompt path");
+    }
     return ASD_OK;
 }
 
@@ -495,10 +575,11 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
 // the bounded waits of the pass kernel report through eight device words; word 0 = 0 means no error
 static int check_device_error(asd_ctx* x, const int32_t* w) {
     if (w[0] == 0) return ASD_OK;
-    static const char* names[] = {"", "a ring slot was never filled", "a ring slot was never released", "the grid barrier never completed"};
+    static const char* names[] = {"", "a ring slot was never filled", "a ring slot was never released", "the grid barrier never completed",
+                                  "a pipeline barrier of the prompt GEMM never completed"};
     char buf[256];
-    snprintf(buf, sizeof buf, "pass kernel gave up waiting: %s (stage %d, item %d, slot %d, CTA %d, thread %d, tag %d, parity %d)",
-             (w[0] >= 1 && w[0] <= 3) ? names[w[0]] : "unknown", w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+    snprintf(buf, sizeof buf, "a kernel gave up waiting: %s (stage %d, item %d, slot %d, CTA %d, thread %d, tag %d, parity %d)",
+             (w[0] >= 1 && w[0] <= 4) ? names[w[0]] : "unknown", w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
     return fail(x, ASD_ERR_DEVICE_TIMEOUT, buf);
 }
 
@@ -643,6 +724,17 @@ static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size
     return ASD_OK;
 }
 
+// Row-major copy of one matrix for the dense prompt path: row n of the copy is host row row(n).
+template <class RowFn>
+static int upload_rowmajor(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, std::vector<unsigned char>& staging) {
+    staging.resize(n_rows * n_in * 2);
+#pragma omp parallel for schedule(static)
+    for (long long n = 0; n < (long long)n_rows; ++n) memcpy(staging.data() + (size_t)n * n_in * 2, row((size_t)n), n_in * 2);
+    ASD_CUDA(x, cudaMemcpyAsync(dev_dst, staging.data(), staging.size(), cudaMemcpyHostToDevice, x->stream));
+    ASD_CUDA(x, cudaStreamSynchronize(x->stream));  // staging is reused by the next matrix
+    return ASD_OK;
+}
+
 static int upload_weights(asd_ctx* x, const asd_host_weights& w) {
     const asd_config& c = x->c;
     const Layout& ly = x->lay;
@@ -680,6 +772,23 @@ static int upload_weights(asd_ctx* x, const asd_host_weights& w) {
             return rc;
         const uint16_t* wd = w.wd + (size_t)l * d * f;
         if ((rc = upload_packed(x, lw + ly.l_wd, d, f, [&](size_t r) { return wd + r * f; }, plain_pair, staging))) return rc;
+        if (ly.pf_rows > 0) {
+            // dense prompt path: inside every q and k head the rotary partners (j, j + head_dim/2) become neighbouring
+            // rows (2j, 2j+1); gate_i and up_i alternate; the other matrices keep their order
+            unsigned char* rw = x->ws + ly.rm_layers + (size_t)l * ly.rm_layer_stride;
+            auto qkv_rm = [&](size_t n) {
+                if (n >= d + kvd) return wv + (n - d - kvd) * d;
+                const uint16_t* basep = n < d ? wq : wk;
+                const size_t c = n < d ? n : n - d;
+                const size_t head = c / hd, local = c % hd;
+                return basep + (head * hd + local / 2 + (local & 1) * half) * d;
+            };
+            if ((rc = upload_rowmajor(x, rw + ly.rm_wqkv, d + 2 * kvd, d, qkv_rm, staging))) return rc;
+            if ((rc = upload_rowmajor(x, rw + ly.rm_wo, d, d, [&](size_t r) { return wo + r * d; }, staging))) return rc;
+            if ((rc = upload_rowmajor(x, rw + ly.rm_wgu, 2 * f, d, [&](size_t r) { return (r & 1) ? wu + (r / 2) * d : wg + (r / 2) * d; }, staging)))
+                return rc;
+            if ((rc = upload_rowmajor(x, rw + ly.rm_wd, d, f, [&](size_t r) { return wd + r * f; }, staging))) return rc;
+        }
     }
     ASD_CUDA(x, cudaStreamSynchronize(s));
     x->have_weights = true;
@@ -732,6 +841,71 @@ extern "C" int asd_reset(asd_ctx* x) {
 }
 
 // ---------------------------------------------------------------- prefill (Section 3.2)
+// One sublayer product of the dense prompt path: the 64 x 256 weight boxes when that still gives every SM a tile.
+static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which, int M, int N, int K, const GemmEpi& ep) {
+    const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
+    const int bn = (((N + 255) / 256) * m_tiles >= x->dev->num_sms) ? 256 : 128;
+    const CUtensorMap& tm_w = x->tm_w[(size_t)layer * 8 + (bn == 256 ? 4 : 0) + which];
+    ASD_CUDA(x, launch_gemm_tn(tm_a, tm_w, M, N, K, bn, ep, x->stream));
+    x->stats.kernel_launches += 1;
+    return ASD_OK;
+}
+
+// Prompt rows [0, n) at positions pos0 + r through every layer of M as dense products: K/V appended to the cache,
+// each row's cosine similarity of every sublayer added to the sums behind C_l. No LM head: the caller feeds the
+// last prompt row through a one-row pass.
+static int prefill_dense(asd_ctx* x, const int32_t* dev_tokens, int n, int pos0) {
+    const asd_config& c = x->c;
+    const Layout& ly = x->lay;
+    const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers, R = ly.pf_rows;
+    cudaStream_t s = x->stream;
+    float* px = x->at<float>(ly.pf_x);
+    float* pc = x->at<float>(ly.pf_c);
+    float* pcos = x->at<float>(ly.pf_cos);
+    __nv_bfloat16* pxn = x->at<__nv_bfloat16>(ly.pf_xn);
+    __nv_bfloat16* pq = x->at<__nv_bfloat16>(ly.pf_q);
+    __nv_bfloat16* pa = x->at<__nv_bfloat16>(ly.pf_a);
+    __nv_bfloat16* pt = x->at<__nv_bfloat16>(ly.pf_t);
+    int* err = reinterpret_cast<int*>(x->at<unsigned>(ly.sync_words) + 32);
+    const float scale = 1.0f / sqrtf((float)c.head_dim);
+    int rc;
+    for (int c0 = 0; c0 < n; c0 += R) {
+        const int rows = std::min(R, n - c0), p0 = pos0 + c0;
+        auto gain = [&](int l, size_t off) { return reinterpret_cast<const __nv_bfloat16*>(x->layer(l) + off); };
+        ASD_CUDA(x, launch_embed_norm(dev_tokens + c0, rows, d, c.vocab, x->at<__nv_bfloat16>(ly.embed), gain(0, ly.l_attn_norm), c.rms_eps, px, pxn, s));
+        for (int l = 0; l < L; ++l) {
+            __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.kcache + (size_t)l * ly.kv_layer_stride);
+            __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(x->ws + ly.vcache + (size_t)l * ly.kv_layer_stride);
+            GemmEpi e{};
+            e.err = err;
+            e.mode = kGemmQkv;
+            e.q = pq, e.k_cache = kc, e.v_cache = vc;
+            e.rope_cos = x->at<float>(ly.rope_cos), e.rope_sin = x->at<float>(ly.rope_sin);
+            e.pos0 = p0, e.d_model = d, e.kv_dim = kvd, e.head_dim = c.head_dim;
+            if ((rc = dense_gemm(x, x->tm_xn, l, 0, rows, d + 2 * kvd, d, e))) return rc;
+            ASD_CUDA(x, launch_flash_prefill(pq, kc, vc, pa, rows, p0, d, kvd, c.head_dim, c.n_heads, c.n_kv_heads, c.max_seq, scale, s));
+            GemmEpi o{};
+            o.err = err;
+            o.mode = kGemmF32;
+            o.c = pc, o.ldc = d;
+            if ((rc = dense_gemm(x, x->tm_a, l, 1, rows, d, d, o))) return rc;
+            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, gain(l, ly.l_mlp_norm), c.rms_eps, pxn, pcos + (size_t)l * R, s));
+            GemmEpi g{};
+            g.err = err;
+            g.mode = kGemmSwiglu;
+            g.t = pt, g.ldt = f;
+            if ((rc = dense_gemm(x, x->tm_xn, l, 2, rows, 2 * f, d, g))) return rc;
+            if ((rc = dense_gemm(x, x->tm_t, l, 3, rows, d, f, o))) return rc;
+            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, l + 1 < L ? gain(l + 1, ly.l_attn_norm) : nullptr, c.rms_eps, pxn,
+                                          pcos + (size_t)(L + l) * R, s));
+            x->stats.kernel_launches += 3;
+        }
+        ASD_CUDA(x, launch_sumcos(pcos, R, rows, 2 * L, x->at<double>(ly.sumcos), s));
+        x->stats.kernel_launches += 2;
+    }
+    return ASD_OK;
+}
+
 static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int32_t* first_token, bool resolve) {
     if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
     if (n <= 0) return fail(x, ASD_ERR_ARG, "empty prompt");
@@ -740,7 +914,16 @@ static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int3
     int rc = new_event(x, &e0);
     if (rc) return rc;
     int last_rows = 0;
-    for (int c0 = 0, M = 0; c0 < n; c0 += M) {
+    // Long prompts: all rows but the last as dense products on the tensor cores; the last row then takes a one-row
+    // pass, which also runs the LM head. Short prompts (and ASD_PREFILL_ROWS): row passes only.
+    int n_dense = 0;
+    if (x->prefill_mode == ASD_PREFILL_GEMM && x->lay.pf_rows == 0)
+        return fail(x, ASD_ERR_ARG, "the dense prompt path needs head_dim 64 or 128 and at least one layer");
+    if (x->lay.pf_rows > 0 && x->prefill_mode != ASD_PREFILL_ROWS && n > 1 &&
+        (x->prefill_mode == ASD_PREFILL_GEMM || n - 1 >= kPrefillGemmMinRows))
+        n_dense = n - 1;
+    if (n_dense > 0 && (rc = prefill_dense(x, dev_tokens, n_dense, x->n_committed))) return rc;
+    for (int c0 = n_dense, M = 0; c0 < n; c0 += M) {
         // row counts the pass kernel is built for: 16, or 1..9
         const int left = n - c0;
         M = left >= kPrefillRows ? kPrefillRows : (left > kMaxRows ? 8 : left);
@@ -1035,6 +1218,14 @@ extern "C" int asd_set_debug(asd_ctx* x, int32_t flags) {
     return ASD_OK;
 }
 
+extern "C" int asd_set_prefill_mode(asd_ctx* x, int32_t mode) {
+    if (!x || mode < ASD_PREFILL_AUTO || mode > ASD_PREFILL_GEMM) return ASD_ERR_ARG;
+    if (mode == ASD_PREFILL_GEMM && x->lay.pf_rows == 0)
+        return fail(x, ASD_ERR_ARG, "the dense prompt path needs head_dim 64 or 128 and at least one layer");
+    x->prefill_mode = mode;
+    return ASD_OK;
+}
+
 extern "C" int asd_get_last_trace(asd_ctx* x, int32_t* n_stages, int32_t* n_ctas, int64_t* ns_out) {
     if (!x) return ASD_ERR_ARG;
     if (!x->trace || x->last_n_stages == 0) return fail(x, ASD_ERR_STATE, "no pass has run with tracing on (asd_set_debug bit 1)");
@@ -1110,6 +1301,31 @@ extern "C" int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_
     p.x_in_smem = xin;
     if (launch_gemv(M, epilogue, gain != nullptr, p, grid, smem, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return ASD_ERR_CUDA;
+    return ASD_OK;
+}
+
+// ---------------------------------------------------------------- the dense product of the prompt path on its own
+extern "C" int asd_gemm_bf16(void* cuda_stream, int32_t M, int32_t N, int32_t K, const uint16_t* A, const uint16_t* W, float* C,
+                             int32_t* dev_status) {
+    if (!A || !W || !C || !dev_status || M <= 0 || N <= 0 || K <= 0 || K % 8) return ASD_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)W | (uintptr_t)C) % 16) return ASD_ERR_ARG;
+    DeviceInfo* dv = nullptr;
+    if (device_info(&dv) != cudaSuccess) return ASD_ERR_CUDA;
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return ASD_ERR_CUDA;
+    const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
+    const int bn = (((N + 255) / 256) * m_tiles >= dv->num_sms) ? 256 : 128;
+    CUtensorMap tm_a, tm_w;
+    if (!encode_operand_map(encode, &tm_a, const_cast<uint16_t*>(A), (size_t)K, (size_t)M, kGemmBM) ||
+        !encode_operand_map(encode, &tm_w, const_cast<uint16_t*>(W), (size_t)K, (size_t)N, (uint32_t)bn))
+        return ASD_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(dev_status, 0, 32, s) != cudaSuccess) return ASD_ERR_CUDA;
+    GemmEpi e{};
+    e.mode = kGemmF32;
+    e.err = dev_status;
+    e.c = C, e.ldc = N;
+    if (launch_gemm_tn(tm_a, tm_w, M, N, K, bn, e, s) != cudaSuccess) return ASD_ERR_CUDA;
     return ASD_OK;
 }
 

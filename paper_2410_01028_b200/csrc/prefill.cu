@@ -395,7 +395,8 @@ cudaError_t launch_sumcos(const float* cos_rows, int stride, int n_rows, int n_s
 // One CTA = 64 query rows of one head (4 warps x 16 rows); keys and values stream through shared memory in tiles of
 // 64 keys (double-buffered cp.async). Scores are bf16 x bf16 products accumulated in fp32 (mma.sync m16n8k16), the
 // softmax is kept on line in fp32 (running maximum and sum per row), and the probabilities enter the P V product as
-// the sum of two bf16 numbers (p = hi + lo, two MMAs), which keeps 16 bits of each fp32 probability.
+// the sum of three bf16 numbers (p = hi + mid + lo, three MMAs), which represents every fp32 probability exactly:
+// with fewer terms the 2^-17 error of P flips bf16 roundings of the attention output in about every second row.
 constexpr int kFaRows = 64, kFaKeys = 64, kFaThreads = 128;
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
@@ -537,27 +538,32 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
             o[i][0] *= alpha[0], o[i][1] *= alpha[0];
             o[i][2] *= alpha[1], o[i][3] *= alpha[1];
         }
-        // ---- O += P V, P = hi + lo in bf16
+        // ---- O += P V, P = hi + mid + lo in bf16
 #pragma unroll
         for (int kk = 0; kk < kFaKeys / 16; ++kk) {
-            uint32_t a_hi[4], a_lo[4];
+            uint32_t a_hi[4], a_mid[4], a_lo[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int nt = 2 * kk + (u >> 1), e = (u & 1) * 2;
                 const float p0 = sc[nt][e], p1 = sc[nt][e + 1];
                 const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
-                const __nv_bfloat162 lo = __floats2bfloat162_rn(p0 - __low2float(hi), p1 - __high2float(hi));
+                const float r0 = p0 - __low2float(hi), r1 = p1 - __high2float(hi);  // exact
+                const __nv_bfloat162 mid = __floats2bfloat162_rn(r0, r1);
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(r0 - __low2float(mid), r1 - __high2float(mid));
                 a_hi[u] = *reinterpret_cast<const uint32_t*>(&hi);
+                a_mid[u] = *reinterpret_cast<const uint32_t*>(&mid);
                 a_lo[u] = *reinterpret_cast<const uint32_t*>(&lo);
             }
 #pragma unroll
             for (int n2 = 0; n2 < HD / 16; ++n2) {
                 uint32_t b[4];
                 ldsm_x4_trans(b, Vb + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + n2 * 16 + (lane >> 4) * 8);
+                mma16816(o[2 * n2], a_lo, b[0], b[1]);  // smallest terms first
+                mma16816(o[2 * n2 + 1], a_lo, b[2], b[3]);
+                mma16816(o[2 * n2], a_mid, b[0], b[1]);
+                mma16816(o[2 * n2 + 1], a_mid, b[2], b[3]);
                 mma16816(o[2 * n2], a_hi, b[0], b[1]);
                 mma16816(o[2 * n2 + 1], a_hi, b[2], b[3]);
-                mma16816(o[2 * n2], a_lo, b[0], b[1]);
-                mma16816(o[2 * n2 + 1], a_lo, b[2], b[3]);
             }
         }
         __syncthreads();  // this buffer is refilled two iterations from now

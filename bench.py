@@ -56,6 +56,7 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=5, help="ADMG rule subset: 1=CS thresholding, 2=rule 1, 4=rule 2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemv-microbench", action="store_true", help="also time the stand-alone fused GEMV kernel")
+    ap.add_argument("--gemm-microbench", action="store_true", help="also time the stand-alone tensor-core GEMM of the prompt path")
     # reduced cases for profiler captures only (never for a reported number)
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
     ap.add_argument("--max-new", type=int, default=0, help="override the workload's generation length")
@@ -69,6 +70,25 @@ def peaks():
         with open(path) as fh:
             return float(json.load(fh)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def tensor_peak():
+    """Dense bf16 TFLOP/s of a cuBLAS GEMM on this machine: (burst, sustained, kind)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return 1590.0, 1400.0, "fallback"
+
+
+def prefill_flops(shape, S):
+    """Floating-point operations of the prompt pass (Section 3.2): the sublayer products of all S rows, the LM head of
+    the last row, and causal attention (Q K^T and P V over keys <= the row's position)."""
+    d, f, L, kvd = shape.d_model, shape.d_ffn, shape.n_layers, shape.kv_dim
+    per_row = 2.0 * L * (d * (d + 2 * kvd) + d * d + 3 * d * f)
+    attn = 2.0 * 2.0 * L * d * (S * (S + 1) / 2.0)
+    return S * per_row + attn + 2.0 * shape.vocab * d
 
 
 class ClockSampler:
@@ -211,6 +231,37 @@ def gemv_roofline(torch, asd, shape, hbm_peak):
             "us_per_launch": us, "achieved": achieved, "pool_matrices": pool}
 
 
+def gemm_roofline(torch, asd, shape):
+    """Times the stand-alone tcgen05 GEMM of the prompt path at the gate/up shape with 2048 rows (one chunk), over a
+    pool of weight matrices larger than L2, with CUDA events on the launching stream."""
+    d, n_rows, M = shape.d_model, 2 * shape.d_ffn, 2048
+    dev = torch.device("cuda")
+    pool = max(2, int(400e6 // (n_rows * d * 2)) + 1)
+    W = [torch.from_numpy(synth.make_matrix_bf16((n_rows, d), seed=7, stream=100 + i).view(np.int16)).to(dev)
+         .view(torch.bfloat16) for i in range(min(pool, 2))]
+    while len(W) < pool:
+        W.append(W[len(W) % 2].clone())
+    A = torch.from_numpy(synth.make_matrix_bf16((M, d), seed=7, stream=97, std=1.0).view(np.int16)).to(dev).view(torch.bfloat16)
+    C = torch.empty((M, n_rows), dtype=torch.float32, device=dev)
+    status = torch.zeros(8, dtype=torch.int32, device=dev)
+    n = 50
+    for i in range(5):
+        asd.gemm_bf16(A, W[i % pool], C, status)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        asd.gemm_bf16(A, W[i % pool], C, status)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    burst, _, kind = tensor_peak()
+    tf = 2.0 * M * n_rows * d / (us * 1e-6) / 1e12
+    return {"bound": "tensor", "kernel": "gemm_tn_kernel<256> %dx%dx%d (fp32 out)" % (M, n_rows, d), "us_per_launch": us,
+            "achieved": tf, "peak": burst, "unit": "TFLOP/s", "frac": tf / burst, "peak_kind": kind + " burst (kernel timed alone)",
+            "status": int(status[0].item())}
+
+
 def run_ours(args):
     import torch
     import paper_2410_01028_b200 as asd
@@ -312,6 +363,15 @@ def run_ours(args):
                 "how": "CUDA events around every launch inside the timed region, on the launching stream"}
     if args.gemv_microbench:
         roofline["fused_gemv_alone"] = gemv_roofline(torch, asd, shape, hbm_peak)
+    # the prompt pass is the tensor-core part of a step: dense products + causal attention, then one decode pass
+    _, tf_sustained, tf_kind = tensor_peak()
+    pf_ms = agg["ms_prefill"] / args.steps
+    pf_tf = prefill_flops(shape, S) / (pf_ms * 1e-3) / 1e12
+    prefill = {"ms": pf_ms, "bound": "tensor", "achieved": pf_tf, "peak": tf_sustained, "unit": "TFLOP/s",
+               "frac": pf_tf / tf_sustained, "peak_kind": tf_kind + " sustained",
+               "what": "whole prompt pass (GEMMs on tcgen05, flash attention, row kernels, one decode pass for the last row)"}
+    if args.gemm_microbench:
+        prefill["gemm_alone"] = gemm_roofline(torch, asd, shape)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -321,7 +381,7 @@ def run_ours(args):
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "roofline": roofline, "passes": passes,
         "decode_tokens_per_s": (new - 1) / ((agg["ms_total"] - agg["ms_prefill"]) / args.steps * 1e-3),
-        "prefill_ms": agg["ms_prefill"] / args.steps,
+        "prefill_ms": agg["ms_prefill"] / args.steps, "prefill": prefill,
         "ar_tokens_per_s": new / (st_ar["ms_total"] * 1e-3),
         "ar_decode_tokens_per_s": (new - 1) / ((st_ar["ms_total"] - st_ar["ms_prefill"]) * 1e-3),
         "acceptance": agg["accepted"] / max(agg["drafted"], 1), "rounds_per_step": agg["rounds"] / args.steps,

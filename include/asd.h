@@ -180,12 +180,13 @@ int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_m
 int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
 /* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline. */
 int asd_set_debug(asd_ctx* ctx, int32_t flags);
-/* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][8][n_ctas]. Entries 0-3 are device
+/* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][12][n_ctas]. Entries 0-3 are device
  * timestamps in ns of every CTA: 0 = stage entered, 1 = inputs of the stage ready (previous stage finished on
  * all CTAs), 2 = weight streaming done, 3 = stage left. Entries 4 and 5 are SM cycles that the CTA's first
  * consumer warp spent waiting for ring slots and working on them; entries 6 and 7 are timestamps of a GEMV stage
- * after the RMSNorm statistics and after the first activation window is in shared memory. Call first with
- * ns_out = NULL for the sizes. */
+ * after the RMSNorm statistics and after the first activation window is in shared memory. Entries 8-10 are the
+ * producer's: timestamps of its first and last copy of the stage, and the SM cycles it waited for free ring
+ * slots in between (one of its lanes); entry 11 is unused. Call first with ns_out = NULL for the sizes. */
 int asd_get_last_trace(asd_ctx* ctx, int32_t* n_stages, int32_t* n_ctas, int64_t* ns_out);
 /* K and V rows (bf16 patterns, n_kv_heads*head_dim each) of one layer (0-based) at one position. */
 int asd_get_kv(asd_ctx* ctx, int32_t layer, int32_t pos, uint16_t* k, uint16_t* v);

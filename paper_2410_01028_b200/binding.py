@@ -231,10 +231,10 @@ class Decoder:
         self._check(lib().asd_set_prefill_mode(self._ctx, ctypes.c_int32(mode)), "asd_set_prefill_mode")
 
     def get_last_trace(self):
-        """Per-stage device timeline of the last pass: int64 array [n_stages, 8, n_ctas] (see asd_get_last_trace)."""
+        """Per-stage device timeline of the last pass: int64 array [n_stages, 12, n_ctas] (see asd_get_last_trace)."""
         ns, nc = ctypes.c_int32(), ctypes.c_int32()
         self._check(lib().asd_get_last_trace(self._ctx, ctypes.byref(ns), ctypes.byref(nc), None), "asd_get_last_trace")
-        out = np.zeros((ns.value, 8, nc.value), np.int64)
+        out = np.zeros((ns.value, 12, nc.value), np.int64)
         self._check(lib().asd_get_last_trace(self._ctx, ctypes.byref(ns), ctypes.byref(nc), _vp(out)), "asd_get_last_trace")
         return out
 

@@ -2,6 +2,7 @@
 // and the C ABI declared in include/asd.h.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -242,7 +243,7 @@ static Layout make_layout(const asd_config& c) {
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
     L.sync_words = take(256);
     L.resid_tab = take((size_t)2 * (2 * std::max(c.n_layers, 1)) * sizeof(ResidOut));
-    L.trace = take((size_t)L.max_stages * 8 * kMaxGemvGrid * 8);
+    L.trace = take((size_t)L.max_stages * kTraceEntries * kMaxGemvGrid * 8);
     L.pf_rows = 0;
     if (dense_prefill_supported(c)) {
         L.pf_rows = (int)std::min<size_t>(kPrefillChunk, (S + kGemmBM - 1) / kGemmBM * kGemmBM);
@@ -1232,7 +1233,7 @@ extern "C" int asd_get_last_trace(asd_ctx* x, int32_t* n_stages, int32_t* n_ctas
     if (n_stages) *n_stages = x->last_n_stages;
     if (n_ctas) *n_ctas = x->dev->num_sms;
     if (ns_out) {
-        ASD_CUDA(x, cudaMemcpyAsync(ns_out, x->ws + x->lay.trace, (size_t)x->last_n_stages * 8 * x->dev->num_sms * 8, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaMemcpyAsync(ns_out, x->ws + x->lay.trace, (size_t)x->last_n_stages * kTraceEntries * x->dev->num_sms * 8, cudaMemcpyDeviceToHost, x->stream));
         ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     }
     return ASD_OK;

@@ -92,7 +92,7 @@ struct PassParams {
     int* accept_out;
     float* logits_out;
     int acc_sim;
-    long long* trace;  // optional [n_stages][8][gridDim.x] device timestamps (ns) and cycle counts, or null
+    long long* trace;  // optional [n_stages][kTraceEntries][gridDim.x] device timestamps (ns) and cycle counts, or null
     // shared-memory plan (bytes from the 1024-aligned base)
     int ns;            // ring slots
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
@@ -100,6 +100,7 @@ struct PassParams {
     int off_bars, off_misc, off_psum, off_reg_a;
 };
 
+constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)
 constexpr int kSegK = 512;     // inputs per ring item (16 column blocks of 32; the last item of a row may hold fewer)
 constexpr int kBoxKeys = 64;   // keys per K/V box (one ring slot)
 constexpr int kOctRows = 8;    // weight rows per ring item (four pairs): the N of one m16n8k16 tensor-core step
@@ -229,8 +230,25 @@ __device__ __forceinline__ int ring_acquire(const PassParams& p, const PassSmem&
     return slot;
 }
 
+__device__ __forceinline__ long long global_ns() {
+    long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// producer side of the timeline (lane 0 of the producer warp): when it issued its first and last copy of the stage
+// and how many cycles it waited for free slots in between
+__device__ __forceinline__ void producer_trace(const PassParams& p, int stage, long long t_first, long long stall_cycles) {
+    if (!p.trace || (threadIdx.x & 31) != 0) return;
+    long long* t = p.trace + (size_t)stage * kTraceEntries * gridDim.x + blockIdx.x;
+    t[(size_t)8 * gridDim.x] = t_first;
+    t[(size_t)9 * gridDim.x] = global_ns();
+    t[(size_t)10 * gridDim.x] = stall_cycles;
+}
+
 // ============================================================================================ producer
-// The whole producer warp feeds the ring: lane l takes ring items l, l+32, ... of each stage.
+// The whole producer warp feeds the ring: lane l takes ring items l, l+32, ... of each stage. (Asking L2 for the
+// items beyond the ring with cp.async.bulk.prefetch.L2 while the ring is full was measured twice and slows the pass
+// down, by 17 % at 32 items ahead and more at larger distances; the ring alone is the prefetch buffer.)
 template <int M>
 __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     const int lane = threadIdx.x & 31;
@@ -249,6 +267,8 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
             const uint32_t box_bytes = (uint32_t)kBoxKeys * box_cols * 2u;
             const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
             const int n_items = n_local * 2 * tile_slots;
+            const long long tp0 = (p.trace && lane == 0) ? global_ns() : 0;
+            long long stall = 0;
             for (int idx = lane; idx < n_items; idx += 32) {
                 const int j = idx / (2 * tile_slots), r = idx - j * 2 * tile_slots;
                 const int which = r / tile_slots, t = r - which * tile_slots;
@@ -256,13 +276,16 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 const int item = first + j;
                 const int kvh = item / n_chunks, chunk = item - kvh * n_chunks;
                 const uint32_t g = gi + (uint32_t)idx;
+                const long long ts0 = (p.trace && lane == 0) ? clock64() : 0;
                 const int slot = ring_acquire(p, sm, g, s, M);
+                if (p.trace && lane == 0) stall += clock64() - ts0;
                 mbar_expect_tx(&sm.full[slot], box_bytes);
                 tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, which ? st.tm_v : st.tm_k, kvh * p.head_dim + hb * 64,
                             chunk * kAttnChunk + rg * kBoxKeys, &sm.full[slot]);
                 issued[1] = issued[0], issued[0] = g, ++n_issued;
             }
             gi += (uint32_t)n_items;
+            producer_trace(p, s, tp0, stall);
             continue;
         }
         // GEMV stage: this CTA's slab is contiguous and already in ring order (segment-major, octets inside)
@@ -273,19 +296,24 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
         const int n_items = n_oct * n_seg;
         const int row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
         const unsigned char* slab = st.W + (size_t)pair0 * row_blocks * 128;
+        const long long tp0 = (p.trace && lane == 0) ? global_ns() : 0;
+        long long stall = 0;
         for (int idx = lane; idx < n_items; idx += 32) {
             const int seg = idx / n_oct, o = idx - seg * n_oct;
             const int nblk = min(16, row_blocks - seg * 16);  // column blocks of this segment
             const int rows = 2 * min(4, np - 4 * o);
             const uint32_t bytes = (uint32_t)(nblk * rows * 64);
             const uint32_t g = gi + (uint32_t)idx;
+            const long long ts0 = (p.trace && lane == 0) ? clock64() : 0;
             const int slot = ring_acquire(p, sm, g, s, M);
+            if (p.trace && lane == 0) stall += clock64() - ts0;
             mbar_expect_tx(&sm.full[slot], bytes);
             tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)seg * np * 2048 + (size_t)o * nblk * 512, bytes,
                              &sm.full[slot], pol_stream);
             issued[1] = issued[0], issued[0] = g, ++n_issued;
         }
         gi += (uint32_t)n_items;
+        producer_trace(p, s, tp0, stall);
     }
     // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let this lane's
     // last two copies land (bounded) before the CTA exits (the ring holds at most two items of a lane).
@@ -301,14 +329,9 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     }
 }
 
-__device__ __forceinline__ long long global_ns() {
-    long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
 // per-stage timeline of every CTA (debugging aid): 0 = stage entered, 1 = inputs ready, 2 = streaming done, 3 = stage left
 __device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k) {
-    if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * 8 + k) * gridDim.x + blockIdx.x] = global_ns();
+    if (p.trace && threadIdx.x == 0) p.trace[((size_t)stage * kTraceEntries + k) * gridDim.x + blockIdx.x] = global_ns();
 }
 
 // ============================================================================================ grid barrier
@@ -559,8 +582,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     consumers_sync();
     trace_mark(p, stage, 2);
     if (p.trace && tid == 0) {
-        p.trace[((size_t)stage * 8 + 4) * gridDim.x + blockIdx.x] = cyc_wait;
-        p.trace[((size_t)stage * 8 + 5) * gridDim.x + blockIdx.x] = cyc_work;
+        p.trace[((size_t)stage * kTraceEntries + 4) * gridDim.x + blockIdx.x] = cyc_wait;
+        p.trace[((size_t)stage * kTraceEntries + 5) * gridDim.x + blockIdx.x] = cyc_work;
     }
 
     // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
@@ -1089,7 +1112,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     if (p.trace && threadIdx.x == 0) {  // which SM runs this CTA (entry 4 of the embedding stage, which streams nothing)
         unsigned smid;
         asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        p.trace[((size_t)0 * 8 + 4) * gridDim.x + blockIdx.x] = smid;
+        p.trace[((size_t)0 * kTraceEntries + 4) * gridDim.x + blockIdx.x] = smid;
     }
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);

@@ -246,74 +246,125 @@ __device__ __forceinline__ void producer_trace(const PassParams& p, int stage, l
 }
 
 // ============================================================================================ producer
-// The whole producer warp feeds the ring: lane l takes ring items l, l+32, ... of each stage. (Asking L2 for the
-// items beyond the ring with cp.async.bulk.prefetch.L2 while the ring is full was measured twice and slows the pass
-// down, by 17 % at 32 items ahead and more at larger distances; the ring alone is the prefetch buffer.)
+// The whole producer warp feeds the ring: lane l takes ring items l, l+32, ... of each stage. The lanes poll in ONE
+// converged loop (each lane looks at the slot of its own next item, the lanes whose slot is free issue their copy
+// and move on), so the warp costs its scheduler a dozen instructions per round however many lanes are waiting, and
+// a freed slot is refilled within one round. (Asking L2 for the items beyond the ring with
+// cp.async.bulk.prefetch.L2 while the ring is full was measured twice and slows the pass down, by 17 % at 32 items
+// ahead and more at larger distances; the ring alone is the prefetch buffer.)
+struct ProdState {
+    int s, type, idx, n_items;
+    uint32_t gi;  // ring index of item 0 of the stage
+    // GEMV stage: this CTA's slab is contiguous and already in ring order (segment-major, octets inside)
+    const unsigned char* slab;
+    int np, n_oct, row_blocks;
+    // attention stage
+    const CUtensorMap *tm_k, *tm_v;
+    int n_chunks, first;
+};
+
+// move to the next stage that streams anything for this lane; false when the pass has no more
+template <int M>
+__device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& c, int lane) {
+    for (;;) {
+        c.gi += (uint32_t)c.n_items;
+        c.n_items = 0;
+        if (++c.s >= p.n_stages) return false;
+        const StageDesc st = p.stages[c.s];
+        c.type = st.type;
+        if (st.type == kStEmbed || st.type == kStFinish) continue;
+        if (st.type == kStAttn) {
+            const int n_local = attn_local_items(p, M, c.n_chunks, c.first);
+            const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
+            c.n_items = n_local * 2 * (kAttnChunk / kBoxKeys) * nhb;
+            c.tm_k = st.tm_k, c.tm_v = st.tm_v;
+        } else {
+            int pair0;
+            cta_pairs(st.n_rows, pair0, c.np);
+            c.n_oct = (c.np + 3) >> 2;
+            c.n_items = c.n_oct * ((st.n_in + kSegK - 1) / kSegK);
+            c.row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
+            c.slab = st.W + (size_t)pair0 * c.row_blocks * 128;
+        }
+        c.idx = lane;
+        if (c.idx < c.n_items) return true;
+    }
+}
+
 template <int M>
 __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     const int lane = threadIdx.x & 31;
     volatile int* err = p.err;
-    uint32_t gi = 0, issued[2] = {0, 0};
+    uint32_t issued[2] = {0, 0};
     int n_issued = 0;
     const uint64_t pol_stream = make_policy_evict_first();  // weights are read once per pass: do not let them age in L2
-    for (int s = 0; s < p.n_stages; ++s) {
-        const StageDesc st = p.stages[s];
-        if (st.type == kStEmbed || st.type == kStFinish) continue;
-        if (st.type == kStAttn) {
-            int n_chunks, first;
-            const int n_local = attn_local_items(p, M, n_chunks, first);
-            const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
-            const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
-            const uint32_t box_bytes = (uint32_t)kBoxKeys * box_cols * 2u;
-            const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
-            const int n_items = n_local * 2 * tile_slots;
-            const long long tp0 = (p.trace && lane == 0) ? global_ns() : 0;
-            long long stall = 0;
-            for (int idx = lane; idx < n_items; idx += 32) {
-                const int j = idx / (2 * tile_slots), r = idx - j * 2 * tile_slots;
-                const int which = r / tile_slots, t = r - which * tile_slots;
-                const int rg = t / nhb, hb = t - rg * nhb;
-                const int item = first + j;
-                const int kvh = item / n_chunks, chunk = item - kvh * n_chunks;
-                const uint32_t g = gi + (uint32_t)idx;
-                const long long ts0 = (p.trace && lane == 0) ? clock64() : 0;
-                const int slot = ring_acquire(p, sm, g, s, M);
-                if (p.trace && lane == 0) stall += clock64() - ts0;
-                mbar_expect_tx(&sm.full[slot], box_bytes);
-                tma_load_2d(sm.ring + (size_t)slot * kSlotBytes, which ? st.tm_v : st.tm_k, kvh * p.head_dim + hb * 64,
-                            chunk * kAttnChunk + rg * kBoxKeys, &sm.full[slot]);
+    ProdState c{};
+    c.s = -1;
+    bool active = prod_next_stage<M>(p, c, lane);
+    long long t_progress = clock64();
+    long long tp_first = (p.trace && lane == 0) ? global_ns() : 0, stall = 0, t_blocked = 0;
+    bool blocked = false;
+    for (unsigned round = 1; __any_sync(0xffffffffu, active); ++round) {
+        if (active) {
+            const uint32_t g = c.gi + (uint32_t)c.idx;
+            int slot;
+            uint32_t gen;
+            ring_locate(p, g, slot, gen);
+            // the slot may be overwritten once generation gen-1 of it has been consumed (counter first: the barrier's
+            // phase parity alone is ambiguous for a waiter that is more than one phase behind)
+            const bool free_now = gen == 0 || (sm.consumed[slot] >= gen && mbar_try_wait(&sm.empty[slot], (gen - 1) & 1));
+            if (free_now) {
+                if (p.trace && lane == 0 && blocked) stall += clock64() - t_blocked;
+                blocked = false;
+                unsigned char* dst = sm.ring + (size_t)slot * kSlotBytes;
+                if (c.type == kStAttn) {
+                    const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
+                    const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
+                    const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
+                    const int j = c.idx / (2 * tile_slots), r = c.idx - j * 2 * tile_slots;
+                    const int which = r / tile_slots, t = r - which * tile_slots;
+                    const int rg = t / nhb, hb = t - rg * nhb;
+                    const int item = c.first + j;
+                    const int kvh = item / c.n_chunks, chunk = item - kvh * c.n_chunks;
+                    mbar_expect_tx(&sm.full[slot], (uint32_t)kBoxKeys * box_cols * 2u);
+                    tma_load_2d(dst, which ? c.tm_v : c.tm_k, kvh * p.head_dim + hb * 64, chunk * kAttnChunk + rg * kBoxKeys,
+                                &sm.full[slot]);
+                } else {
+                    const int seg = c.idx / c.n_oct, o = c.idx - seg * c.n_oct;
+                    const int nblk = min(16, c.row_blocks - seg * 16);  // column blocks of this segment
+                    const int rows = 2 * min(4, c.np - 4 * o);
+                    const uint32_t bytes = (uint32_t)(nblk * rows * 64);
+                    mbar_expect_tx(&sm.full[slot], bytes);
+                    tma_load_1d_hint(dst, c.slab + (size_t)seg * c.np * 2048 + (size_t)o * nblk * 512, bytes, &sm.full[slot], pol_stream);
+                }
                 issued[1] = issued[0], issued[0] = g, ++n_issued;
+                t_progress = clock64();
+                c.idx += 32;
+                if (c.idx >= c.n_items) {
+                    if (p.trace && lane == 0) {
+                        producer_trace(p, c.s, tp_first, stall);
+                        stall = 0;
+                    }
+                    active = prod_next_stage<M>(p, c, lane);
+                    if (p.trace && lane == 0) tp_first = global_ns();
+                }
+            } else {
+                if (p.trace && lane == 0 && !blocked) t_blocked = clock64();
+                blocked = true;
+                if ((round & 255u) == 0) {  // the error word lives in global memory: look at it only now and then
+                    if (*err != kErrNone) {
+                        active = false;
+                    } else if (clock64() - t_progress > kWaitCycles) {
+                        if (atomicCAS(p.err, kErrNone, kErrEmptyWait) == kErrNone) {
+                            p.err[1] = c.s, p.err[2] = (int)g, p.err[3] = slot, p.err[4] = blockIdx.x, p.err[5] = threadIdx.x;
+                            p.err[6] = M, p.err[7] = (int)((gen - 1) & 1);
+                        }
+                        active = false;
+                    }
+                }
             }
-            gi += (uint32_t)n_items;
-            producer_trace(p, s, tp0, stall);
-            continue;
         }
-        // GEMV stage: this CTA's slab is contiguous and already in ring order (segment-major, octets inside)
-        int pair0, np;
-        cta_pairs(st.n_rows, pair0, np);
-        const int n_seg = (st.n_in + kSegK - 1) / kSegK;
-        const int n_oct = (np + 3) >> 2;
-        const int n_items = n_oct * n_seg;
-        const int row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
-        const unsigned char* slab = st.W + (size_t)pair0 * row_blocks * 128;
-        const long long tp0 = (p.trace && lane == 0) ? global_ns() : 0;
-        long long stall = 0;
-        for (int idx = lane; idx < n_items; idx += 32) {
-            const int seg = idx / n_oct, o = idx - seg * n_oct;
-            const int nblk = min(16, row_blocks - seg * 16);  // column blocks of this segment
-            const int rows = 2 * min(4, np - 4 * o);
-            const uint32_t bytes = (uint32_t)(nblk * rows * 64);
-            const uint32_t g = gi + (uint32_t)idx;
-            const long long ts0 = (p.trace && lane == 0) ? clock64() : 0;
-            const int slot = ring_acquire(p, sm, g, s, M);
-            if (p.trace && lane == 0) stall += clock64() - ts0;
-            mbar_expect_tx(&sm.full[slot], bytes);
-            tma_load_1d_hint(sm.ring + (size_t)slot * kSlotBytes, slab + (size_t)seg * np * 2048 + (size_t)o * nblk * 512, bytes,
-                             &sm.full[slot], pol_stream);
-            issued[1] = issued[0], issued[0] = g, ++n_issued;
-        }
-        gi += (uint32_t)n_items;
-        producer_trace(p, s, tp0, stall);
+        __syncwarp();
     }
     // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let this lane's
     // last two copies land (bounded) before the CTA exits (the ring holds at most two items of a lane).
@@ -376,6 +427,13 @@ __device__ __forceinline__ bool last_cta_consumers(unsigned* counter, int* flag_
     return last;
 }
 
+// Every stage starts by waiting for the previous stage of all CTAs. Whatever does not depend on activations (the
+// stage descriptor, index arithmetic, zeroing of partial sums, RMSNorm gains) is done before this wait.
+__device__ __forceinline__ void stage_begin(const PassParams& p, int s) {
+    if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);
+    trace_mark(p, s, 1);
+}
+
 // ============================================================================================ GEMV stage
 template <int M>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
@@ -395,11 +453,26 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
+    // Few octets (the d x d matrices leave ~28 rows to a CTA): several warps share an octet, warp set ks taking the
+    // segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are added
+    // in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
+    const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
+    const int copy_stride = np * 2 * M;
+    for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
+    constexpr bool kKeepX = (M <= 2);
+    const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
+    uint2 gpre[3] = {make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)};  // this thread's RMSNorm gains
+    if (keep) {
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            const int i = (tid + c * kPassConsumers) * 4;
+            if (i < n_in) gpre[c] = *reinterpret_cast<const uint2*>(st.gain + i);
+        }
+    }
+    stage_begin(p, stage);
 
     // ---- RMSNorm statistics (same arithmetic for every row count). With one or two rows the hidden state read
     //      here stays in registers for the window fill below (one L2 round trip less per stage).
-    constexpr bool kKeepX = (M <= 2);
-    const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
     float4 xr[kKeepX ? M : 1][3];
     float inv[M];
     if (norm) {
@@ -441,12 +514,6 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             inv[m] = 1.0f / sqrtf(s / (float)n_in + p.eps);
         }
     }
-    // Few octets (the d x d matrices leave ~28 rows to a CTA): several warps share an octet, warp set ks taking the
-    // segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are added
-    // in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
-    const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
-    const int copy_stride = np * 2 * M;
-    for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
     trace_mark(p, stage, 6);
 
     long long cyc_wait = 0, cyc_work = 0;  // when tracing: cycles this warp spent waiting for slots / working on them
@@ -463,8 +530,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 const int i = (tid + c * kPassConsumers) * 4;
                 if (i < wlen) {
                     const bool in = i < n_in;
-                    uint2 gv = make_uint2(0u, 0u);
-                    if (in) gv = *reinterpret_cast<const uint2*>(st.gain + i);
+                    const uint2 gv = gpre[c];
                     const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
 #pragma unroll
                     for (int m = 0; m < M; ++m) {
@@ -537,24 +603,36 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes + g8 * 64 + q4 * 16;
                 const int blk = rows * 64;
                 const int nblk = min(16, ((n_in + 31) >> 5) - seg * 16);
-                float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+                // Four independent accumulators (column block parity x half of the block), so that an item is four
+                // chains of 8 dependent tensor-core steps instead of two chains of 16: the latency of an item, and with
+                // it the time its ring slot stays occupied, is set by the chain length. They are added in a fixed order.
+                float acc[4][4];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {  // two halves of 8 column blocks: weights of a half in registers, then 16 steps
-                    uint4 wv[8];
+                for (int a = 0; a < 4; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        wv[j] = (g8 < rows && h * 8 + j < nblk) ? *reinterpret_cast<const uint4*>(sl + (h * 8 + j) * blk)
-                                                                 : make_uint4(0u, 0u, 0u, 0u);
-                    if (h * 8 < nblk) {
+                for (int h = 0; h < 4; ++h) {  // four quarters of 4 column blocks: operands of a quarter in registers, then 8 steps
+                    if (h * 4 < nblk) {
+                        uint4 wv[4], al[4], ah[4];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const uint4 al = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + (h * 8 + j) * 32);
-                            uint4 ah = make_uint4(0u, 0u, 0u, 0u);
-                            if (M > 8) ah = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + (h * 8 + j) * 32);
-                            mma_bf16_16816(c0, al.x, ah.x, al.y, ah.y, wv[j].x, wv[j].y);
-                            mma_bf16_16816(c1, al.z, ah.z, al.w, ah.w, wv[j].z, wv[j].w);
+                        for (int j = 0; j < 4; ++j) {
+                            wv[j] = (g8 < rows && h * 4 + j < nblk) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk)
+                                                                     : make_uint4(0u, 0u, 0u, 0u);
+                            al[j] = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + (h * 4 + j) * 32);
+                            ah[j] = make_uint4(0u, 0u, 0u, 0u);
+                            if (M > 8) ah[j] = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + (h * 4 + j) * 32);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            mma_bf16_16816(acc[(j & 1) * 2 + 0], al[j].x, ah[j].x, al[j].y, ah[j].y, wv[j].x, wv[j].y);
+                            mma_bf16_16816(acc[(j & 1) * 2 + 1], al[j].z, ah[j].z, al[j].w, ah[j].w, wv[j].z, wv[j].w);
                         }
                     }
+                }
+                float c0[4], c1[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    c0[e] = acc[0][e] + acc[2][e];
+                    c1[e] = acc[1][e] + acc[3][e];
                 }
                 __syncwarp();
                 if (lane == 0) ring_release(p, sm, g);
@@ -832,6 +910,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     const int n_local = attn_local_items(p, M, n_chunks, first);
     const uint32_t gi0 = gi;
     gi += (uint32_t)(n_local * 2 * tile_slots);
+    stage_begin(p, stage);  // all consumer warps, also those without attention work
     const int grp = warp >> 2;
     if (grp >= p.attn_groups) return;
 
@@ -1116,10 +1195,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     }
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);
-        if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);
-        trace_mark(p, s, 1);
-        const StageDesc st = p.stages[s];
+        const StageDesc st = p.stages[s];  // static: read before waiting for the previous stage
         if (st.type == kStEmbed) {
+            stage_begin(p, s);
             const int d = p.d_model;
             for (int i = blockIdx.x * kPassConsumers + threadIdx.x; i < M * d; i += gridDim.x * kPassConsumers) {
                 const int m = i / d, e = i - m * d;
@@ -1128,6 +1206,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
                 p.x[i] = __bfloat162float(p.embed[(size_t)t * d + e]);
             }
         } else if (st.type == kStFinish) {
+            stage_begin(p, s);
             finish_stage<M>(p, sm);
         } else if (st.type == kStAttn) {
             attn_stage<M>(p, st, sm, gi, s);

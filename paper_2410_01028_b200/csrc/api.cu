@@ -118,7 +118,7 @@ static bool plan_gemv(const DeviceInfo& dv, int M, int n_rows, int n_in, bool no
 // Shared-memory plan of the persistent pass kernel for M rows: ring slots, barriers, reduction scratch,
 // per-pair partial sums, activation window / attention scratch.
 struct PassPlan {
-    int ns, attn_groups, off_bars, off_misc, off_psum, off_reg_a;
+    int ns, attn_groups, off_bars, off_misc, off_psum, off_reg_a, xs_bytes;
     size_t smem;
 };
 
@@ -130,7 +130,11 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const size_t psum = ((size_t)std::max<long long>(np_max, 64) * 2 * M * 4 + 15) & ~(size_t)15;
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
-    const size_t xs = (size_t)M * ((size_t)pass_wseg(M) * kSegK + kXsPad) * 2;
+    // activation window: whole rows (the longest reduction dimension, in segments) when they fit the budget, so that
+    // short passes leave more shared memory to the ring
+    const size_t seg_max = ((size_t)std::max(c.d_model, c.d_ffn) + kSegK - 1) / kSegK;
+    const int xs_bytes = (int)std::min<size_t>(kXsBudget, (size_t)M * (seg_max * kSegK + kXsPad) * 2);
+    const size_t xs = (size_t)M * ((size_t)pass_wseg(M, xs_bytes) * kSegK + kXsPad) * 2;
     // up to three groups of four warps work on attention items, as many as their scratch fits the window's bytes
     const int groups_by_scratch = (int)std::max<size_t>(1, std::min<size_t>(3, (size_t)kXsBudget / attn_scratch));
     const size_t reg_a = (std::max(xs, groups_by_scratch * attn_scratch) + 15) & ~(size_t)15;
@@ -139,6 +143,7 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const int tile_slots = (kAttnChunk / kBoxKeys) * std::max(1, c.head_dim / 64);
     if (ns < 2 * tile_slots || ns < 8) return false;
     pl->ns = ns;
+    pl->xs_bytes = xs_bytes;
     pl->attn_groups = std::max(1, std::min(groups_by_scratch, ns / (2 * tile_slots)));
     pl->off_bars = ns * kSlotBytes;
     pl->off_misc = pl->off_bars + 2 * 64 * 8;
@@ -554,6 +559,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.ns = pl.ns, p.attn_groups = pl.attn_groups;
     p.ns_magic = (unsigned)((1ull << 32) / (unsigned)pl.ns + 1);
     p.off_bars = pl.off_bars, p.off_misc = pl.off_misc, p.off_psum = pl.off_psum, p.off_reg_a = pl.off_reg_a;
+    p.xs_bytes = pl.xs_bytes;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));
     x->bar_base += (uint32_t)p.n_stages * (uint32_t)grid;

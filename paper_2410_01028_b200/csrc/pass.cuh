@@ -46,7 +46,7 @@ namespace asd {
 constexpr int kPassConsumerWarps = 15;
 constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
-constexpr int kXsBudget = 40960;                    // bytes of shared memory for the activation window / attention scratch
+constexpr int kXsBudget = 40960;                    // most shared memory the activation window / attention scratch may take
 
 enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead, kStFinish };
 
@@ -98,6 +98,7 @@ struct PassParams {
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
     int attn_groups;   // 1 to 3 groups of 4 warps work on attention items
     int off_bars, off_misc, off_psum, off_reg_a;
+    int xs_bytes;      // bytes of the activation window: whole rows when they fit kXsBudget (the rest goes to the ring)
 };
 
 constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)
@@ -107,8 +108,8 @@ constexpr int kOctRows = 8;    // weight rows per ring item (four pairs): the N 
 constexpr int kXsPad = 32;     // bf16 elements of padding per activation row (64 bytes: conflict-free 16-byte reads)
 
 // 256-input segments whose activations (M rows, bf16, padded rows) fit the shared-memory window
-__host__ __device__ inline int pass_wseg(int M) {
-    const int w = (kXsBudget / M - kXsPad * 2) / (kSegK * 2);
+__host__ __device__ inline int pass_wseg(int M, int xs_bytes) {
+    const int w = (xs_bytes / M - kXsPad * 2) / (kSegK * 2);
     return w < 1 ? 1 : w;
 }
 
@@ -445,7 +446,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     cta_pairs(n_rows, pair0, np);
     const int n_seg = (n_in + kSegK - 1) / kSegK;
     const int n_oct = (np + 3) >> 2;
-    const int wseg = pass_wseg(M);
+    const int wseg = pass_wseg(M, p.xs_bytes);
     const int xstride = wseg * kSegK + kXsPad;  // bf16 elements per activation row in the window
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
     float* red = sm.red;

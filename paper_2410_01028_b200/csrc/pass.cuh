@@ -477,10 +477,12 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     float4 xr[kKeepX ? M : 1][3];
     float inv[M];
     if (norm) {
+        float ssq[M];  // this thread's share of every row's sum of squares; per row the additions run in index order
 #pragma unroll
-        for (int m = 0; m < M; ++m) {
-            float s = 0.f;
-            if (keep) {
+        for (int m = 0; m < M; ++m) ssq[m] = 0.f;
+        if (keep) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
 #pragma unroll
                 for (int c = 0; c < 3; ++c) {
                     const int i = (tid + c * kPassConsumers) * 4;
@@ -488,22 +490,40 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     if (i < n_in) v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
                     xr[kKeepX ? m : 0][c] = v;
                     if (i < n_in) {
+                        float s = ssq[m];
                         s = fmaf(v.x, v.x, s);
                         s = fmaf(v.y, v.y, s);
                         s = fmaf(v.z, v.z, s);
                         s = fmaf(v.w, v.w, s);
+                        ssq[m] = s;
                     }
                 }
-            } else {
-                for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
-                    s = fmaf(v.x, v.x, s);
-                    s = fmaf(v.y, v.y, s);
-                    s = fmaf(v.z, v.z, s);
-                    s = fmaf(v.w, v.w, s);
+            }
+        } else {
+            // the loads of up to four rows are in flight together (one memory round trip per four rows and stride)
+            for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
+#pragma unroll
+                for (int m0 = 0; m0 < M; m0 += 4) {
+                    float4 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (m0 + u < M) v[u] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (m0 + u < M) {
+                            float s = ssq[m0 + u];
+                            s = fmaf(v[u].x, v[u].x, s);
+                            s = fmaf(v[u].y, v[u].y, s);
+                            s = fmaf(v[u].z, v[u].z, s);
+                            s = fmaf(v[u].w, v[u].w, s);
+                            ssq[m0 + u] = s;
+                        }
                 }
             }
-            s = warp_sum(s);
+        }
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            const float s = warp_sum(ssq[m]);
             if (lane == 0) red[warp * (kPassMaxRows * 4) + m] = s;
         }
         consumers_sync();
@@ -556,16 +576,24 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 if (in) gv = *reinterpret_cast<const uint2*>(st.gain + k0 + i);
                 const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
 #pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    uint2 o = make_uint2(0u, 0u);
-                    if (in) {
-                        const float4 v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + k0 + i));
-                        __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv[m] * g0, v.y * inv[m] * g1);
-                        __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv[m] * g2, v.w * inv[m] * g3);
-                        o.x = *reinterpret_cast<uint32_t*>(&lo);
-                        o.y = *reinterpret_cast<uint32_t*>(&hi);
-                    }
-                    *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                for (int m0 = 0; m0 < M; m0 += 4) {
+                    float4 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (m0 + u < M && in) v[u] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + k0 + i));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (m0 + u < M) {
+                            const int m = m0 + u;
+                            uint2 o = make_uint2(0u, 0u);
+                            if (in) {
+                                __nv_bfloat162 lo = __floats2bfloat162_rn(v[u].x * inv[m] * g0, v[u].y * inv[m] * g1);
+                                __nv_bfloat162 hi = __floats2bfloat162_rn(v[u].z * inv[m] * g2, v[u].w * inv[m] * g3);
+                                o.x = *reinterpret_cast<uint32_t*>(&lo);
+                                o.y = *reinterpret_cast<uint32_t*>(&hi);
+                            }
+                            *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                        }
                 }
             }
         } else {
@@ -701,6 +729,17 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         int ra, rb;
         stage_pair_rows(type, p, pair0 + pl, ra, rb);
         const bool has_b = rb < n_rows;
+        // rotary factors of all rows first: the stores below may alias them as far as the compiler knows, and one
+        // memory round trip per row would add up
+        float rc[M], rs[M];
+        if (type == kStQkv && ra < p.d_model + p.kv_dim) {
+            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                rc[m] = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
+                rs[m] = p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
+            }
+        }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
             float va = psum[(pl * 2 + 0) * M + m], vb = psum[(pl * 2 + 1) * M + m];
@@ -713,12 +752,11 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 p.t[(size_t)m * (n_rows >> 1) + (pair0 + pl)] = __float2bfloat16_rn(t);
             } else if (type == kStQkv) {
                 const int pos = p.pos0 + m;
-                const int half = p.head_dim >> 1;
                 if (ra < p.d_model + p.kv_dim) {  // q or k: rotate the pair (j, j + head_dim/2) by pos * theta_j
-                    const int j = ra % p.head_dim;
-                    const float c = p.rope_cos[(size_t)pos * half + j], s = p.rope_sin[(size_t)pos * half + j];
-                    const float r0 = va * c - vb * s;
-                    const float r1 = vb * c + va * s;
+                    // explicit roundings: the same arithmetic whatever the row count the kernel was compiled for
+                    const float c = rc[m], s = rs[m];
+                    const float r0 = __fmaf_rn(va, c, -__fmul_rn(vb, s));
+                    const float r1 = __fmaf_rn(vb, c, __fmul_rn(va, s));
                     va = r0;
                     vb = r1;
                 }

@@ -1,11 +1,11 @@
-// One persistent kernel per decoder pass (decode, draft, verify, prefill chunk).
+// One persistent kernel per decoder pass (decode, draft, verify, row pass of a short prompt).
 //
 // Why: at batch 1 a pass is ~200 dependent sublayer stages of 5-30 us each. Launching them one by one leaves
 // HBM idle at every boundary (launch latency, RMSNorm prologue, drain). Weights, however, never depend on
 // activations. So here one CTA per SM stays resident for the whole pass (cooperative launch) and is split in
 // two roles:
 //   * a producer warp walks this CTA's share of EVERY stage's weights (and of the old part of the KV cache)
-//     in order and keeps a shared-memory ring of 4 KB slots full with TMA copies (cp.async.bulk, and
+//     in order and keeps a shared-memory ring of 8 KB slots full with TMA copies (cp.async.bulk, and
 //     cp.async.bulk.tensor with 128-byte swizzle for K/V boxes). It never waits for activations, so HBM keeps
 //     streaming across stage boundaries, grid barriers and prologues. Weights are stored in HBM in exactly
 //     the order the ring consumes them (see "packed weights" below), so a CTA's slab of a stage is one

@@ -199,36 +199,62 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------- GPU legs
-def gemv_roofline(torch, asd, shape, hbm_peak):
-    """Times the stand-alone sublayer kernel: the fused RMSNorm -> gate/up GEMV -> SwiGLU product at M = 1,
-    over a pool of distinct weight matrices larger than L2, with CUDA events on the launching stream."""
-    d, f = shape.d_model, shape.d_ffn
-    n_rows = 2 * f
+def gemv_roofline(torch, asd, d, n_rows, M, epi, hbm_peak):
+    """Times the stand-alone sublayer kernel (fused RMSNorm -> GEMV -> epilogue) on one shape, over a pool of distinct
+    weight matrices larger than L2, with CUDA events on the launching stream."""
     per_launch = n_rows * d * 2
-    pool = max(2, int(400e6 // per_launch) + 1)
+    pool = max(2, int(300e6 // per_launch) + 1)
     dev = torch.device("cuda")
     W = [torch.from_numpy(synth.make_matrix_bf16((n_rows, d), seed=7, stream=100 + i).view(np.int16)).to(dev)
-         .view(torch.bfloat16) for i in range(min(pool, 4))]
+         .view(torch.bfloat16) for i in range(min(pool, 2))]
     while len(W) < pool:
-        W.append(W[len(W) % 4].clone())
-    x = torch.from_numpy(synth.make_array_f32((1, d), seed=7, stream=99)).to(dev)
+        W.append(W[len(W) % 2].clone())
+    x = torch.from_numpy(synth.make_array_f32((M, d), seed=7, stream=99)).to(dev)
     gain = torch.from_numpy(synth.make_matrix_bf16((d,), seed=7, stream=98, mean=1.0).view(np.int16)).to(dev).view(torch.bfloat16)
-    out = torch.empty((1, f), dtype=torch.bfloat16, device=dev)
+    if epi == asd.EPI_SWIGLU:
+        out = torch.empty((M, n_rows // 2), dtype=torch.bfloat16, device=dev)
+    else:
+        out = torch.zeros((M, n_rows), dtype=torch.float32, device=dev)
+    cos = torch.zeros(16, dtype=torch.float32, device=dev)
     scratch = torch.zeros(asd.fused_gemv_scratch_bytes(), dtype=torch.uint8, device=dev)
-    n = 200
-    for i in range(20):
-        asd.fused_gemv(x, W[i % pool], asd.EPI_SWIGLU, out, gain=gain, scratch=scratch)
+    # the launches are captured in a CUDA graph (one pass over the pool per replay) so that the host's launch cost
+    # does not bound the small shapes
+    for i in range(pool):
+        asd.fused_gemv(x, W[i % pool], epi, out, gain=gain, cos=cos, scratch=scratch)
+    torch.cuda.synchronize()
+    n_graph = max(pool, 20)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(n_graph):
+            asd.fused_gemv(x, W[i % pool], epi, out, gain=gain, cos=cos, scratch=scratch)
+    graph.replay()
+    reps = 10
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     e0.record()
-    for i in range(n):
-        asd.fused_gemv(x, W[i % pool], asd.EPI_SWIGLU, out, gain=gain, scratch=scratch)
+    for _ in range(reps):
+        graph.replay()
     e1.record()
     torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / n
+    us = e0.elapsed_time(e1) * 1e3 / (reps * n_graph)
     achieved = per_launch / (us * 1e-6) / 1e9
-    return {"kernel": "gemv_kernel<M=1, swiglu, rmsnorm> %dx%d" % (n_rows, d), "bytes_per_launch": per_launch,
-            "us_per_launch": us, "achieved": achieved, "pool_matrices": pool}
+    names = {asd.EPI_PLAIN: "plain", asd.EPI_SWIGLU: "swiglu", asd.EPI_RESIDUAL: "residual+cosine"}
+    return {"in": d, "out": n_rows, "rows": M, "epilogue": names[epi], "bytes_per_launch": per_launch, "us_per_launch": round(us, 2),
+            "GBps": round(achieved, 1), "frac": round(achieved / hbm_peak, 3)}
+
+
+def gemv_sweep(torch, asd, hbm_peak):
+    """The stand-alone fused kernel over the sublayer shapes of d_model 2048..8192 (out = d with the residual + cosine
+    epilogue, 3d plain, 2.6875d rows alternating gate / up with SwiGLU, and the W_d shape in = 2.6875d -> out = d), at
+    1 and 5 rows, RMSNorm prologue on."""
+    res = []
+    for d in (2048, 4096, 5120, 8192):
+        f2 = int(2.6875 * d)
+        for M in (1, 5):
+            for n_in, n_rows, epi in ((d, d, asd.EPI_RESIDUAL), (d, 3 * d, asd.EPI_PLAIN), (d, f2, asd.EPI_SWIGLU),
+                                      (f2, d, asd.EPI_RESIDUAL)):
+                res.append(gemv_roofline(torch, asd, n_in, n_rows, M, epi, hbm_peak))
+    return res
 
 
 def gemm_roofline(torch, asd, shape):
@@ -362,7 +388,7 @@ def run_ours(args):
                 "launches": int(n_launch), "bytes_per_launch": bytes_per_launch, "us_per_launch": us_per_launch,
                 "how": "CUDA events around every launch inside the timed region, on the launching stream"}
     if args.gemv_microbench:
-        roofline["fused_gemv_alone"] = gemv_roofline(torch, asd, shape, hbm_peak)
+        roofline["fused_gemv_alone"] = gemv_sweep(torch, asd, hbm_peak)
     # the prompt pass is the tensor-core part of a step: dense products + causal attention, then one decode pass
     _, tf_sustained, tf_kind = tensor_peak()
     pf_ms = agg["ms_prefill"] / args.steps

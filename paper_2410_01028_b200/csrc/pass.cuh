@@ -391,16 +391,16 @@ __device__ __forceinline__ void consumers_sync() { bar_sync(1, kPassConsumers); 
 
 __device__ __forceinline__ void grid_arrive(const PassParams& p) {
     consumers_sync();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(p.grid_bar, 1u);
-    }
+    // one release at GPU scope: cumulative over the writes of the whole CTA, which the barrier above ordered before it
+    if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p.grid_bar), "r"(1u) : "memory");
 }
 __device__ __forceinline__ void grid_wait(const PassParams& p, unsigned target) {
     if (threadIdx.x == 0) {
         volatile int* err = p.err;
         const long long t0 = clock64();
-        while ((int)(ld_acquire_gpu(p.grid_bar) - target) < 0) {
+        // every poll is a round trip to L2; the error word and the clock are looked at only now and then
+        for (unsigned spin = 1; (int)(ld_acquire_gpu(p.grid_bar) - target) < 0; ++spin) {
+            if ((spin & 63u) != 0) continue;
             if (*err != kErrNone) break;
             if (clock64() - t0 > kWaitCycles) {
                 if (atomicCAS(p.err, kErrNone, kErrGridWait) == kErrNone) {
@@ -1235,6 +1235,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);
         const StageDesc st = p.stages[s];  // static: read before waiting for the previous stage
+        // the next descriptor is requested now so that reading it at the next stage boundary hits L1
+        if (threadIdx.x < 2 && s + 1 < p.n_stages)
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(p.stages + s + 1) + threadIdx.x * 64));
         if (st.type == kStEmbed) {
             stage_begin(p, s);
             const int d = p.d_model;

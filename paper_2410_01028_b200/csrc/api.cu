@@ -126,8 +126,9 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const int kvd = c.n_kv_heads * c.head_dim;
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
     const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
-    // per-pair partial sums; when a CTA has fewer than 8 octets up to 15 warps keep copies (at most 60 pairs in all)
-    const size_t psum = ((size_t)std::max<long long>(np_max, 64) * 2 * M * 4 + 15) & ~(size_t)15;
+    // per-pair partial sums; when a CTA has fewer than 8 groups of 8 pairs up to 15 warps keep copies (at most 15 / groups
+    // copies of at most 8 * groups pairs: 120 pairs in all)
+    const size_t psum = ((size_t)std::max<long long>(np_max, 120) * 2 * M * 4 + 15) & ~(size_t)15;
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     // activation window: whole rows (the longest reduction dimension, in segments) when they fit the budget, so that
@@ -691,9 +692,9 @@ extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : 
 
 // Repack one matrix into the pass kernel's layout and copy it to the device. The logical matrix has n_rows
 // rows of n_in inputs; row(r) returns the host pointer of logical row r. CTA b of a G-CTA grid owns pairs
-// [b*P/G, (b+1)*P/G) in octets of four pairs (the last may be smaller); its slab is segment-major (for each
-// segment of 512 inputs: for each octet), and an item of R rows is a run of column blocks of 32 inputs, each
-// block R rows x 64 bytes (16 blocks, fewer in the last segment). Inputs past n_in are zero.
+// [b*P/G, (b+1)*P/G) in groups of eight pairs (the last may be smaller); its slab is segment-major (for each
+// segment of 256 inputs: for each group), and an item of R rows is a run of column blocks of 32 inputs, each
+// block R rows x 64 bytes (8 blocks, fewer in the last segment). Inputs past n_in are zero.
 template <class RowFn, class PairFn>
 static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, PairFn pair_rows_of,
                          std::vector<unsigned char>& staging) {
@@ -706,13 +707,13 @@ static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size
         const size_t pair0 = (size_t)b * n_pairs / G, pair1 = (size_t)(b + 1) * n_pairs / G, np = pair1 - pair0;
         unsigned char* slab = staging.data() + pair0 * row_blocks * 128;
         for (size_t sg = 0; sg < n_seg; ++sg) {
-            const size_t nblk = std::min<size_t>(16, row_blocks - sg * 16);
-            for (size_t o = 0; o * 4 < np; ++o) {
-                const size_t pairs = std::min<size_t>(4, np - 4 * o), R = 2 * pairs;
-                unsigned char* item = slab + sg * np * 2048 + o * nblk * 512;
+            const size_t nblk = std::min<size_t>(kSegBlocks, row_blocks - sg * kSegBlocks);
+            for (size_t o = 0; o * kGrpPairs < np; ++o) {
+                const size_t pairs = std::min<size_t>(kGrpPairs, np - kGrpPairs * o), R = 2 * pairs;
+                unsigned char* item = slab + sg * np * (kSegK * 4) + o * nblk * (kGrpRows * 64);
                 for (size_t pq = 0; pq < pairs; ++pq) {
                     size_t rr[2];
-                    pair_rows_of(pair0 + 4 * o + pq, rr[0], rr[1]);
+                    pair_rows_of(pair0 + kGrpPairs * o + pq, rr[0], rr[1]);
                     for (int h = 0; h < 2; ++h) {
                         if (rr[h] >= n_rows) continue;
                         const uint16_t* src = row(rr[h]);

@@ -18,16 +18,16 @@
 // weights are streamed and no K/V is touched for them.
 //
 // Packed weights: a matrix [n_rows, n_in] is cut into PAIRS of rows (the two rotary partners of a q/k head,
-// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 512 inputs. CTA b owns pairs [b*P/G, (b+1)*P/G)
-// and groups them into OCTETS of four pairs (the last octet may hold fewer). One ring item = one octet x one
-// segment of 512 inputs = up to 8 rows x 1 KB = one 8 KB slot, stored as up to 16 column blocks of 32 inputs
+// gate_i and up_i, or two neighbouring rows) and SEGMENTS of 256 inputs. CTA b owns pairs [b*P/G, (b+1)*P/G)
+// and groups them into GROUPS of eight pairs (the last group may hold fewer). One ring item = one group x one
+// segment of 256 inputs = up to 16 rows x 512 bytes = one 8 KB slot, stored as up to 8 column blocks of 32 inputs
 // (rows x 64 bytes each; the last segment of a row simply has fewer blocks). The CTA's slab is
-// segment-major (for seg: for octet), so consecutive ring items belong to different consumer warps and are
+// segment-major (for seg: for group), so consecutive ring items belong to different consumer warps and are
 // consumed as soon as they land, and no padding crosses HBM for input sizes that are multiples of 32.
 //
-// The products run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate): the activation rows are the
-// 16-row A operand, the 8 weight rows of an item the B operand, so one step serves any row count up to 16 and
-// the arithmetic of a row does not depend on how many rows share the pass. tcgen05 is not used here on
+// The products run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate): the 16 weight rows of an item
+// are the A operand, the activation rows the 8 columns of the B operand (two B tiles for more than 8 rows), so one
+// step serves any row count up to 8 and the arithmetic of a row does not depend on how many rows share the pass. tcgen05 is not used here on
 // purpose: its smallest tile (64 weight rows) does not fit a 148-way row split that leaves ~28 rows of the
 // d x d matrices to a CTA, and its A operand would need the activations padded to 64+ rows in shared memory.
 //
@@ -102,9 +102,11 @@ struct PassParams {
 };
 
 constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)
-constexpr int kSegK = 512;     // inputs per ring item (16 column blocks of 32; the last item of a row may hold fewer)
+constexpr int kSegK = 256;     // inputs per ring item (8 column blocks of 32; the last item of a row may hold fewer)
 constexpr int kBoxKeys = 64;   // keys per K/V box (one ring slot)
-constexpr int kOctRows = 8;    // weight rows per ring item (four pairs): the N of one m16n8k16 tensor-core step
+constexpr int kGrpPairs = 8;   // pairs of weight rows per ring item: 16 rows, the M of one m16n8k16 tensor-core step
+constexpr int kGrpRows = 2 * kGrpPairs;
+constexpr int kSegBlocks = kSegK / 32;  // column blocks of 32 inputs per full segment
 constexpr int kXsPad = 32;     // bf16 elements of padding per activation row (64 bytes: conflict-free 16-byte reads)
 
 // 256-input segments whose activations (M rows, bf16, padded rows) fit the shared-memory window
@@ -282,7 +284,7 @@ __device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& 
         } else {
             int pair0;
             cta_pairs(st.n_rows, pair0, c.np);
-            c.n_oct = (c.np + 3) >> 2;
+            c.n_oct = (c.np + kGrpPairs - 1) / kGrpPairs;
             c.n_items = c.n_oct * ((st.n_in + kSegK - 1) / kSegK);
             c.row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
             c.slab = st.W + (size_t)pair0 * c.row_blocks * 128;
@@ -332,11 +334,12 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                                 &sm.full[slot]);
                 } else {
                     const int seg = c.idx / c.n_oct, o = c.idx - seg * c.n_oct;
-                    const int nblk = min(16, c.row_blocks - seg * 16);  // column blocks of this segment
-                    const int rows = 2 * min(4, c.np - 4 * o);
+                    const int nblk = min(kSegBlocks, c.row_blocks - seg * kSegBlocks);  // column blocks of this segment
+                    const int rows = 2 * min(kGrpPairs, c.np - kGrpPairs * o);
                     const uint32_t bytes = (uint32_t)(nblk * rows * 64);
                     mbar_expect_tx(&sm.full[slot], bytes);
-                    tma_load_1d_hint(dst, c.slab + (size_t)seg * c.np * 2048 + (size_t)o * nblk * 512, bytes, &sm.full[slot], pol_stream);
+                    tma_load_1d_hint(dst, c.slab + (size_t)seg * c.np * (kSegK * 4) + (size_t)o * nblk * (kGrpRows * 64), bytes, &sm.full[slot],
+                                     pol_stream);
                 }
                 issued[1] = issued[0], issued[0] = g, ++n_issued;
                 t_progress = clock64();
@@ -445,7 +448,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     int pair0, np;
     cta_pairs(n_rows, pair0, np);
     const int n_seg = (n_in + kSegK - 1) / kSegK;
-    const int n_oct = (np + 3) >> 2;
+    const int n_oct = (np + kGrpPairs - 1) / kGrpPairs;  // groups of 16 rows (8 pairs; the last group may hold fewer)
     const int wseg = pass_wseg(M, p.xs_bytes);
     const int xstride = wseg * kSegK + kXsPad;  // bf16 elements per activation row in the window
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
@@ -454,9 +457,9 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
-    // Few octets (the d x d matrices leave ~28 rows to a CTA): several warps share an octet, warp set ks taking the
-    // segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are added
-    // in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
+    // Fewer groups than warps (the d x d matrices leave ~28 rows to a CTA): several warps share a group, warp set ks
+    // taking the segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are
+    // added in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
     const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
     const int copy_stride = np * 2 * M;
     for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
@@ -610,72 +613,79 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         consumers_sync();
 
         if (w0 == 0) trace_mark(p, stage, 7);
-        // Ring order is segment-major: consecutive items are different octets, i.e. different warps. One item is
-        // up to 8 weight rows x 512 inputs, stored as column blocks of 32 inputs ([block][row][64 bytes]); lane
-        // (g8, q4) owns inputs 32*block + 8*q4 .. +7 of row g8. Two m16n8k16 steps per block: the activations are
-        // the 16-row A operand (rows >= M repeat row M-1 and are ignored), the weights the 8-column B operand.
-        const __nv_bfloat16* xlo = xs + (size_t)min(g8, M - 1) * xstride + q4 * 8;
-        const __nv_bfloat16* xhi = xs + (size_t)min(g8 + 8, M - 1) * xstride + q4 * 8;
+        // Ring order is segment-major: consecutive items are different groups, i.e. different warps. One item is up to
+        // 16 weight rows x 256 inputs, stored as column blocks of 32 inputs ([block][row][64 bytes]); lane (g8, q4)
+        // owns inputs 32*block + 8*q4 .. +7 of rows g8 and g8 + 8. Two m16n8k16 steps per block: the weights are the
+        // 16-row A operand, the activation rows the 8 columns of the B operand (columns >= M are zero), so every
+        // step covers 16 weight rows and nothing of the tile is wasted on padding rows.
+        const __nv_bfloat16* xa = xs + (size_t)min(g8, M - 1) * xstride + q4 * 8;
+        const __nv_bfloat16* xb2 = xs + (size_t)min(g8 + 8, M - 1) * xstride + q4 * 8;
         const int ks = (S > 1) ? warp / n_oct : 0;                 // which copy of the partial sums this warp adds into
         const int o_first = (S > 1) ? ((ks < S) ? warp - ks * n_oct : n_oct) : warp;
-        const int o_step = (S > 1) ? n_oct : kPassConsumerWarps;  // S > 1: exactly one octet per warp
+        const int o_step = (S > 1) ? n_oct : kPassConsumerWarps;  // S > 1: exactly one group per warp
         float* psum_w = psum + (size_t)ks * copy_stride;
         for (int sg = 0; sg < ws; ++sg) {
             const int seg = w0 + sg;
             if (S > 1 && seg % S != ks) continue;
             for (int o = o_first; o < n_oct; o += o_step) {
                 const uint32_t g = gi + (uint32_t)(seg * n_oct + o);
-                const int rows = 2 * min(4, np - 4 * o);
+                const int rows = 2 * min(kGrpPairs, np - kGrpPairs * o);
                 const long long tw0 = p.trace ? clock64() : 0;
                 const int slot = ring_wait_full(p, sm, g, stage, M * 1000 + seg);
                 const long long tw1 = p.trace ? clock64() : 0;
                 const unsigned char* sl = sm.ring + (size_t)slot * kSlotBytes + g8 * 64 + q4 * 16;
                 const int blk = rows * 64;
-                const int nblk = min(16, ((n_in + 31) >> 5) - seg * 16);
-                // Four independent accumulators (column block parity x half of the block), so that an item is four
-                // chains of 8 dependent tensor-core steps instead of two chains of 16: the latency of an item, and with
-                // it the time its ring slot stays occupied, is set by the chain length. They are added in a fixed order.
-                float acc[4][4];
+                const int nblk = min(kSegBlocks, ((n_in + 31) >> 5) - seg * kSegBlocks);
+                // Four independent accumulators (column block parity x half of the block), added in a fixed order;
+                // acc2 holds activation rows 8..15 (row passes of a prompt with more than 8 rows).
+                float acc[4][4], acc2[M > 8 ? 4 : 1][4];
 #pragma unroll
                 for (int a = 0; a < 4; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
 #pragma unroll
-                for (int h = 0; h < 4; ++h) {  // four quarters of 4 column blocks: operands of a quarter in registers, then 8 steps
+                for (int a = 0; a < (M > 8 ? 4 : 1); ++a) acc2[a][0] = acc2[a][1] = acc2[a][2] = acc2[a][3] = 0.f;
+#pragma unroll
+                for (int h = 0; h < kSegBlocks / 4; ++h) {  // halves of 4 column blocks: operands in registers, then 8 steps
                     if (h * 4 < nblk) {
-                        uint4 wv[4], al[4], ah[4];
+                        uint4 wlo[4], whi[4], xv[4], xv2[M > 8 ? 4 : 1];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            wv[j] = (g8 < rows && h * 4 + j < nblk) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk)
-                                                                     : make_uint4(0u, 0u, 0u, 0u);
-                            al[j] = *reinterpret_cast<const uint4*>(xlo + sg * kSegK + (h * 4 + j) * 32);
-                            ah[j] = make_uint4(0u, 0u, 0u, 0u);
-                            if (M > 8) ah[j] = *reinterpret_cast<const uint4*>(xhi + sg * kSegK + (h * 4 + j) * 32);
+                            const bool inb = h * 4 + j < nblk;
+                            wlo[j] = (inb && g8 < rows) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk) : make_uint4(0u, 0u, 0u, 0u);
+                            whi[j] = (inb && g8 + 8 < rows) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk + 8 * 64)
+                                                           : make_uint4(0u, 0u, 0u, 0u);
+                            xv[j] = (g8 < M) ? *reinterpret_cast<const uint4*>(xa + sg * kSegK + (h * 4 + j) * 32) : make_uint4(0u, 0u, 0u, 0u);
+                            if (M > 8)
+                                xv2[j] = (g8 + 8 < M) ? *reinterpret_cast<const uint4*>(xb2 + sg * kSegK + (h * 4 + j) * 32)
+                                                      : make_uint4(0u, 0u, 0u, 0u);
                         }
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            mma_bf16_16816(acc[(j & 1) * 2 + 0], al[j].x, ah[j].x, al[j].y, ah[j].y, wv[j].x, wv[j].y);
-                            mma_bf16_16816(acc[(j & 1) * 2 + 1], al[j].z, ah[j].z, al[j].w, ah[j].w, wv[j].z, wv[j].w);
+                            mma_bf16_16816(acc[(j & 1) * 2 + 0], wlo[j].x, whi[j].x, wlo[j].y, whi[j].y, xv[j].x, xv[j].y);
+                            mma_bf16_16816(acc[(j & 1) * 2 + 1], wlo[j].z, whi[j].z, wlo[j].w, whi[j].w, xv[j].z, xv[j].w);
+                            if (M > 8) {
+                                mma_bf16_16816(acc2[(j & 1) * 2 + 0], wlo[j].x, whi[j].x, wlo[j].y, whi[j].y, xv2[j].x, xv2[j].y);
+                                mma_bf16_16816(acc2[(j & 1) * 2 + 1], wlo[j].z, whi[j].z, wlo[j].w, whi[j].w, xv2[j].z, xv2[j].w);
+                            }
                         }
                     }
-                }
-                float c0[4], c1[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    c0[e] = acc[0][e] + acc[2][e];
-                    c1[e] = acc[1][e] + acc[3][e];
                 }
                 __syncwarp();
                 if (lane == 0) ring_release(p, sm, g);
-                // c[0], c[1]: activation row g8, weight rows 2*q4, 2*q4+1 of the octet (= pair 4*o + q4); c[2], c[3]: row g8 + 8.
-                // Segments of a pair are added in ascending order, always by this lane.
-                const int pl = 4 * o + q4;
-                if (pl < np) {
-                    if (g8 < M) {
-                        psum_w[(pl * 2 + 0) * M + g8] += c0[0] + c1[0];
-                        psum_w[(pl * 2 + 1) * M + g8] += c0[1] + c1[1];
-                    }
-                    if (M > 8 && g8 + 8 < M) {
-                        psum_w[(pl * 2 + 0) * M + g8 + 8] += c0[2] + c1[2];
-                        psum_w[(pl * 2 + 1) * M + g8 + 8] += c0[3] + c1[3];
+                // c[0], c[1]: weight row g8 of the group, activation rows 2*q4 and 2*q4 + 1; c[2], c[3]: weight row g8 + 8.
+                // Local weight row 16*o + r is row (r & 1) of local pair 8*o + r/2. Segments are added in ascending
+                // order, always by this lane.
+#pragma unroll
+                for (int hr = 0; hr < 2; ++hr) {
+                    const int wr = g8 + 8 * hr;
+                    if (wr < rows) {
+                        float* dst = psum_w + (size_t)(kGrpRows * o + wr) * M;
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int mm = 2 * q4 + e;
+                            if (mm < M) dst[mm] += (acc[0][2 * hr + e] + acc[2][2 * hr + e]) + (acc[1][2 * hr + e] + acc[3][2 * hr + e]);
+                            if (M > 8 && mm + 8 < M)
+                                dst[mm + 8] += (acc2[0][2 * hr + e] + acc2[2][2 * hr + e]) + (acc2[1][2 * hr + e] + acc2[3][2 * hr + e]);
+                        }
                     }
                 }
                 if (p.trace) {

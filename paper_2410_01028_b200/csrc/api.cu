@@ -134,7 +134,10 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     // activation window: whole rows (the longest reduction dimension, in segments) when they fit the budget, so that
     // short passes leave more shared memory to the ring
     const size_t seg_max = ((size_t)std::max(c.d_model, c.d_ffn) + kSegK - 1) / kSegK;
-    const int xs_bytes = (int)std::min<size_t>(kXsBudget, (size_t)M * (seg_max * kSegK + kXsPad) * 2);
+    // otherwise at least whole rows of d_model inputs when that stays modest (every stage but W_d then needs one window)
+    const size_t seg_d = ((size_t)c.d_model + kSegK - 1) / kSegK;
+    const size_t full_f = (size_t)M * (seg_max * kSegK + kXsPad) * 2, full_d = (size_t)M * (seg_d * kSegK + kXsPad) * 2;
+    const int xs_bytes = (int)(full_f <= (size_t)kXsBudget ? full_f : (full_d <= 57344 ? std::max<size_t>(full_d, kXsBudget) : (size_t)kXsBudget));
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M, xs_bytes) * kSegK + kXsPad) * 2;
     // up to three groups of four warps work on attention items, as many as their scratch fits the window's bytes
     const int groups_by_scratch = (int)std::max<size_t>(1, std::min<size_t>(3, (size_t)kXsBudget / attn_scratch));

@@ -72,6 +72,24 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def measured_traffic_ratio():
+    """DRAM bytes per algorithmic byte of the one-row pass kernel, from the ncu capture summarised under profiles/
+    (taken on a 4-layer case; the kernel's traffic is its weight stream, which grows in proportion to the layers).
+    None when the kernel sources have changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "pass_kernel_m1_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    rec = dict(line.strip().split("=", 1) for line in open(path) if "=" in line and not line.startswith("#"))
+    h = hashlib.sha256()
+    for name in ("pass.cuh", "ring.cuh", "common.cuh"):
+        with open(os.path.join(ROOT, "paper_2410_01028_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    if rec.get("sources_sha256") != h.hexdigest():
+        return None
+    return float(rec["dram_bytes"]) / float(rec["algorithmic_bytes"])
+
+
 def tensor_peak():
     """Dense bf16 TFLOP/s of a cuBLAS GEMM on this machine: (burst, sustained, kind)."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -382,8 +400,12 @@ def run_ours(args):
     us_per_launch = dom_st["ms_" + dom] / n_launch * 1e3
     bytes_per_launch = dom_st["bytes_" + dom] / n_launch
     achieved = bytes_per_launch / (us_per_launch * 1e-6) / 1e9
+    ratio = measured_traffic_ratio()
     roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                "traffic": None, "peak_kind": peak_kind,
+                "traffic": None if ratio is None else ratio * bytes_per_launch,
+                "traffic_how": None if ratio is None else "ncu dram__bytes_read.sum + dram__bytes_write.sum of a 4-layer pass, scaled by "
+                               "algorithmic bytes (%.4f DRAM bytes per algorithmic byte)" % ratio,
+                "peak_kind": peak_kind,
                 "kernel": "pass_kernel<1> (%s pass: one persistent launch per pass)" % dom,
                 "launches": int(n_launch), "bytes_per_launch": bytes_per_launch, "us_per_launch": us_per_launch,
                 "how": "CUDA events around every launch inside the timed region, on the launching stream"}

@@ -1036,37 +1036,44 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             bar_sync(bar_id, 128);
 
             if (j == 0 && g == 0) trace_mark(p, stage, 2);  // attention timeline: 2 = inputs staged, 4 = softmax done, 5 = P V done, 6 = ticket taken, 7 = merged
-            // ---- scores: thread t owns key key0 + t
+            // ---- scores: thread t owns key key0 + t. Four independent partial sums per row (16-byte chunk parity x half
+            //      of the chunk) keep the chains of dependent FMAs short; they are added in a fixed order.
             float sc[M];
-#pragma unroll
-            for (int m = 0; m < M; ++m) sc[m] = 0.f;
             {
+                float s4[M][4];
+#pragma unroll
+                for (int m = 0; m < M; ++m) s4[m][0] = s4[m][1] = s4[m][2] = s4[m][3] = 0.f;
                 const int rg = gt / kBoxKeys, rr = gt % kBoxKeys;
-                const int chunks_per_box = box_cols / 8;
+                const int chunks_per_box = box_cols / 8;  // even: head_dim >= 16
                 for (int hb = 0; hb < nhb; ++hb) {
                     const unsigned char* krow = slot_ptr(gk + rg * nhb + hb) + rr * ta.row_bytes;
-                    for (int cc = 0; cc < chunks_per_box; ++cc) {
-                        const int c = hb * 8 + cc;
-                        const uint4 kv = *reinterpret_cast<const uint4*>(krow + ((ta.swz ? (cc ^ (rr & 7)) : cc) << 4));
-                        const float kf[8] = {bf_lo(kv.x), bf_hi(kv.x), bf_lo(kv.y), bf_hi(kv.y),
-                                             bf_lo(kv.z), bf_hi(kv.z), bf_lo(kv.w), bf_hi(kv.w)};
+                    for (int cc0 = 0; cc0 < chunks_per_box; cc0 += 2) {
 #pragma unroll
-                        for (int m = 0; m < M; ++m) {
-                            const float4 q0 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8);
-                            const float4 q1 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8 + 4);
-                            float a = sc[m];
-                            a = fmaf(q0.x, kf[0], a);
-                            a = fmaf(q0.y, kf[1], a);
-                            a = fmaf(q0.z, kf[2], a);
-                            a = fmaf(q0.w, kf[3], a);
-                            a = fmaf(q1.x, kf[4], a);
-                            a = fmaf(q1.y, kf[5], a);
-                            a = fmaf(q1.z, kf[6], a);
-                            a = fmaf(q1.w, kf[7], a);
-                            sc[m] = a;
+                        for (int par = 0; par < 2; ++par) {
+                            const int cc = cc0 + par, c = hb * 8 + cc;
+                            const uint4 kv = *reinterpret_cast<const uint4*>(krow + ((ta.swz ? (cc ^ (rr & 7)) : cc) << 4));
+                            const float kf[8] = {bf_lo(kv.x), bf_hi(kv.x), bf_lo(kv.y), bf_hi(kv.y),
+                                                 bf_lo(kv.z), bf_hi(kv.z), bf_lo(kv.w), bf_hi(kv.w)};
+#pragma unroll
+                            for (int m = 0; m < M; ++m) {
+                                const float4 q0 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8);
+                                const float4 q1 = *reinterpret_cast<const float4*>(qs + m * hd + c * 8 + 4);
+                                float a0 = s4[m][2 * par], a1 = s4[m][2 * par + 1];
+                                a0 = fmaf(q0.x, kf[0], a0);
+                                a1 = fmaf(q1.x, kf[4], a1);
+                                a0 = fmaf(q0.y, kf[1], a0);
+                                a1 = fmaf(q1.y, kf[5], a1);
+                                a0 = fmaf(q0.z, kf[2], a0);
+                                a1 = fmaf(q1.z, kf[6], a1);
+                                a0 = fmaf(q0.w, kf[3], a0);
+                                a1 = fmaf(q1.w, kf[7], a1);
+                                s4[m][2 * par] = a0, s4[m][2 * par + 1] = a1;
+                            }
                         }
                     }
                 }
+#pragma unroll
+                for (int m = 0; m < M; ++m) sc[m] = (s4[m][0] + s4[m][1]) + (s4[m][2] + s4[m][3]);
             }
             // ---- chunk-local softmax statistics; the row at position pos0+m sees keys <= pos0+m
             const int key = key0 + gt;
@@ -1121,28 +1128,58 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                     p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * 2 + 0] = cmax[m];
             }
             if (j == 0 && g == 0) trace_mark(p, stage, 4);
-            // ---- P V: thread e owns output dimension e
-            for (int e = gt; e < hd; e += 128) {
-                float acc[M];
+            // ---- P V: thread (c, kg) owns the 8 output dimensions of 16-byte chunk c for the keys kg, kg + 8, ... (one
+            //      16-byte read per key); the eight key groups of a chunk sit in neighbouring lanes and are added by an
+            //      xor butterfly. Up to six rows share one sweep over the keys (more rows: two or more sweeps).
+            //      Probabilities past n_valid are zero and the tile rows behind them hold finite cache contents.
+            {
+                constexpr int kRowBatch = M <= 6 ? M : (M <= 12 ? (M + 1) / 2 : 4);
+                const int kg = gt & 7;
+                const int n_steps = (n_valid + 7) >> 3;  // keys kg + 8 i, i < n_steps
+                for (int c0 = 0; c0 < (hd >> 3); c0 += 16) {  // every lane runs the loop (the butterfly below is warp-wide)
+                    const bool active = c0 + (gt >> 3) < (hd >> 3);
+                    const int c = active ? c0 + (gt >> 3) : 0;
+                    const int hb = (nhb > 1) ? (c >> 3) : 0, cc = (nhb > 1) ? (c & 7) : c;
+                    const int coff = (ta.swz ? (cc ^ kg) : cc) << 4;  // key & 7 == kg for every key of this thread
+#pragma unroll 1
+                    for (int m0 = 0; m0 < M; m0 += kRowBatch) {
+                        float acc[kRowBatch][8];
 #pragma unroll
-                for (int m = 0; m < M; ++m) acc[m] = 0.f;
-                const int c = e >> 3, sub = (e & 7) * 2;
-                const int hb = (nhb > 1) ? (c >> 3) : 0, cc = (nhb > 1) ? (c & 7) : c;
-                for (int rg = 0; rg * kBoxKeys < n_valid; ++rg) {  // keys in ascending order, one box after the other
-                    const unsigned char* vbox = slot_ptr(gv + rg * nhb + hb) + sub;
-                    const int nk = min(kBoxKeys, n_valid - rg * kBoxKeys);
-                    const float* prow = Ps + rg * kBoxKeys;
-#pragma unroll 4
-                    for (int rr = 0; rr < nk; ++rr) {
-                        const float v = __bfloat162float(
-                            *reinterpret_cast<const __nv_bfloat16*>(vbox + rr * ta.row_bytes + ((ta.swz ? (cc ^ (rr & 7)) : cc) << 4)));
+                        for (int u = 0; u < kRowBatch; ++u)
 #pragma unroll
-                        for (int m = 0; m < M; ++m) acc[m] = fmaf(prow[m * kAttnChunk + rr], v, acc[m]);
+                            for (int d8 = 0; d8 < 8; ++d8) acc[u][d8] = 0.f;
+                        for (int i = 0; i < n_steps; ++i) {
+                            const int key = kg + 8 * i;
+                            const unsigned char* vrow = slot_ptr(gv + (key / kBoxKeys) * nhb + hb) + (key % kBoxKeys) * ta.row_bytes + coff;
+                            const uint4 vv = *reinterpret_cast<const uint4*>(vrow);
+                            const float vf[8] = {bf_lo(vv.x), bf_hi(vv.x), bf_lo(vv.y), bf_hi(vv.y), bf_lo(vv.z), bf_hi(vv.z), bf_lo(vv.w), bf_hi(vv.w)};
+#pragma unroll
+                            for (int u = 0; u < kRowBatch; ++u)
+                                if (m0 + u < M) {
+                                    const float pw = Ps[(m0 + u) * kAttnChunk + key];
+#pragma unroll
+                                    for (int d8 = 0; d8 < 8; ++d8) acc[u][d8] = fmaf(pw, vf[d8], acc[u][d8]);
+                                }
+                        }
+#pragma unroll
+                        for (int u = 0; u < kRowBatch; ++u)
+                            if (m0 + u < M) {
+#pragma unroll
+                                for (int d8 = 0; d8 < 8; ++d8) {
+                                    float v = acc[u][d8];
+                                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                                    acc[u][d8] = v;
+                                }
+                                if (kg == 0 && active) {
+                                    float* dst = p.part_acc + (((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m0 + u) * hd + c * 8;
+                                    reinterpret_cast<float4*>(dst)[0] = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
+                                    reinterpret_cast<float4*>(dst)[1] = make_float4(acc[u][4], acc[u][5], acc[u][6], acc[u][7]);
+                                }
+                            }
                     }
                 }
-#pragma unroll
-                for (int m = 0; m < M; ++m)
-                    p.part_acc[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * hd + e] = acc[m];
             }
         }
         if (j == 0) trace_mark(p, stage, 5);

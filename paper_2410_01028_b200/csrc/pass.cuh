@@ -1206,35 +1206,45 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         if (*flag) {
             __threadfence();
             if (gt == 0) p.attn_counters[kvh] = 0u;
+            // warp w of the group merges rows w, w+4, ...; a lane owns four neighbouring output dimensions. The chunks
+            // are merged in ascending order, eight loads of a batch in flight together; explicit roundings keep the
+            // arithmetic identical in every instantiation of the kernel.
             for (int g = 0; g < group; ++g) {
                 const int head = kvh * group + g;
-                for (int e = gt; e < hd; e += 128) {
-#pragma unroll
-                    for (int m = 0; m < M; ++m) {
+                for (int e4 = glane * 4; e4 < hd; e4 += 128) {
+                    for (int m = gwarp; m < M; m += 4) {
                         const int nc = (p.pos0 + m) / kAttnChunk + 1;
-                        float mx = -INFINITY, l = 0.f, acc = 0.f;
-                        for (int c0 = 0; c0 < nc; c0 += 8) {  // loads of a batch are independent; the merge stays in chunk order
-                            float cm[8], cl[8], pa[8];
+                        float mx = -INFINITY, l = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        for (int c0 = 0; c0 < nc; c0 += 8) {
+                            float2 ml[8];
+                            float4 pa[8];
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 const int c = min(c0 + i, nc - 1);
                                 const size_t b = ((size_t)head * p.chunk_stride + c) * kPassMaxRows + m;
-                                cm[i] = __ldcg(p.part_ml + b * 2 + 0);
-                                cl[i] = __ldcg(p.part_ml + b * 2 + 1);
-                                pa[i] = __ldcg(p.part_acc + b * hd + e);
+                                ml[i] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + b * 2));
+                                pa[i] = __ldcg(reinterpret_cast<const float4*>(p.part_acc + b * hd + e4));
                             }
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 if (c0 + i < nc) {
-                                    const float mn = fmaxf(mx, cm[i]);
-                                    const float s_old = expf(mx - mn), s_new = expf(cm[i] - mn);
-                                    acc = acc * s_old + pa[i] * s_new;
-                                    l = l * s_old + cl[i] * s_new;
+                                    const float mn = fmaxf(mx, ml[i].x);
+                                    const float s_old = expf(mx - mn), s_new = expf(ml[i].x - mn);
+                                    acc[0] = __fmaf_rn(acc[0], s_old, __fmul_rn(pa[i].x, s_new));
+                                    acc[1] = __fmaf_rn(acc[1], s_old, __fmul_rn(pa[i].y, s_new));
+                                    acc[2] = __fmaf_rn(acc[2], s_old, __fmul_rn(pa[i].z, s_new));
+                                    acc[3] = __fmaf_rn(acc[3], s_old, __fmul_rn(pa[i].w, s_new));
+                                    l = __fmaf_rn(l, s_old, __fmul_rn(ml[i].y, s_new));
                                     mx = mn;
                                 }
                             }
                         }
-                        p.a[(size_t)m * p.d_model + (size_t)head * hd + e] = __float2bfloat16_rn(acc / l);
+                        const __nv_bfloat162 o01 = __floats2bfloat162_rn(__fdiv_rn(acc[0], l), __fdiv_rn(acc[1], l));
+                        const __nv_bfloat162 o23 = __floats2bfloat162_rn(__fdiv_rn(acc[2], l), __fdiv_rn(acc[3], l));
+                        uint2 o;
+                        o.x = *reinterpret_cast<const uint32_t*>(&o01);
+                        o.y = *reinterpret_cast<const uint32_t*>(&o23);
+                        *reinterpret_cast<uint2*>(p.a + (size_t)m * p.d_model + (size_t)head * hd + e4) = o;
                     }
                 }
             }

@@ -199,7 +199,7 @@ def oracle_sample(args, model, shape, prompt, steps, warmup):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+    _, rank, _ = rank_env()
     if rank != 0:
         return
     shape, S, new, desc = workload(args)
@@ -306,13 +306,37 @@ def gemm_roofline(torch, asd, shape):
             "status": int(status[0].item())}
 
 
+def rank_env():
+    """(world size, rank, local rank) from the environment torch.distributed.run sets up; (1, 0, 0) without it."""
+    return int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def max_over_ranks(value, world, device):
+    """A timing taken on every replica becomes the slowest replica's (replicas only: no data-path collective)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, steps, new_tokens, ms):
+    """Tokens per second of all replicas together: every replica generates `new_tokens` per step."""
+    return world * steps * new_tokens / (ms * 1e-3)
+
+
+def replica_prompt(vocab, n, rank):
+    """Every replica decodes its own sequence."""
+    return synth.make_prompt(vocab, n, seed=1 + rank)
+
+
 def run_ours(args):
     import torch
     import paper_2410_01028_b200 as asd
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     torch.cuda.set_device(local)
@@ -325,7 +349,7 @@ def run_ours(args):
     model = synth.make_model(shape, seed=0)
     dec = asd.Decoder(shape, max_seq=S + new + 16, max_draft=8, device="cuda:%d" % local)
     dec.load_weights_host(model)
-    prompt = synth.make_prompt(shape.vocab, S, seed=1 + rank)       # every replica decodes its own sequence
+    prompt = replica_prompt(shape.vocab, S, rank)
     dev_prompt = torch.from_numpy(prompt).cuda()
     dev_out = torch.zeros(new, dtype=torch.int32, device="cuda")
     kw = admg_kwargs(args)
@@ -355,13 +379,9 @@ def run_ours(args):
     e1.record()
     barrier()
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
     lossless = bool((dev_out.cpu().numpy() == ar_tokens).all())
-    value = world * args.steps * new / (ms * 1e-3)
+    value = whole_job_value(world, args.steps, new, ms)
 
     # end to end through the host-buffer entry point: prompt from pinned host memory, tokens back to the host
     pinned = torch.from_numpy(prompt).pin_memory()
@@ -371,12 +391,8 @@ def run_ours(args):
     for _ in range(args.steps):
         toks, _ = dec.generate(host_prompt, new, mode=asd.MODE_SPEC, **kw)
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * args.steps * new / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
+    e2e_s = max_over_ranks(time.perf_counter() - t0, world, "cuda")
+    e2e = {"value": whole_job_value(world, args.steps, new, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
            "d2h_bytes_per_step": int(toks.nbytes) + 4 * int(agg["rounds"] // args.steps) * (args.draft_len + 2)}
 
     if rank != 0:

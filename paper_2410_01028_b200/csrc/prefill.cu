@@ -158,14 +158,18 @@ __device__ __forceinline__ void epi_qkv(const GemmEpi& ep, int row, int col0, in
 }
 
 // ============================================================================================ the GEMM
-// One CTA computes a 128 x BN tile. Warp 0 (one lane) is the TMA producer, warp 1 (one lane) issues the MMAs and
-// owns the tensor-memory allocation, warps 2-5 are the epilogue (warp w reads lanes 32 * (w % 4) .. + 31 of tensor
-// memory, the quarter its position in the warp group gives it access to). Stages: full[s] (TMA bytes landed),
-// empty[s] (the MMAs reading stage s have finished: tcgen05.commit), acc (all MMAs of the tile have finished).
-// Ragged edges: TMA fills out-of-range rows and reduction elements with zeros; the epilogue skips rows >= M and
-// columns >= N. Every wait is bounded; after a failed wait the roles fall through to the common exit, where the
-// producer lets its copies in flight land and the tensor memory is freed.
+// Persistent CTAs (one per SM) walk the 128 x BN tiles of the product, row tiles fastest. Warp 0 (one lane) is the TMA
+// producer, warp 1 (one lane) issues the MMAs and owns the tensor-memory allocation, warps 2-5 are the epilogue (warp
+// w reads lanes 32 * (w % 4) .. + 31 of tensor memory, the quarter its position in the warp group gives it access
+// to). The accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of a tile runs while the
+// MMAs of the next tile are already filling the other buffer. Barriers: full[s] (TMA bytes landed in stage s),
+// empty[s] (the MMAs reading stage s have finished: tcgen05.commit), acc_full[b] (all MMAs of the tile in buffer b
+// have finished), acc_empty[b] (the 128 epilogue threads have read buffer b). Ragged edges: TMA fills out-of-range
+// rows and reduction elements with zeros; the epilogue skips rows >= M and columns >= N. Every wait is bounded; after
+// a failed wait the roles fall through to the common exit, where the producer lets its copies in flight land and
+// the tensor memory is freed.
 constexpr int kGemmThreads = 192;
+static int g_gemm_ctas = 148;  // persistent CTAs per launch: the SM count of the device (set by configure_prefill)
 
 template <int BN>
 struct GemmCfg {
@@ -179,20 +183,18 @@ struct GemmCfg {
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, int M, int N, int K, int m_tiles,
-               const GemmEpi ep) {
+               int n_tiles_total, const GemmEpi ep) {
     using Cfg = GemmCfg<BN>;
     constexpr int kStages = Cfg::kStages;
     extern __shared__ unsigned char gemm_smem_raw[];
     unsigned char* base = gemm_smem_raw + ((1024u - (smem_u32(gemm_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)kStages * Cfg::kStageBytes);
     uint64_t* empty = full + kStages;
-    uint64_t* acc_bar = empty + kStages;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+    uint64_t* acc_full = empty + kStages;   // [2]
+    uint64_t* acc_empty = acc_full + 2;     // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // row tiles vary fastest: CTAs that run together share their weight tile (read once from HBM, then from L2)
-    const int m_tile = blockIdx.x % m_tiles, n_tile = blockIdx.x / m_tiles;
-    const int m0 = m_tile * kGemmBM, n0 = n_tile * BN;
     const int num_kb = (K + kGemmBK - 1) / kGemmBK;
     volatile int* err = ep.err;
 
@@ -201,11 +203,14 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(acc_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 128);
+        }
         mbar_fence_init();
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, BN);
+        tmem_alloc(tmem_slot, 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -215,23 +220,27 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     if (warp == 0) {
         if (lane == 0) {
-            int issued = 0;
+            int issued = 0;  // k-blocks requested so far, over all tiles of this CTA
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % kStages;
-                if (kb >= kStages) ok = mbar_wait(&empty[s], (uint32_t)((kb / kStages - 1) & 1), err, kErrGemmWait, 0, kb, s, 1);
-                if (!ok) break;
-                unsigned char* a_dst = base + (size_t)s * Cfg::kStageBytes;
-                mbar_expect_tx(&full[s], Cfg::kStageBytes);
-                tma_load_2d(a_dst, &tm_a, kb * kGemmBK, m0, &full[s]);
-                tma_load_2d(a_dst + Cfg::kABytes, &tm_w, kb * kGemmBK, n0, &full[s]);
-                issued = kb + 1;
+            for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
+                // row tiles vary fastest: CTAs that run together share their weight tile (read once from HBM, then from L2)
+                const int m0 = (tile % m_tiles) * kGemmBM, n0 = (tile / m_tiles) * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    const int s = issued % kStages;
+                    if (issued >= kStages) ok = mbar_wait(&empty[s], (uint32_t)((issued / kStages - 1) & 1), err, kErrGemmWait, 0, issued, s, 1);
+                    if (!ok) break;
+                    unsigned char* a_dst = base + (size_t)s * Cfg::kStageBytes;
+                    mbar_expect_tx(&full[s], Cfg::kStageBytes);
+                    tma_load_2d(a_dst, &tm_a, kb * kGemmBK, m0, &full[s]);
+                    tma_load_2d(a_dst + Cfg::kABytes, &tm_w, kb * kGemmBK, n0, &full[s]);
+                    ++issued;
+                }
             }
             if (!ok || *err != kErrNone) {
                 // abandoned: let the copies still in flight land before the CTA gives its shared memory back
-                for (int kb = max(0, issued - kStages); kb < issued; ++kb) {
+                for (int i = max(0, issued - kStages); i < issued; ++i) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&full[kb % kStages], (uint32_t)((kb / kStages) & 1)) && clock64() - t0 < 20000000LL) {
+                    while (!mbar_try_wait(&full[i % kStages], (uint32_t)((i / kStages) & 1)) && clock64() - t0 < 20000000LL) {
                     }
                 }
             }
@@ -239,52 +248,70 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, BN);
+            int done = 0, local = 0;  // k-blocks consumed so far; tiles of this CTA started so far
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % kStages;
-                ok = mbar_wait(&full[s], (uint32_t)((kb / kStages) & 1), err, kErrGemmWait, 1, kb, s, 2);
+            for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+                const int buf = local & 1;
+                // the epilogue must have read this buffer's previous tile (tile local - 2) before it is overwritten
+                if (local >= 2) ok = mbar_wait(&acc_empty[buf], (uint32_t)((local / 2 - 1) & 1), err, kErrGemmWait, 3, local, buf, 4);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(base + (size_t)s * Cfg::kStageBytes);
-                const uint64_t a_desc = umma_desc_k128(a_addr), b_desc = umma_desc_k128(a_addr + Cfg::kABytes);
+                const uint32_t tmem_d = tmem + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    const int s = done % kStages;
+                    ok = mbar_wait(&full[s], (uint32_t)((done / kStages) & 1), err, kErrGemmWait, 1, done, s, 2);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(base + (size_t)s * Cfg::kStageBytes);
+                    const uint64_t a_desc = umma_desc_k128(a_addr), b_desc = umma_desc_k128(a_addr + Cfg::kABytes);
 #pragma unroll
-                for (int k = 0; k < kGemmBK / 16; ++k)  // 16 elements = 32 bytes further along the swizzled row: +2 in the address field
-                    tc_mma_bf16(tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
-                tc_commit(&empty[s]);  // the stage may be refilled once these MMAs have read it
+                    for (int k = 0; k < kGemmBK / 16; ++k)  // 16 elements = 32 bytes further along the swizzled row: +2 in the address field
+                        tc_mma_bf16(tmem_d, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc_commit(&empty[s]);  // the stage may be refilled once these MMAs have read it
+                    ++done;
+                }
+                tc_commit(&acc_full[buf]);  // arrives when every MMA issued above has finished
             }
-            tc_commit(acc_bar);  // arrives when every MMA issued above has finished (at once if none was issued)
         }
     } else {
         const int quarter = warp & 3;
-        const int row = m0 + quarter * 32 + lane;
-        const bool ok = mbar_wait(acc_bar, 0u, err, kErrGemmWait, 2, 0, 0, 3);
-        tc_fence_after();
-        if (ok && *err == kErrNone && num_kb > 0) {
+        bool ok = true;
+        int local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+            const int buf = local & 1;
+            const int m0 = (tile % m_tiles) * kGemmBM, n0 = (tile / m_tiles) * BN;
+            const int row = m0 + quarter * 32 + lane;
+            ok = mbar_wait(&acc_full[buf], (uint32_t)((local / 2) & 1), err, kErrGemmWait, 2, local, buf, 3) && *err == kErrNone;
+            tc_fence_after();
+            if (!ok) break;
             for (int cb = 0; cb < BN / 32; ++cb) {
                 const int col0 = n0 + cb * 32;
                 if (col0 >= N) break;  // uniform across the warp
                 float v[32];
-                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 32), v);
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cb * 32), v);
                 if (row < M) {
                     if (ep.mode == kGemmF32) epi_f32(ep, row, col0, N, v);
                     else if (ep.mode == kGemmSwiglu) epi_swiglu(ep, row, col0, N, v);
                     else epi_qkv(ep, row, col0, N, v);
                 }
             }
+            tc_fence_before();
+            mbar_arrive(&acc_empty[buf]);  // this thread has read its lanes of the buffer
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, BN);
+        tmem_dealloc(tmem, 2 * BN);
     }
 }
 
 template <int BN>
 static cudaError_t launch_gemm_bn(const CUtensorMap& tm_a, const CUtensorMap& tm_w, int M, int N, int K, const GemmEpi& ep, cudaStream_t s) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM, n_tiles = (N + BN - 1) / BN;
-    gemm_tn_kernel<BN><<<m_tiles * n_tiles, kGemmThreads, GemmCfg<BN>::kSmem, s>>>(tm_a, tm_w, M, N, K, m_tiles, ep);
+    const int total = m_tiles * n_tiles;
+    gemm_tn_kernel<BN><<<total < g_gemm_ctas ? total : g_gemm_ctas, kGemmThreads, GemmCfg<BN>::kSmem, s>>>(tm_a, tm_w, M, N, K, m_tiles, total, ep);
     return cudaGetLastError();
 }
 
@@ -605,6 +632,10 @@ cudaError_t launch_flash_prefill(const __nv_bfloat16* q, const __nv_bfloat16* k_
 cudaError_t configure_prefill(int max_smem) {
     cudaError_t e;
     (void)max_smem;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if (sms > 0) g_gemm_ctas = sms;
     if ((e = cudaFuncSetAttribute(gemm_tn_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<256>::kSmem)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(gemm_tn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<128>::kSmem)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(flash_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fa_smem_bytes<128>())) != cudaSuccess) return e;

@@ -26,10 +26,13 @@ def _pair(shape, max_seq, seed=0):
     return model, dec, oracle.Oracle(model, max_seq=max_seq)
 
 
-@pytest.mark.parametrize("base,layers,S,new", [(synth.LLAMA_7B, 2, 43, 6), (synth.LLAMA_13B, 1, 21, 4)])
-def test_full_width_few_layers_teacher_forced(base, layers, S, new):
+@pytest.mark.parametrize("base,layers,S,new,mode", [(synth.LLAMA_7B, 2, 43, 6, "gemm"), (synth.LLAMA_7B, 2, 43, 6, "rows"),
+                                                    (synth.LLAMA_13B, 1, 21, 4, "rows"), (synth.LLAMA_13B, 1, 37, 4, "gemm")])
+def test_full_width_few_layers_teacher_forced(base, layers, S, new, mode):
+    import paper_2410_01028_b200 as asd
     shape = dataclasses.replace(base, n_layers=layers)
     _, dec, orc = _pair(shape, max_seq=S + new + 16)
+    dec.set_prefill_mode(asd.PREFILL_GEMM if mode == "gemm" else asd.PREFILL_ROWS)   # both prompt paths at full width
     prompt = synth.make_prompt(shape.vocab, S, seed=1)
     teacher_forced_compare(dec, orc, prompt, new)
     ca_g, cm_g, _ = dec.get_similarity()

@@ -519,15 +519,16 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         // ---- scores of 16 rows x 64 keys
         float sc[8][4];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+        for (int nt = 0; nt < 8; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
 #pragma unroll
-            for (int k2 = 0; k2 < HD / 32; ++k2) {
-                uint32_t b[4];
-                ldsm_x4(b, Kb + (size_t)(nt * 8 + (lane & 7)) * LD + k2 * 32 + (lane >> 3) * 8);
-                mma16816(sc[nt], qf[2 * k2], b[0], b[1]);
-                mma16816(sc[nt], qf[2 * k2 + 1], b[2], b[3]);
-            }
+        for (int k2 = 0; k2 < HD / 32; ++k2) {  // 32 dimensions at a time over all 8 key blocks: consecutive MMAs are independent
+            uint32_t b[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) ldsm_x4(b[nt], Kb + (size_t)(nt * 8 + (lane & 7)) * LD + k2 * 32 + (lane >> 3) * 8);
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) mma16816(sc[nt], qf[2 * k2], b[nt][0], b[nt][1]);
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) mma16816(sc[nt], qf[2 * k2 + 1], b[nt][2], b[nt][3]);
         }
         // ---- scale, causal mask (the row at position p sees keys <= p), running maximum
         const int key0 = kt * kFaKeys + 2 * q4;
@@ -581,16 +582,26 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                 a_mid[u] = *reinterpret_cast<const uint32_t*>(&mid);
                 a_lo[u] = *reinterpret_cast<const uint32_t*>(&lo);
             }
+            // all value fragments of the 16 keys first, then one term of the probabilities after the other (smallest first)
+            // over all output blocks: consecutive MMAs never depend on each other
+            uint32_t b[HD / 16][4];
+#pragma unroll
+            for (int n2 = 0; n2 < HD / 16; ++n2)
+                ldsm_x4_trans(b[n2], Vb + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + n2 * 16 + (lane >> 4) * 8);
 #pragma unroll
             for (int n2 = 0; n2 < HD / 16; ++n2) {
-                uint32_t b[4];
-                ldsm_x4_trans(b, Vb + (size_t)(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + n2 * 16 + (lane >> 4) * 8);
-                mma16816(o[2 * n2], a_lo, b[0], b[1]);  // smallest terms first
-                mma16816(o[2 * n2 + 1], a_lo, b[2], b[3]);
-                mma16816(o[2 * n2], a_mid, b[0], b[1]);
-                mma16816(o[2 * n2 + 1], a_mid, b[2], b[3]);
-                mma16816(o[2 * n2], a_hi, b[0], b[1]);
-                mma16816(o[2 * n2 + 1], a_hi, b[2], b[3]);
+                mma16816(o[2 * n2], a_lo, b[n2][0], b[n2][1]);
+                mma16816(o[2 * n2 + 1], a_lo, b[n2][2], b[n2][3]);
+            }
+#pragma unroll
+            for (int n2 = 0; n2 < HD / 16; ++n2) {
+                mma16816(o[2 * n2], a_mid, b[n2][0], b[n2][1]);
+                mma16816(o[2 * n2 + 1], a_mid, b[n2][2], b[n2][3]);
+            }
+#pragma unroll
+            for (int n2 = 0; n2 < HD / 16; ++n2) {
+                mma16816(o[2 * n2], a_hi, b[n2][0], b[n2][1]);
+                mma16816(o[2 * n2 + 1], a_hi, b[n2][2], b[n2][3]);
             }
         }
         __syncthreads();  // this buffer is refilled two iterations from now

@@ -451,7 +451,7 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
 }
 
 template <int HD>
-__global__ void __launch_bounds__(kFaThreads)
+__global__ void __launch_bounds__(kFaThreads, 3)
 flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc, const __nv_bfloat16* __restrict__ vc,
                      __nv_bfloat16* __restrict__ out, int n_rows, int pos0, int d_model, int kv_dim, int group, int max_seq, float scale) {
     constexpr int LD = HD + 8;  // padded row: rows stay 16-byte aligned and ldmatrix reads are free of bank conflicts
@@ -459,7 +459,7 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     extern __shared__ __align__(16) unsigned char fa_smem[];
     __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(fa_smem);  // [2][64][LD]
     __nv_bfloat16* Vs = Ks + 2 * kFaKeys * LD;                      // [2][64][LD]
-    __nv_bfloat16* Qs = Vs + 2 * kFaKeys * LD;                      // [64][LD]
+    __nv_bfloat16* Qs = Vs + kFaKeys * LD;  // [64][LD]: the queries are staged in the second V buffer, which is first filled after they are in registers
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q4 = lane & 3;
     const int qt = gridDim.x - 1 - blockIdx.x;  // the tiles with the most keys start first
@@ -496,6 +496,7 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     uint32_t qf[HD / 16][4];
 #pragma unroll
     for (int kk = 0; kk < HD / 16; ++kk) ldsm_x4(qf[kk], Qs + (size_t)(warp * 16 + (lane & 15)) * LD + kk * 16 + (lane >> 4) * 8);
+    __syncthreads();  // every warp has its queries: the buffer may now receive values
 
     const int pos_a = pos0 + min(r0 + warp * 16 + g, n_rows - 1);
     const int pos_b = pos0 + min(r0 + warp * 16 + g + 8, n_rows - 1);
@@ -623,7 +624,7 @@ flash_prefill_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 }
 
 template <int HD>
-static constexpr size_t fa_smem_bytes() { return (size_t)5 * 64 * (HD + 8) * 2; }
+static constexpr size_t fa_smem_bytes() { return (size_t)4 * kFaKeys * (HD + 8) * 2; }
 
 cudaError_t launch_flash_prefill(const __nv_bfloat16* q, const __nv_bfloat16* k_cache, const __nv_bfloat16* v_cache, __nv_bfloat16* out,
                                  int n_rows, int pos0, int d_model, int kv_dim, int head_dim, int n_heads, int n_kv_heads, int max_seq,

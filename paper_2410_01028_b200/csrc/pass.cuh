@@ -473,7 +473,28 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             if (i < n_in) gpre[c] = *reinterpret_cast<const uint2*>(st.gain + i);
         }
     }
+    // One or two rows: what the epilogue will need from global memory is requested ahead of the weight stream
+    // (the rotary factors of this thread's pair before the barrier, the old hidden state of its row after it),
+    // so the epilogue does not wait for a memory round trip.
+    constexpr bool kPre = (M <= 2);
+    float pre[kPre ? 2 * M : 1];
+    if (kPre && type == kStQkv && tid < np) {
+        int ra, rb;
+        stage_pair_rows(type, p, pair0 + tid, ra, rb);
+        if (ra < p.d_model + p.kv_dim) {
+            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+#pragma unroll
+            for (int m = 0; m < (kPre ? M : 0); ++m) {
+                pre[m] = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
+                pre[M + m] = p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
+            }
+        }
+    }
     stage_begin(p, stage);
+    if (kPre && (type == kStOproj || type == kStDown) && tid < np * 2 && 2 * pair0 + tid < n_rows) {
+#pragma unroll
+        for (int m = 0; m < (kPre ? M : 0); ++m) pre[m] = __ldcg(p.x + (size_t)m * n_rows + 2 * pair0 + tid);
+    }
 
     // ---- RMSNorm statistics (same arithmetic for every row count). With one or two rows the hidden state read
     //      here stays in registers for the window fill below (one L2 round trip less per stage).
@@ -722,7 +743,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             if (row >= n_rows) continue;
             float xv[M];
 #pragma unroll
-            for (int m = 0; m < M; ++m) xv[m] = __ldcg(out + (size_t)m * n_rows + row);
+            for (int m = 0; m < M; ++m) xv[m] = (kPre && e == tid) ? pre[kPre ? m : 0] : __ldcg(out + (size_t)m * n_rows + row);
 #pragma unroll
             for (int m = 0; m < M; ++m) {
                 float v = psum[e * M + m];
@@ -746,8 +767,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             const int half = p.head_dim >> 1, jr = ra % p.head_dim;
 #pragma unroll
             for (int m = 0; m < M; ++m) {
-                rc[m] = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
-                rs[m] = p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
+                rc[m] = (kPre && pl == tid) ? pre[kPre ? m : 0] : p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
+                rs[m] = (kPre && pl == tid) ? pre[kPre ? M + m : 0] : p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
             }
         }
 #pragma unroll
@@ -1004,9 +1025,24 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             const int m = i / hd, e = i - m * hd;
             qreg[u] = (i < M * hd && q_head != kvh * group) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
         }
-        for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
         const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
         const int n_fresh = fresh1 - fresh0 + 1;
+        // one or two rows: the fresh V rows are requested here too, so patching the V tile later costs no round trip
+        constexpr bool kVEarly = (M <= 2);
+        constexpr int kVPre = kVEarly ? (M * 32 + 127) / 128 : 1;  // head_dim <= 256: at most 32 vectors per row
+        uint4 vpre[kVPre];
+        if (kVEarly) {
+#pragma unroll
+            for (int u = 0; u < kVPre; ++u) {
+                const int i = gt + u * 128;
+                vpre[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (i < n_fresh * vec_per_row) {
+                    const int fr = i / vec_per_row, c = i - fr * vec_per_row;
+                    vpre[u] = __ldcg(reinterpret_cast<const uint4*>(st.v_cache + (size_t)(fresh0 + fr) * p.kv_dim + (size_t)kvh * hd + c * 8));
+                }
+            }
+        }
+        for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
         if (n_fresh > 0) {
             for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
                 const int fr = i / vec_per_row, c = i - fr * vec_per_row;
@@ -1106,7 +1142,18 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
             if (g == 0) {  // V tile: wait and patch once per item
                 for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gv + t, stage, M * 1000 + 500 + j);
-                if (n_fresh > 0) {
+                if (kVEarly) {
+#pragma unroll
+                    for (int u = 0; u < kVPre; ++u) {
+                        const int i = gt + u * 128;
+                        if (i < n_fresh * vec_per_row) {
+                            const int fr = i / vec_per_row, c = i - fr * vec_per_row;
+                            int sit, off;
+                            ta.locate(fresh0 + fr - key0, c, sit, off);
+                            *reinterpret_cast<uint4*>(slot_ptr(gv + sit) + off) = vpre[u];
+                        }
+                    }
+                } else if (n_fresh > 0) {
                     for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
                         const int fr = i / vec_per_row, c = i - fr * vec_per_row;
                         const int r = fresh0 + fr - key0;
@@ -1188,13 +1235,15 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         ++run_cnt;
         const int jn = j + p.attn_groups;
         const bool report = (jn >= n_local) || ((first + jn) / n_chunks != kvh);
-        if (report) __threadfence();
         bar_sync(bar_id, 128);
         if (gt == 0) {
             fence_proxy_async_smem();
             for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
             if (report) {
-                const unsigned tk = atomicAdd(p.attn_counters + kvh, run_cnt);
+                // release: the group's partial results (ordered before this thread by the barrier above) are visible
+                // to whoever reads the count; acquire: so are those of the groups that reported earlier
+                unsigned tk;
+                asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(tk) : "l"(p.attn_counters + kvh), "r"(run_cnt) : "memory");
                 *flag = (tk + run_cnt == (unsigned)n_chunks) ? 1 : 0;
             } else {
                 *flag = 0;
@@ -1204,7 +1253,6 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         bar_sync(bar_id, 128);
         if (j == 0) trace_mark(p, stage, 6);
         if (*flag) {
-            __threadfence();
             if (gt == 0) p.attn_counters[kvh] = 0u;
             // warp w of the group merges rows w, w+4, ...; a lane owns four neighbouring output dimensions. The chunks
             // are merged in ascending order, eight loads of a batch in flight together; explicit roundings keep the

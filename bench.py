@@ -56,6 +56,10 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=5, help="ADMG rule subset: 1=CS thresholding, 2=rule 1, 4=rule 2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemv-microbench", action="store_true", help="also time the stand-alone fused GEMV kernel")
+    ap.add_argument("--ablation", action="store_true", help="also time the rule subsets of the paper's ablation (Table 5) and "
+                    "the two extensions (MLP similarity threshold, running similarities) end to end")
+    ap.add_argument("--alpha-mlp", type=float, default=0.9995, help="MLP similarity threshold of the ablation's extension rows")
+    ap.add_argument("--refresh", type=int, default=8, help="rounds between mask updates of the ablation's running-similarity row")
     ap.add_argument("--gemm-microbench", action="store_true", help="also time the stand-alone tensor-core GEMM of the prompt path")
     # reduced cases for profiler captures only (never for a reported number)
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
@@ -306,6 +310,27 @@ def gemm_roofline(torch, asd, shape):
             "status": int(status[0].item())}
 
 
+def ablation(torch, asd, dec, dev_prompt, dev_out, new, args, ar_tokens):
+    """One speculative generation per rule subset of the paper's ablation (Table 5: similarity threshold alone, with
+    rule 2, rules 1 and 2 alone, all three) and per extension, with the hyper-parameters of the command line."""
+    CS, R1, R2 = asd.USE_CS, asd.USE_RULE1, asd.USE_RULE2
+    rows = [("CS", CS), ("CS + rule 2", CS | R2), ("rules 1 and 2", R1 | R2), ("CS + rules 1 and 2 (Algorithm 1)", CS | R1 | R2),
+            ("CS + rule 2 + MLP threshold", CS | R2 | asd.USE_CS_MLP),
+            ("CS + rule 2 + MLP threshold, running similarities", CS | R2 | asd.USE_CS_MLP | asd.RUNNING_C)]
+    out = []
+    for name, flags in rows:
+        kw = dict(draft_len=args.draft_len, alpha=args.alpha, m=args.m, n=args.n, flags=flags, alpha_mlp=args.alpha_mlp,
+                  refresh=args.refresh if flags & asd.RUNNING_C else 0)
+        dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)  # warm-up
+        _, st = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        same = bool((dev_out.cpu().numpy() == ar_tokens).all())
+        ra, rm = dec.admg_update(args.alpha, args.m, args.n, flags, alpha_mlp=args.alpha_mlp)
+        out.append({"rules": name, "flags": flags, "tokens_per_s": new / (st["ms_total"] * 1e-3),
+                    "acceptance": st["accepted"] / max(st["drafted"], 1), "removed_attn": int(ra.sum()), "removed_mlp": int(rm.sum()),
+                    "draft_ms": st["ms_draft"] / max(st["draft_passes"], 1), "spec_equals_ar": same})
+    return out
+
+
 def rank_env():
     """(world size, rank, local rank) from the environment torch.distributed.run sets up; (1, 0, 0) without it."""
     return int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
@@ -451,6 +476,8 @@ def run_ours(args):
         "acceptance": agg["accepted"] / max(agg["drafted"], 1), "rounds_per_step": agg["rounds"] / args.steps,
         "spec_equals_ar": lossless,
     }
+    if args.ablation:
+        line["ablation"] = ablation(torch, asd, dec, dev_prompt, dev_out, new, args, ar_tokens)
     if not args.no_cpu_baseline:
         cb, _ = oracle_sample(args, model, shape, synth.make_prompt(shape.vocab, S, seed=1), 1, 0)
         line["cpu_baseline"] = cb

@@ -75,10 +75,20 @@ typedef struct {
 #define ASD_USE_RULE1 2u /* remove every m-th attention and MLP layer */
 #define ASD_USE_RULE2 4u /* never remove the last n layers */
 #define ASD_ADMG_ALL 7u
+/* Two extensions that the paper does not have, both off unless their flag is set:
+ *   ASD_USE_CS_MLP  Table 1 measures the MLP similarities but Algorithm 1 never looks at them. With this flag an MLP
+ *                   layer l <= L - n is also removed when its own C_l reaches alpha_mlp (remove_ATTN is unchanged).
+ *   ASD_RUNNING_C   Section 3.2 computes C_l over the prompt only. With this flag every row that a full-model pass
+ *                   commits after the prompt (decode steps, the accepted rows of a verify pass) joins the mean, and
+ *                   asd_generate runs Algorithm 1 again on the refreshed C_l every `refresh` rounds (0 = never). */
+#define ASD_USE_CS_MLP 8u
+#define ASD_RUNNING_C 16u
 typedef struct {
     float alpha;
     int32_t m, n;
     uint32_t flags;
+    float alpha_mlp; /* threshold of ASD_USE_CS_MLP; ignored without that flag */
+    int32_t refresh; /* rounds between mask updates under ASD_RUNNING_C; ignored without that flag */
 } asd_admg_params;
 
 #define ASD_MODE_AR 0               /* plain greedy decoding with M */
@@ -133,6 +143,10 @@ int asd_get_similarity(asd_ctx* ctx, float* c_attn, float* c_mlp, int32_t* n_row
 /* Algorithm 1 on the current C: computes remove_ATTN / remove_MLP, installs them as the draft model's skip
  * mask and optionally returns them (uint8[L], 1 = removed). Resets the draft cursor. */
 int asd_admg_update(asd_ctx* ctx, const asd_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp);
+/* Turns the running similarities (ASD_RUNNING_C, see asd_admg_params) on or off for the single-step calls:
+ * while on, asd_decode_step adds its row and asd_verify its a+1 committed rows to the sums behind C_l.
+ * asd_generate sets it from its parameters' flags. asd_reset leaves it as it is. */
+int asd_set_running_similarity(asd_ctx* ctx, int32_t on);
 /* Install a mask by hand (uint8[L] each, non-zero = skip). Resets the draft cursor. */
 int asd_set_skip_mask(asd_ctx* ctx, const uint8_t* skip_attn, const uint8_t* skip_mlp);
 
@@ -248,6 +262,10 @@ int asd_fused_gemv_static(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_
 
 /* Algorithm 1 as a pure host function (no context): C[L] -> remove_attn[L], remove_mlp[L]. */
 int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp);
+/* Algorithm 1 plus the MLP threshold of ASD_USE_CS_MLP: C_attn[L], C_mlp[L] (C_mlp may be NULL unless that flag is
+ * set) -> remove_attn[L], remove_mlp[L]. Pure host function. Errors: ARG. */
+int asd_admg_ext(const float* C_attn, const float* C_mlp, int32_t L, const asd_admg_params* p, uint8_t* remove_attn,
+                 uint8_t* remove_mlp);
 
 #ifdef __cplusplus
 }

@@ -17,6 +17,7 @@ _SRC = os.path.join(_HERE, "orc.cpp")
 _LIB = os.path.join(_HERE, "liborc.so")
 
 USE_CS, USE_RULE1, USE_RULE2 = 1, 2, 4
+USE_CS_MLP, RUNNING_C = 8, 16  # extensions beyond Algorithm 1, off by default
 ADMG_ALL = USE_CS | USE_RULE1 | USE_RULE2
 MODE_AR, MODE_SPEC, MODE_SPEC_MANUAL_MASK = 0, 1, 2
 FLAG_NO_ROUNDING = 1
@@ -42,7 +43,8 @@ class Weights(ctypes.Structure):
 
 
 class AdmgParams(ctypes.Structure):
-    _fields_ = [("alpha", ctypes.c_float), ("m", ctypes.c_int32), ("n", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+    _fields_ = [("alpha", ctypes.c_float), ("m", ctypes.c_int32), ("n", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("alpha_mlp", ctypes.c_float), ("refresh", ctypes.c_int32)]
 
 
 class GenParams(ctypes.Structure):
@@ -102,6 +104,19 @@ def admg(C, alpha: float, m: int, n: int, flags: int = ADMG_ALL):
     _check(lib().orc_admg(ctypes.c_void_p(C.ctypes.data), ctypes.c_int32(L), ctypes.c_float(alpha), ctypes.c_int32(m),
                           ctypes.c_int32(n), ctypes.c_uint32(flags), ctypes.c_void_p(ra.ctypes.data),
                           ctypes.c_void_p(rm.ctypes.data)), "orc_admg")
+    return ra, rm
+
+
+def admg_ext(C_attn, C_mlp, alpha: float, alpha_mlp: float, m: int, n: int, flags: int):
+    """Algorithm 1 plus the optional MLP similarity threshold (``USE_CS_MLP``).  Returns (remove_attn, remove_mlp)."""
+    C_attn, C_mlp = _f32(C_attn), _f32(C_mlp)
+    L = C_attn.size
+    assert C_mlp.size == L
+    ra, rm = np.zeros(L, np.uint8), np.zeros(L, np.uint8)
+    _check(lib().orc_admg_ext(ctypes.c_void_p(C_attn.ctypes.data), ctypes.c_void_p(C_mlp.ctypes.data), ctypes.c_int32(L),
+                              ctypes.c_float(alpha), ctypes.c_float(alpha_mlp), ctypes.c_int32(m), ctypes.c_int32(n),
+                              ctypes.c_uint32(flags), ctypes.c_void_p(ra.ctypes.data), ctypes.c_void_p(rm.ctypes.data)),
+           "orc_admg_ext")
     return ra, rm
 
 
@@ -195,10 +210,13 @@ class Oracle:
         _check(lib().orc_set_skip_mask(self._ctx, ctypes.c_void_p(a.ctypes.data), ctypes.c_void_p(b.ctypes.data)),
                "orc_set_skip_mask")
 
-    def admg_update(self, alpha=0.985, m=3, n=2, flags=ADMG_ALL):
+    def set_running_similarity(self, on: bool):
+        _check(lib().orc_set_running_similarity(self._ctx, ctypes.c_int32(1 if on else 0)), "orc_set_running_similarity")
+
+    def admg_update(self, alpha=0.985, m=3, n=2, flags=ADMG_ALL, alpha_mlp=1.0, refresh=0):
         L = self.shape.n_layers
         a, b = np.zeros(L, np.uint8), np.zeros(L, np.uint8)
-        p = AdmgParams(alpha, m, n, flags)
+        p = AdmgParams(alpha, m, n, flags, alpha_mlp, refresh)
         _check(lib().orc_admg_update(self._ctx, ctypes.byref(p), ctypes.c_void_p(a.ctypes.data),
                                      ctypes.c_void_p(b.ctypes.data)), "orc_admg_update")
         return a, b
@@ -223,10 +241,10 @@ class Oracle:
         return a.value, out[: a.value + 1].copy()
 
     def generate(self, prompt, max_new: int, mode: int = MODE_AR, draft_len: int = 4, alpha=0.985, m=3, n=2,
-                 flags=ADMG_ALL, eos_id: int = -1):
+                 flags=ADMG_ALL, eos_id: int = -1, alpha_mlp=1.0, refresh=0):
         """Returns (tokens, margins, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags))
+        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh))
         out = np.zeros(max_new, np.int32)
         margins = np.zeros(max_new, np.float32)
         n_out = ctypes.c_int32()

@@ -35,6 +35,10 @@
 // attention output equals the value row; rotation at position 0 is the
 // identity; a numpy restatement of single sublayers; speculative == greedy
 // autoregressive output for every mask and draft length.
+// Two opt-in extensions that the paper does not have (off by default): MLP sublayers removed by their own
+// similarity (orc_admg_ext; pinned by brute force over all masks on L=2), and C_l kept running over the rows
+// committed after the prompt, with Algorithm 1 run again every few rounds (pinned: the running C_l after a
+// generation equals the C_l of one prefill over prompt + emitted tokens, for both decoding modes).
 // Parity unpinned: absolute token ids / logits of the random synthetic models
 // (the paper prints no worked example).
 #include <algorithm>
@@ -111,7 +115,7 @@ typedef struct {  // bf16 bit patterns, row-major [out,in], stacked over layers;
     const uint16_t *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *wg, *wu, *wd;
 } orc_weights;
 
-typedef struct { float alpha; int32_t m, n; uint32_t flags; } orc_admg_params;
+typedef struct { float alpha; int32_t m, n; uint32_t flags; float alpha_mlp; int32_t refresh; } orc_admg_params;
 typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; } orc_gen_params;
 typedef struct {
     int64_t full_passes, draft_passes, verify_passes, rounds, drafted, accepted, prefill_rows;
@@ -119,7 +123,7 @@ typedef struct {
 } orc_stats;
 
 enum { ORC_FLAG_NO_ROUNDING = 1u };
-enum { ORC_USE_CS = 1u, ORC_USE_RULE1 = 2u, ORC_USE_RULE2 = 4u };
+enum { ORC_USE_CS = 1u, ORC_USE_RULE1 = 2u, ORC_USE_RULE2 = 4u, ORC_USE_CS_MLP = 8u, ORC_RUNNING_C = 16u };
 enum { ORC_MODE_AR = 0, ORC_MODE_SPEC = 1, ORC_MODE_SPEC_MANUAL_MASK = 2 };
 enum { ORC_OK = 0, ORC_ERR_ARG = -1, ORC_ERR_STATE = -2, ORC_ERR_OVERFLOW = -4 };
 
@@ -157,6 +161,22 @@ int orc_admg(const float* C, int32_t L, float alpha, int32_t m, int32_t n, uint3
     return ORC_OK;
 }
 
+// Extension beyond Algorithm 1 (the paper measures the MLP similarities, Table 1, but its rule never looks at
+// them): with ORC_USE_CS_MLP an MLP sublayer is also removed when its own similarity reaches alpha_mlp, under
+// the same protection of the last n layers.  remove_ATTN stays exactly Algorithm 1's set.
+//   remove_MLP' = remove_MLP  union  { l : Cmlp_l >= alpha_mlp, l <= L-n }
+int orc_admg_ext(const float* C_attn, const float* C_mlp, int32_t L, float alpha, float alpha_mlp, int32_t m, int32_t n,
+                 uint32_t flags, uint8_t* remove_attn, uint8_t* remove_mlp) {
+    const int rc = orc_admg(C_attn, L, alpha, m, n, flags, remove_attn, remove_mlp);
+    if (rc) return rc;
+    if (!(flags & ORC_USE_CS_MLP)) return ORC_OK;
+    if (!C_mlp) return ORC_ERR_ARG;
+    const int32_t n_eff = (flags & ORC_USE_RULE2) ? n : 0;
+    for (int32_t l = 1; l <= L - n_eff; ++l)
+        if (C_mlp[l - 1] >= alpha_mlp) remove_mlp[l - 1] = 1;
+    return ORC_OK;
+}
+
 // ---------------------------------------------------------------- decoder state
 struct orc_ctx {
     orc_config c;
@@ -170,6 +190,7 @@ struct orc_ctx {
     std::vector<uint8_t> skip_attn, skip_mlp;
     std::vector<double> sumcos_attn, sumcos_mlp;  // running sums over prompt rows
     int64_t n_sim_rows = 0;
+    bool running_c = false;          // fold the rows committed after the prompt into the sums as well (opt-in)
     // results of the last pass
     int32_t last_M = 0;
     std::vector<float> last_logits;              // [M][V]
@@ -397,6 +418,24 @@ static int forward_rows(orc_ctx* x, const int32_t* tokens, int M, int pos0, bool
     return ORC_OK;
 }
 
+// Opt-in extension (the paper computes C_l over the prompt only): the first n rows of the last full-model pass,
+// which the caller has just committed, join the mean.  C_l then is the mean over every committed row.
+static void fold_committed_rows(orc_ctx* x, int n) {
+    const int M = x->last_M;
+    for (int l = 0; l < x->c.n_layers; ++l)
+        for (int m = 0; m < n; ++m) {
+            x->sumcos_attn[l] += (double)x->last_cos_attn[(size_t)l * M + m];
+            x->sumcos_mlp[l] += (double)x->last_cos_mlp[(size_t)l * M + m];
+        }
+    x->n_sim_rows += n;
+}
+
+int orc_set_running_similarity(orc_ctx* x, int32_t on) {
+    if (!x) return ORC_ERR_ARG;
+    x->running_c = on != 0;
+    return ORC_OK;
+}
+
 // Section 3.2: the whole input context goes through M, fills the KV cache, yields t_1 and the
 // per-layer similarity sums.  May be called repeatedly to feed the prompt in pieces.
 int orc_prefill(orc_ctx* x, const int32_t* tokens, int32_t n, int32_t* first_token) {
@@ -437,11 +476,11 @@ int orc_set_skip_mask(orc_ctx* x, const uint8_t* skip_attn, const uint8_t* skip_
 // Algorithm 1 on the attention similarities of the prompt; installs the result as the draft model's mask
 int orc_admg_update(orc_ctx* x, const orc_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp) {
     if (!x || !p) return ORC_ERR_ARG;
-    std::vector<float> C(x->c.n_layers);
-    int rc = orc_get_similarity(x, C.data(), nullptr, nullptr);
+    std::vector<float> C(x->c.n_layers), Cm(x->c.n_layers);
+    int rc = orc_get_similarity(x, C.data(), Cm.data(), nullptr);
     if (rc) return rc;
     std::vector<uint8_t> a(x->c.n_layers), b(x->c.n_layers);
-    rc = orc_admg(C.data(), x->c.n_layers, p->alpha, p->m, p->n, p->flags, a.data(), b.data());
+    rc = orc_admg_ext(C.data(), Cm.data(), x->c.n_layers, p->alpha, p->alpha_mlp, p->m, p->n, p->flags, a.data(), b.data());
     if (rc) return rc;
     orc_set_skip_mask(x, a.data(), b.data());
     if (skip_attn) std::memcpy(skip_attn, a.data(), a.size());
@@ -457,6 +496,7 @@ int orc_decode_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
     if (rc) return rc;
     x->n_committed += 1;
     x->draft_cursor = x->n_committed;
+    if (x->running_c) fold_committed_rows(x, 1);
     x->stats.full_passes += 1;
     x->stats.ms_full += now_ms() - t0;
     if (token_out) *token_out = x->last_argmax[0];
@@ -493,6 +533,7 @@ int orc_verify(orc_ctx* x, const int32_t* tokens, int32_t k, int32_t* n_accepted
     if (n_accepted) *n_accepted = a;
     x->n_committed += a + 1;
     x->draft_cursor = x->n_committed;
+    if (x->running_c) fold_committed_rows(x, a + 1);
     x->stats.verify_passes += 1;
     x->stats.drafted += k;
     x->stats.accepted += a;
@@ -510,6 +551,7 @@ int orc_generate(orc_ctx* x, const int32_t* prompt, int32_t n_prompt, const orc_
     std::vector<uint8_t> ka = x->skip_attn, km = x->skip_mlp;
     orc_reset(x);
     if (gp->mode == ORC_MODE_SPEC_MANUAL_MASK) orc_set_skip_mask(x, ka.data(), km.data());
+    x->running_c = (gp->admg.flags & ORC_RUNNING_C) != 0;
     const double t0 = now_ms();
     int32_t last;
     int rc = orc_prefill(x, prompt, n_prompt, &last);
@@ -555,6 +597,11 @@ int orc_generate(orc_ctx* x, const int32_t* prompt, int32_t n_prompt, const orc_
             stop = (gp->eos_id >= 0 && acc[j] == gp->eos_id);
         }
         last = acc[a];
+        // running similarities: Algorithm 1 is run again on the refreshed C_l every `refresh` rounds
+        if (gp->mode == ORC_MODE_SPEC && x->running_c && gp->admg.refresh > 0 && x->stats.rounds % gp->admg.refresh == 0) {
+            rc = orc_admg_update(x, &gp->admg, nullptr, nullptr);
+            if (rc) return rc;
+        }
     }
     *n_out = produced;
     x->stats.ms_total = now_ms() - t0;

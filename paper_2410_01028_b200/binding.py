@@ -9,6 +9,7 @@ import numpy as np
 from . import build as _build
 
 USE_CS, USE_RULE1, USE_RULE2, ADMG_ALL = 1, 2, 4, 7
+USE_CS_MLP, RUNNING_C = 8, 16  # extensions beyond Algorithm 1 (see asd_admg_params), off by default
 MODE_AR, MODE_SPEC, MODE_SPEC_MANUAL_MASK = 0, 1, 2
 EPI_PLAIN, EPI_SWIGLU, EPI_RESIDUAL = 0, 1, 2
 PREFILL_AUTO, PREFILL_ROWS, PREFILL_GEMM = 0, 1, 2
@@ -27,7 +28,8 @@ class HostWeights(ctypes.Structure):
 
 
 class AdmgParams(ctypes.Structure):
-    _fields_ = [("alpha", ctypes.c_float), ("m", ctypes.c_int32), ("n", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+    _fields_ = [("alpha", ctypes.c_float), ("m", ctypes.c_int32), ("n", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("alpha_mlp", ctypes.c_float), ("refresh", ctypes.c_int32)]
 
 
 class GenParams(ctypes.Structure):
@@ -52,7 +54,7 @@ EXPORTS = (
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
     "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
-    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_set_prefill_mode", "asd_gemm_bf16",
+    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_admg_ext", "asd_set_running_similarity", "asd_set_prefill_mode", "asd_gemm_bf16",
 )
 
 _lib = None
@@ -109,6 +111,19 @@ def admg(C, alpha, m, n, flags=ADMG_ALL):
     rc = lib().asd_admg(_vp(C), ctypes.c_int32(C.size), ctypes.byref(p), _vp(ra), _vp(rm))
     if rc:
         raise AsdError(rc, "asd_admg")
+    return ra, rm
+
+
+def admg_ext(C_attn, C_mlp, alpha, alpha_mlp, m, n, flags):
+    """Algorithm 1 plus the MLP similarity threshold of ``USE_CS_MLP``: (remove_attn, remove_mlp)."""
+    C_attn = np.ascontiguousarray(C_attn, dtype=np.float32)
+    C_mlp = np.ascontiguousarray(C_mlp, dtype=np.float32)
+    assert C_attn.size == C_mlp.size
+    ra, rm = np.zeros(C_attn.size, np.uint8), np.zeros(C_attn.size, np.uint8)
+    p = AdmgParams(alpha, m, n, flags, alpha_mlp, 0)
+    rc = lib().asd_admg_ext(_vp(C_attn), _vp(C_mlp), ctypes.c_int32(C_attn.size), ctypes.byref(p), _vp(ra), _vp(rm))
+    if rc:
+        raise AsdError(rc, "asd_admg_ext")
     return ra, rm
 
 
@@ -258,10 +273,13 @@ class Decoder:
         self._check(lib().asd_get_similarity(self._ctx, _vp(ca), _vp(cm), ctypes.byref(n)), "asd_get_similarity")
         return ca, cm, n.value
 
-    def admg_update(self, alpha=0.985, m=3, n=2, flags=ADMG_ALL):
+    def set_running_similarity(self, on):
+        self._check(lib().asd_set_running_similarity(self._ctx, ctypes.c_int32(1 if on else 0)), "asd_set_running_similarity")
+
+    def admg_update(self, alpha=0.985, m=3, n=2, flags=ADMG_ALL, alpha_mlp=1.0, refresh=0):
         L = self.shape.n_layers
         a, b = np.zeros(L, np.uint8), np.zeros(L, np.uint8)
-        p = AdmgParams(alpha, m, n, flags)
+        p = AdmgParams(alpha, m, n, flags, alpha_mlp, refresh)
         self._check(lib().asd_admg_update(self._ctx, ctypes.byref(p), _vp(a), _vp(b)), "asd_admg_update")
         return a, b
 
@@ -289,13 +307,14 @@ class Decoder:
         self._check(lib().asd_verify(self._ctx, _vp(t), ctypes.c_int32(k), ctypes.byref(a), _vp(out)), "asd_verify")
         return a.value, out[: a.value + 1].copy()
 
-    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id):
-        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags))
+    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp=1.0, refresh=0):
+        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh))
 
-    def generate(self, prompt, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2, flags=ADMG_ALL, eos_id=-1):
+    def generate(self, prompt, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2, flags=ADMG_ALL, eos_id=-1,
+                 alpha_mlp=1.0, refresh=0):
         """Host buffers in, host buffers out. Returns (tokens, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh)
         out = np.zeros(max_new, np.int32)
         n_out = ctypes.c_int32()
         st = Stats()
@@ -304,9 +323,9 @@ class Decoder:
         return out[: n_out.value].copy(), st.as_dict()
 
     def generate_device(self, dev_prompt, dev_out, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2,
-                        flags=ADMG_ALL, eos_id=-1):
+                        flags=ADMG_ALL, eos_id=-1, alpha_mlp=1.0, refresh=0):
         """Prompt and output are int32 CUDA tensors. Returns (n_out, stats dict)."""
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh)
         n_out = ctypes.c_int32()
         st = Stats()
         self._check(lib().asd_generate_device(self._ctx, _vp(dev_prompt), ctypes.c_int32(dev_prompt.numel()),

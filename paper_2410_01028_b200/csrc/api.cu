@@ -297,6 +297,10 @@ struct asd_ctx {
     int n_committed = 0, draft_cursor = 0;
     std::vector<uint8_t> skip_attn, skip_mlp;
     int64_t n_sim_rows = 0;
+    // running similarities (ASD_RUNNING_C): sums over the rows committed after the prompt, kept on the host
+    bool running_c = false;
+    std::vector<double> run_attn, run_mlp;
+    int64_t n_run_rows = 0;
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, trace = false;
     int last_n_stages = 0;
@@ -602,20 +606,51 @@ static int read_back(asd_ctx* x, const int* dev_src, int n) {
     return check_device_error(x, x->pinned + 32);
 }
 
+// Running similarities: request the per-row cosines of the pass that has just been launched (before the caller's
+// read_back, whose synchronisation also covers this copy) ...
+static int request_cosines(asd_ctx* x) {
+    if (!x->running_c) return ASD_OK;
+    const size_t n = (size_t)2 * std::max(x->c.n_layers, 1) * kPassMaxRows;
+    ASD_CUDA(x, cudaMemcpyAsync(x->pinned + 1024, x->ws + x->lay.cosv, n * 4, cudaMemcpyDeviceToHost, x->stream));
+    return ASD_OK;
+}
+// ... and add its first n_rows rows, which the caller has just committed, to the sums (rows in order, in double).
+static void fold_committed_rows(asd_ctx* x, int n_rows) {
+    if (!x->running_c) return;
+    const int L = x->c.n_layers;
+    const float* h = reinterpret_cast<const float*>(x->pinned + 1024);
+    for (int l = 0; l < L; ++l)
+        for (int r = 0; r < n_rows; ++r) {
+            x->run_attn[l] += (double)h[((size_t)0 * L + l) * kPassMaxRows + r];
+            x->run_mlp[l] += (double)h[((size_t)1 * L + l) * kPassMaxRows + r];
+        }
+    x->n_run_rows += n_rows;
+}
+
 // ---------------------------------------------------------------- Algorithm 1
 // remove_MLP = { l : l = j*m, j >= 1, l <= L-n };  remove_ATTN = { l : C_l >= alpha, l <= L-n } U remove_MLP,
 // layers numbered from 1. flags drop individual rules (Table 5).
-extern "C" int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp) {
-    if (!C || !p || !remove_attn || !remove_mlp || L < 0 || p->m < 0 || p->n < 0) return ASD_ERR_ARG;
+// With ASD_USE_CS_MLP (not in the paper) an MLP layer l <= L-n also goes when its own similarity reaches alpha_mlp;
+// remove_ATTN keeps Algorithm 1's definition (its union is with rule 1's set only).
+extern "C" int asd_admg_ext(const float* C_attn, const float* C_mlp, int32_t L, const asd_admg_params* p, uint8_t* remove_attn,
+                            uint8_t* remove_mlp) {
+    if (!C_attn || !p || !remove_attn || !remove_mlp || L < 0 || p->m < 0 || p->n < 0) return ASD_ERR_ARG;
     const bool cs = p->flags & ASD_USE_CS, r1 = (p->flags & ASD_USE_RULE1) && p->m >= 1, r2 = p->flags & ASD_USE_RULE2;
+    const bool cs_mlp = p->flags & ASD_USE_CS_MLP;
+    if (cs_mlp && !C_mlp) return ASD_ERR_ARG;
     const int32_t last_removable = L - (r2 ? p->n : 0);
     for (int32_t i = 0; i < L; ++i) {
         const int32_t l = i + 1;
         const bool free_to_go = l <= last_removable;
-        remove_mlp[i] = (r1 && free_to_go && l % p->m == 0) ? 1 : 0;
-        remove_attn[i] = (remove_mlp[i] || (cs && free_to_go && C[i] >= p->alpha)) ? 1 : 0;
+        const bool every_mth = r1 && free_to_go && l % p->m == 0;
+        remove_attn[i] = (every_mth || (cs && free_to_go && C_attn[i] >= p->alpha)) ? 1 : 0;
+        remove_mlp[i] = (every_mth || (cs_mlp && free_to_go && C_mlp[i] >= p->alpha_mlp)) ? 1 : 0;
     }
     return ASD_OK;
+}
+
+extern "C" int asd_admg(const float* C, int32_t L, const asd_admg_params* p, uint8_t* remove_attn, uint8_t* remove_mlp) {
+    return asd_admg_ext(C, nullptr, L, p, remove_attn, remove_mlp);
 }
 
 // ---------------------------------------------------------------- life cycle
@@ -636,6 +671,8 @@ extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t byt
     x->kv_dim = cfg->n_kv_heads * cfg->head_dim;
     x->skip_attn.assign(cfg->n_layers, 0);
     x->skip_mlp.assign(cfg->n_layers, 0);
+    x->run_attn.assign(cfg->n_layers, 0.0);
+    x->run_mlp.assign(cfg->n_layers, 0.0);
     auto bail = [&](cudaError_t e) {
         fprintf(stderr, "asd_create: %s\n", cudaGetErrorString(e));
         if (x->pinned) cudaFreeHost(x->pinned);
@@ -651,7 +688,8 @@ extern "C" int asd_create(const asd_config* cfg, void* dev_workspace, size_t byt
             return ASD_ERR_ARG;
         }
     }
-    if ((e = cudaHostAlloc((void**)&x->pinned, 4096, cudaHostAllocDefault)) != cudaSuccess) return bail(e);
+    // 4 KB of token / status words, then room for the per-row cosines of one pass ([2][L][kPassMaxRows] floats)
+    if ((e = cudaHostAlloc((void**)&x->pinned, 4096 + (size_t)2 * std::max(cfg->n_layers, 1) * kPassMaxRows * 4, cudaHostAllocDefault)) != cudaSuccess) return bail(e);
     // rotary table: angle(p, j) = p * theta^(-2j/head_dim), evaluated in double, stored as float
     {
         const int half = cfg->head_dim / 2;
@@ -842,6 +880,9 @@ extern "C" int asd_reset(asd_ctx* x) {
     std::fill(x->skip_attn.begin(), x->skip_attn.end(), 0);
     std::fill(x->skip_mlp.begin(), x->skip_mlp.end(), 0);
     x->n_sim_rows = 0;
+    std::fill(x->run_attn.begin(), x->run_attn.end(), 0.0);
+    std::fill(x->run_mlp.begin(), x->run_mlp.end(), 0.0);
+    x->n_run_rows = 0;
     x->last_M = 0;
     x->stats = asd_stats{};
     x->spans.clear();
@@ -984,15 +1025,16 @@ extern "C" int asd_prefill(asd_ctx* x, const int32_t* tokens, int32_t n, int32_t
 
 extern "C" int asd_get_similarity(asd_ctx* x, float* c_attn, float* c_mlp, int32_t* n_rows) {
     if (!x) return ASD_ERR_ARG;
-    if (n_rows) *n_rows = (int32_t)x->n_sim_rows;
+    const int64_t rows = x->n_sim_rows + x->n_run_rows;
+    if (n_rows) *n_rows = (int32_t)rows;
     if (x->n_sim_rows == 0) return fail(x, ASD_ERR_STATE, "no prompt row has been processed");
     const int L = x->c.n_layers;
     std::vector<double> h(2 * (size_t)std::max(L, 1));
     ASD_CUDA(x, cudaMemcpyAsync(h.data(), x->ws + x->lay.sumcos, h.size() * 8, cudaMemcpyDeviceToHost, x->stream));
     ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     for (int l = 0; l < L; ++l) {
-        if (c_attn) c_attn[l] = (float)(h[l] / (double)x->n_sim_rows);
-        if (c_mlp) c_mlp[l] = (float)(h[L + l] / (double)x->n_sim_rows);
+        if (c_attn) c_attn[l] = (float)((h[l] + x->run_attn[l]) / (double)rows);
+        if (c_mlp) c_mlp[l] = (float)((h[L + l] + x->run_mlp[l]) / (double)rows);
     }
     return ASD_OK;
 }
@@ -1007,14 +1049,20 @@ extern "C" int asd_set_skip_mask(asd_ctx* x, const uint8_t* skip_attn, const uin
     return build_stage_tables(x);
 }
 
+extern "C" int asd_set_running_similarity(asd_ctx* x, int32_t on) {
+    if (!x) return ASD_ERR_ARG;
+    x->running_c = on != 0;
+    return ASD_OK;
+}
+
 extern "C" int asd_admg_update(asd_ctx* x, const asd_admg_params* p, uint8_t* skip_attn, uint8_t* skip_mlp) {
     if (!x || !p) return ASD_ERR_ARG;
     const int L = x->c.n_layers;
-    std::vector<float> C(std::max(L, 1));
-    int rc = asd_get_similarity(x, C.data(), nullptr, nullptr);
+    std::vector<float> C(std::max(L, 1)), Cm(std::max(L, 1));
+    int rc = asd_get_similarity(x, C.data(), Cm.data(), nullptr);
     if (rc) return rc;
     std::vector<uint8_t> a(std::max(L, 1)), b(std::max(L, 1));
-    rc = asd_admg(C.data(), L, p, a.data(), b.data());
+    rc = asd_admg_ext(C.data(), Cm.data(), L, p, a.data(), b.data());
     if (rc) return fail(x, rc, "bad ADMG parameters");
     rc = asd_set_skip_mask(x, a.data(), b.data());
     if (rc) return rc;
@@ -1050,7 +1098,9 @@ extern "C" int asd_decode_step(asd_ctx* x, int32_t token_in, int32_t* token_out)
     if (rc) return rc;
     rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, x->at<int>(x->lay.tok_in), false, nullptr, false);
     if (rc) return rc;
+    if ((rc = request_cosines(x))) return rc;
     if ((rc = read_back(x, x->at<int>(x->lay.argmax), 1))) return rc;
+    fold_committed_rows(x, 1);
     x->n_committed += 1;
     x->draft_cursor = x->n_committed;
     if (token_out) *token_out = x->pinned[0];
@@ -1080,8 +1130,10 @@ extern "C" int asd_verify(asd_ctx* x, const int32_t* tokens, int32_t k, int32_t*
     if (rc) return rc;
     rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, x->at<int>(x->lay.draft_toks), false, nullptr, true);
     if (rc) return rc;
+    if ((rc = request_cosines(x))) return rc;
     if ((rc = read_back(x, x->at<int>(x->lay.accept), k + 2))) return rc;
     const int a = x->pinned[0];
+    fold_committed_rows(x, a + 1);
     if (n_accepted) *n_accepted = a;
     if (out_tokens)
         for (int j = 0; j <= a; ++j) out_tokens[j] = x->pinned[1 + j];
@@ -1104,6 +1156,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
     int rc = asd_reset(x);
     if (rc) return rc;
     if (gp->mode == ASD_MODE_SPEC_MANUAL_MASK) asd_set_skip_mask(x, ka.data(), km.data());
+    x->running_c = (gp->admg.flags & ASD_RUNNING_C) != 0;
     cudaStream_t s = x->stream;
     size_t ev_begin, ev_end;
     if ((rc = new_event(x, &ev_begin))) return rc;
@@ -1131,9 +1184,11 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, dev_out + produced - 1, false, dev_out + produced, false);
             if (rc) return rc;
             x->n_committed += 1;
-            if (need_host_token) {
+            if (need_host_token || x->running_c) {  // running similarities: one host read-back per step
+                if ((rc = request_cosines(x))) return rc;
                 if ((rc = read_back(x, dev_out + produced, 1))) return rc;
-                stop = x->pinned[0] == gp->eos_id;
+                fold_committed_rows(x, 1);
+                stop = need_host_token && x->pinned[0] == gp->eos_id;
             }
             ++produced;
         }
@@ -1151,8 +1206,10 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             }
             rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, draft, false, nullptr, true);
             if (rc) return rc;
+            if ((rc = request_cosines(x))) return rc;
             if ((rc = read_back(x, accept, k + 2))) return rc;
             const int a = x->pinned[0];
+            fold_committed_rows(x, a + 1);
             int emit = a + 1;
             if (gp->eos_id >= 0)
                 for (int j = 0; j <= a; ++j)
@@ -1170,6 +1227,12 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             x->stats.rounds += 1;
             x->stats.drafted += k;
             x->stats.accepted += a;
+            // running similarities: Algorithm 1 again on the refreshed C_l every `refresh` rounds (the draft cursor is
+            // at the committed length here, so the new mask takes effect with the next round's first draft step)
+            if (gp->mode == ASD_MODE_SPEC && x->running_c && gp->admg.refresh > 0 && x->stats.rounds % gp->admg.refresh == 0) {
+                rc = asd_admg_update(x, &gp->admg, nullptr, nullptr);
+                if (rc) return rc;
+            }
         }
     }
     if ((rc = new_event(x, &ev_end))) return rc;

@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
     ap.add_argument("--draft-len", type=int, default=4)
-    ap.add_argument("--alpha", type=float, default=0.9995)
+    ap.add_argument("--alpha", type=float, default=0.9997)
     ap.add_argument("--m", type=int, default=3)
     ap.add_argument("--n", type=int, default=2)
     ap.add_argument("--flags", type=int, default=5, help="ADMG rule subset: 1=CS thresholding, 2=rule 1, 4=rule 2")

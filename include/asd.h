@@ -98,6 +98,11 @@ typedef struct {
     int32_t mode, draft_len, max_new;
     int32_t eos_id; /* -1 = none */
     asd_admg_params admg;
+    /* Draft exiting (Section 4 takes the mechanism from Draft & Verify without restating it; this is its fixed-threshold
+     * form): a round stops drafting after the first draft token whose confidence in the draft model D, measured as
+     * the gap between D's largest and second-largest logit, is below this value; that token is still verified.
+     * 0 = off (every round drafts draft_len tokens). Costs one host read-back per draft step. */
+    float draft_exit_margin;
 } asd_gen_params;
 
 /* Counters and device times (CUDA events) accumulated since the last asd_reset / asd_generate start.
@@ -190,6 +195,9 @@ int asd_set_prefill_mode(asd_ctx* ctx, int32_t mode);
 /* Per-row results of the last pass of M rows: cosines [L][M] (NaN where the sublayer was skipped),
  * argmax [M]. *M receives the row count. Any output may be NULL. */
 int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_mlp);
+/* Top-2 logit gap (largest minus second-largest logit; 0 when two tokens tie) of every row of the last pass that
+ * ran the LM head, margins[M]. margins may be NULL to query M. Errors: STATE if no such pass has run. */
+int asd_get_last_margins(asd_ctx* ctx, int32_t* M, float* margins);
 /* Logits [M][vocab] of the last pass; only recorded while bit 0 of asd_set_debug's flags is set. */
 int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
 /* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline. */

@@ -49,7 +49,7 @@ class AdmgParams(ctypes.Structure):
 
 class GenParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("draft_len", ctypes.c_int32), ("max_new", ctypes.c_int32),
-                ("eos_id", ctypes.c_int32), ("admg", AdmgParams)]
+                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float)]
 
 
 class Stats(ctypes.Structure):
@@ -241,10 +241,10 @@ class Oracle:
         return a.value, out[: a.value + 1].copy()
 
     def generate(self, prompt, max_new: int, mode: int = MODE_AR, draft_len: int = 4, alpha=0.985, m=3, n=2,
-                 flags=ADMG_ALL, eos_id: int = -1, alpha_mlp=1.0, refresh=0):
+                 flags=ADMG_ALL, eos_id: int = -1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
         """Returns (tokens, margins, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh))
+        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin)
         out = np.zeros(max_new, np.int32)
         margins = np.zeros(max_new, np.float32)
         n_out = ctypes.c_int32()

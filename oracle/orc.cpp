@@ -116,7 +116,7 @@ typedef struct {  // bf16 bit patterns, row-major [out,in], stacked over layers;
 } orc_weights;
 
 typedef struct { float alpha; int32_t m, n; uint32_t flags; float alpha_mlp; int32_t refresh; } orc_admg_params;
-typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; } orc_gen_params;
+typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; float draft_exit_margin; } orc_gen_params;
 typedef struct {
     int64_t full_passes, draft_passes, verify_passes, rounds, drafted, accepted, prefill_rows;
     double ms_prefill, ms_full, ms_draft, ms_verify, ms_total;
@@ -587,6 +587,9 @@ int orc_generate(orc_ctx* x, const int32_t* prompt, int32_t n_prompt, const orc_
         for (int j = 0; j < k; ++j) {
             rc = orc_draft_step(x, row[j], &row[j + 1]);
             if (rc) return rc;
+            // draft exiting (fixed-threshold form of the mechanism Section 4 takes from Draft & Verify): the first draft
+            // token whose top-2 logit gap in D is below the threshold ends the run; it is still verified
+            if (gp->draft_exit_margin > 0.f && j + 1 < k && x->last_margin[0] < gp->draft_exit_margin) k = j + 1;
         }
         int32_t a = 0;
         rc = orc_verify(x, row.data(), k, &a, acc.data());

@@ -34,7 +34,7 @@ class AdmgParams(ctypes.Structure):
 
 class GenParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("draft_len", ctypes.c_int32), ("max_new", ctypes.c_int32),
-                ("eos_id", ctypes.c_int32), ("admg", AdmgParams)]
+                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float)]
 
 
 class Stats(ctypes.Structure):
@@ -53,7 +53,7 @@ EXPORTS = (
     "asd_workspace_bytes", "asd_create", "asd_destroy", "asd_last_error", "asd_load_weights_host",
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
-    "asd_get_last_cosines", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
+    "asd_get_last_cosines", "asd_get_last_margins", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
     "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_admg_ext", "asd_set_running_similarity", "asd_set_prefill_mode", "asd_gemm_bf16",
 )
 
@@ -307,14 +307,14 @@ class Decoder:
         self._check(lib().asd_verify(self._ctx, _vp(t), ctypes.c_int32(k), ctypes.byref(a), _vp(out)), "asd_verify")
         return a.value, out[: a.value + 1].copy()
 
-    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp=1.0, refresh=0):
-        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh))
+    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
+        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin)
 
     def generate(self, prompt, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2, flags=ADMG_ALL, eos_id=-1,
-                 alpha_mlp=1.0, refresh=0):
+                 alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
         """Host buffers in, host buffers out. Returns (tokens, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin)
         out = np.zeros(max_new, np.int32)
         n_out = ctypes.c_int32()
         st = Stats()
@@ -323,9 +323,9 @@ class Decoder:
         return out[: n_out.value].copy(), st.as_dict()
 
     def generate_device(self, dev_prompt, dev_out, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2,
-                        flags=ADMG_ALL, eos_id=-1, alpha_mlp=1.0, refresh=0):
+                        flags=ADMG_ALL, eos_id=-1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
         """Prompt and output are int32 CUDA tensors. Returns (n_out, stats dict)."""
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin)
         n_out = ctypes.c_int32()
         st = Stats()
         self._check(lib().asd_generate_device(self._ctx, _vp(dev_prompt), ctypes.c_int32(dev_prompt.numel()),
@@ -341,6 +341,13 @@ class Decoder:
         ca, cm = np.empty((L, M.value), np.float32), np.empty((L, M.value), np.float32)
         self._check(lib().asd_get_last_cosines(self._ctx, ctypes.byref(M), _vp(ca), _vp(cm)), "asd_get_last_cosines")
         return ca, cm
+
+    def get_last_margins(self):
+        M = ctypes.c_int32()
+        self._check(lib().asd_get_last_margins(self._ctx, ctypes.byref(M), None), "asd_get_last_margins")
+        out = np.empty(M.value, np.float32)
+        self._check(lib().asd_get_last_margins(self._ctx, ctypes.byref(M), _vp(out)), "asd_get_last_margins")
+        return out
 
     def get_last_logits(self):
         M = ctypes.c_int32()

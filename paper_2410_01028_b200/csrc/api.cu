@@ -302,7 +302,7 @@ struct asd_ctx {
     std::vector<double> run_attn, run_mlp;
     int64_t n_run_rows = 0;
     int last_M = 0;
-    bool debug_logits = false, last_has_logits = false, trace = false;
+    bool debug_logits = false, last_has_logits = false, last_had_lm_head = false, trace = false;
     int last_n_stages = 0;
     int prefill_mode = ASD_PREFILL_AUTO;
     // tensor maps of the dense prompt path (host copies, passed to the kernels by value): activations with boxes of
@@ -559,6 +559,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.n_stages = lm_head ? n_table : n_table - 1;
     p.row_tokens = accept ? dev_tokens : nullptr;
     p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
+    p.margin_out = reinterpret_cast<float*>(x->at<int>(ly.argmax) + 32);  // second half of the argmax block
     p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
     p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
     p.acc_sim = acc_sim ? 1 : 0;
@@ -582,6 +583,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     }
     if (lm_head) bytes += 2.0 * (double)c.vocab * d;
     x->last_has_logits = lm_head && x->debug_logits;
+    x->last_had_lm_head = lm_head;
     x->last_M = M;
     if (bytes_out) *bytes_out = bytes;
     return ASD_OK;
@@ -1203,6 +1205,14 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             for (int j = 0; j < k; ++j) {  // k steps of the draft model, chained on the device
                 rc = timed_pass(x, SPAN_DRAFT, 1, x->n_committed + j, draft + j, true, draft + j + 1, false);
                 if (rc) return rc;
+                // draft exiting: a draft token whose top-2 logit margin in D falls below the threshold ends the run
+                // (the token itself is still verified); costs one host read-back per draft step
+                if (gp->draft_exit_margin > 0.f && j + 1 < k) {
+                    if ((rc = read_back(x, x->at<int>(x->lay.argmax) + 32, 1))) return rc;
+                    float mg;
+                    memcpy(&mg, x->pinned, 4);
+                    if (mg < gp->draft_exit_margin) k = j + 1;
+                }
             }
             rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, draft, false, nullptr, true);
             if (rc) return rc;
@@ -1318,6 +1328,17 @@ extern "C" int asd_get_last_logits(asd_ctx* x, int32_t* M, float* logits) {
     if (M) *M = x->last_M;
     if (logits) {
         ASD_CUDA(x, cudaMemcpyAsync(logits, x->ws + x->lay.logits, (size_t)x->last_M * x->c.vocab * 4, cudaMemcpyDeviceToHost, x->stream));
+        ASD_CUDA(x, cudaStreamSynchronize(x->stream));
+    }
+    return ASD_OK;
+}
+
+extern "C" int asd_get_last_margins(asd_ctx* x, int32_t* M, float* margins) {
+    if (!x) return ASD_ERR_ARG;
+    if (x->last_M == 0 || !x->last_had_lm_head) return fail(x, ASD_ERR_STATE, "no pass with an LM head has run");
+    if (M) *M = x->last_M;
+    if (margins) {
+        ASD_CUDA(x, cudaMemcpyAsync(margins, x->at<int>(x->lay.argmax) + 32, (size_t)x->last_M * 4, cudaMemcpyDeviceToHost, x->stream));
         ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     }
     return ASD_OK;

@@ -89,6 +89,7 @@ struct PassParams {
     int n_stages;
     const int* row_tokens;
     int* argmax_out;
+    float* margin_out;  // [M] top-1 minus top-2 logit of every row (the confidence that ends a draft run early), or null
     int* accept_out;
     float* logits_out;
     int acc_sim;
@@ -438,6 +439,15 @@ __device__ __forceinline__ void stage_begin(const PassParams& p, int s) {
     trace_mark(p, s, 1);
 }
 
+// LM head: (largest logit, its lowest index, second-largest logit) of two disjoint index sets combined
+__device__ __forceinline__ void top2_merge(float& v, int& i, float& s, float ov, int oi, float os) {
+    s = fmaxf(fminf(v, ov), fmaxf(s, os));
+    if (ov > v || (ov == v && oi < i)) {
+        v = ov;
+        i = oi;
+    }
+}
+
 // ============================================================================================ GEMV stage
 template <int M>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
@@ -726,12 +736,12 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
     float s_loc[M][3];
-    float best_v[M];
+    float best_v[M], sec_v[M];
     int best_i[M];
 #pragma unroll
     for (int m = 0; m < M; ++m) {
         s_loc[m][0] = s_loc[m][1] = s_loc[m][2] = 0.f;
-        best_v[m] = -INFINITY;
+        best_v[m] = sec_v[m] = -INFINITY;
         best_i[m] = INT_MAX;
     }
     const bool resid = (type == kStOproj || type == kStDown);
@@ -807,13 +817,21 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     p.logits_out[(size_t)m * n_rows + ra] = va;
                     if (has_b) p.logits_out[(size_t)m * n_rows + rb] = vb;
                 }
-                if (va > best_v[m]) {
+                if (va > best_v[m]) {  // rows come in ascending order: an equal logit keeps the lower index
+                    sec_v[m] = best_v[m];
                     best_v[m] = va;
                     best_i[m] = ra;
+                } else {
+                    sec_v[m] = fmaxf(sec_v[m], va);
                 }
-                if (has_b && vb > best_v[m]) {
-                    best_v[m] = vb;
-                    best_i[m] = rb;
+                if (has_b) {
+                    if (vb > best_v[m]) {
+                        sec_v[m] = best_v[m];
+                        best_v[m] = vb;
+                        best_i[m] = rb;
+                    } else {
+                        sec_v[m] = fmaxf(sec_v[m], vb);
+                    }
                 }
             }
         }
@@ -840,64 +858,54 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     } else if (type == kStLmHead) {
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-            float v = best_v[m];
+            float v = best_v[m], sc = sec_v[m];
             int i = best_i[m];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 const float ov = __shfl_xor_sync(0xffffffffu, v, o);
                 const int oi = __shfl_xor_sync(0xffffffffu, i, o);
-                if (ov > v || (ov == v && oi < i)) {
-                    v = ov;
-                    i = oi;
-                }
+                const float os = __shfl_xor_sync(0xffffffffu, sc, o);
+                top2_merge(v, i, sc, ov, oi, os);
             }
             if (lane == 0) {
                 red[warp * (kPassMaxRows * 4) + m * 4 + 0] = v;
                 red[warp * (kPassMaxRows * 4) + m * 4 + 1] = __int_as_float(i);
+                red[warp * (kPassMaxRows * 4) + m * 4 + 2] = sc;
             }
         }
         consumers_sync();
         if (tid < M) {
-            float v = -INFINITY;
+            float v = -INFINITY, sc = -INFINITY;
             int i = INT_MAX;
-            for (int w = 0; w < kPassConsumerWarps; ++w) {
-                const float ov = red[w * (kPassMaxRows * 4) + tid * 4 + 0];
-                const int oi = __float_as_int(red[w * (kPassMaxRows * 4) + tid * 4 + 1]);
-                if (ov > v || (ov == v && oi < i)) {
-                    v = ov;
-                    i = oi;
-                }
-            }
+            for (int w = 0; w < kPassConsumerWarps; ++w)
+                top2_merge(v, i, sc, red[w * (kPassMaxRows * 4) + tid * 4 + 0], __float_as_int(red[w * (kPassMaxRows * 4) + tid * 4 + 1]),
+                           red[w * (kPassMaxRows * 4) + tid * 4 + 2]);
             float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kPassMaxRows * 4;
             lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 0] = v;
             lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 1] = __int_as_float(i);
+            lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 2] = sc;
         }
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
             int* g = reinterpret_cast<int*>(red);
             for (int m = warp; m < M; m += kPassConsumerWarps) {  // a warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index
-                float v = -INFINITY;
+                float v = -INFINITY, sc = -INFINITY;
                 int i = INT_MAX;
                 const float* lmp = p.partials + (size_t)p.n_resid * gridDim.x * kPassMaxRows * 4;
                 for (unsigned b = lane; b < gridDim.x; b += 32) {
-                    const float ov = __ldcg(lmp + ((size_t)b * kPassMaxRows + m) * 4 + 0);
-                    const int oi = __float_as_int(__ldcg(lmp + ((size_t)b * kPassMaxRows + m) * 4 + 1));
-                    if (ov > v || (ov == v && oi < i)) {
-                        v = ov;
-                        i = oi;
-                    }
+                    const float4 o4 = __ldcg(reinterpret_cast<const float4*>(lmp + ((size_t)b * kPassMaxRows + m) * 4));
+                    top2_merge(v, i, sc, o4.x, __float_as_int(o4.y), o4.z);
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
                     const float ov = __shfl_xor_sync(0xffffffffu, v, o);
                     const int oi = __shfl_xor_sync(0xffffffffu, i, o);
-                    if (ov > v || (ov == v && oi < i)) {
-                        v = ov;
-                        i = oi;
-                    }
+                    const float os = __shfl_xor_sync(0xffffffffu, sc, o);
+                    top2_merge(v, i, sc, ov, oi, os);
                 }
                 if (lane == 0) {
                     if (i == INT_MAX) i = 0;
                     p.argmax_out[m] = i;
+                    if (p.margin_out) p.margin_out[m] = v - sc;
                     g[m] = i;
                 }
             }

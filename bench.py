@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--m", type=int, default=3)
     ap.add_argument("--n", type=int, default=2)
     ap.add_argument("--flags", type=int, default=5, help="ADMG rule subset: 1=CS thresholding, 2=rule 1, 4=rule 2")
+    ap.add_argument("--draft-exit", type=float, default=0.1, help="draft exiting: stop a round's drafting below this top-2 "
+                    "logit gap of the draft model (0 = every round drafts --draft-len tokens)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemv-microbench", action="store_true", help="also time the stand-alone fused GEMV kernel")
     ap.add_argument("--ablation", action="store_true", help="also time the rule subsets of the paper's ablation (Table 5) and "
@@ -179,7 +181,7 @@ def workload(args):
 
 
 def admg_kwargs(a):
-    return dict(draft_len=a.draft_len, alpha=a.alpha, m=a.m, n=a.n, flags=a.flags)
+    return dict(draft_len=a.draft_len, alpha=a.alpha, m=a.m, n=a.n, flags=a.flags, draft_exit_margin=a.draft_exit)
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle legs
@@ -320,7 +322,7 @@ def ablation(torch, asd, dec, dev_prompt, dev_out, new, args, ar_tokens):
     out = []
     for name, flags in rows:
         kw = dict(draft_len=args.draft_len, alpha=args.alpha, m=args.m, n=args.n, flags=flags, alpha_mlp=args.alpha_mlp,
-                  refresh=args.refresh if flags & asd.RUNNING_C else 0)
+                  refresh=args.refresh if flags & asd.RUNNING_C else 0, draft_exit_margin=args.draft_exit)
         dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)  # warm-up
         _, st = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
         same = bool((dev_out.cpu().numpy() == ar_tokens).all())
@@ -418,7 +420,8 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_s = max_over_ranks(time.perf_counter() - t0, world, "cuda")
     e2e = {"value": whole_job_value(world, args.steps, new, e2e_s * 1e3), "unit": UNIT, "h2d_bytes_per_step": int(prompt.nbytes),
-           "d2h_bytes_per_step": int(toks.nbytes) + 4 * int(agg["rounds"] // args.steps) * (args.draft_len + 2)}
+           "d2h_bytes_per_step": int(toks.nbytes) + 4 * int(agg["rounds"] // args.steps) * (args.draft_len + 2)
+                                 + (4 * int(agg["draft_passes"] // args.steps) if args.draft_exit > 0 else 0)}
 
     if rank != 0:
         return

@@ -157,6 +157,29 @@ def test_gpu_mlp_threshold_equals_oracle():
 
 
 @pytest.mark.gpu
+def test_gpu_error_paths_of_the_extension_calls(tiny_model):
+    import ctypes
+    import paper_2410_01028_b200 as asd
+    from paper_2410_01028_b200 import binding
+    L = 4
+    ca = np.full(L, 0.5, np.float32)
+    ra, rm = np.zeros(L, np.uint8), np.zeros(L, np.uint8)
+    p = binding.AdmgParams(0.9, 0, 0, asd.USE_CS_MLP, 0.9, 0)
+    vp = lambda a: ctypes.c_void_p(a.ctypes.data)
+    # the MLP threshold needs the MLP similarities
+    assert asd.lib().asd_admg_ext(vp(ca), None, ctypes.c_int32(L), ctypes.byref(p), vp(ra), vp(rm)) == binding.ERR_ARG
+    assert asd.lib().asd_admg(vp(ca), ctypes.c_int32(L), ctypes.byref(p), vp(ra), vp(rm)) == binding.ERR_ARG
+    p.flags = asd.USE_CS  # without the flag they may be absent
+    assert asd.lib().asd_admg_ext(vp(ca), None, ctypes.c_int32(L), ctypes.byref(p), vp(ra), vp(rm)) == 0
+    assert asd.lib().asd_set_running_similarity(None, ctypes.c_int32(1)) == binding.ERR_ARG
+    dec = asd.Decoder(synth.TINY, max_seq=64, max_draft=8)
+    dec.load_weights_host(tiny_model)
+    with pytest.raises(asd.AsdError):  # no pass has run the LM head yet
+        dec.get_last_margins()
+    dec.close()
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("k,refresh", [(4, 0), (4, 2), (3, 1)])
 def test_gpu_running_similarity_and_refreshed_masks(tiny_model, tiny_prompt, k, refresh):
     import paper_2410_01028_b200 as asd

@@ -62,6 +62,8 @@ def parse_args():
                     "the two extensions (MLP similarity threshold, running similarities) end to end")
     ap.add_argument("--alpha-mlp", type=float, default=0.9995, help="MLP similarity threshold of the ablation's extension rows")
     ap.add_argument("--refresh", type=int, default=8, help="rounds between mask updates of the ablation's running-similarity row")
+    ap.add_argument("--gemv-shape", default="", help="time the stand-alone fused GEMV on one shape only: "
+                    "n_in,n_rows,rows,epilogue with epilogue one of plain, swiglu, residual (e.g. 4096,22016,1,swiglu)")
     ap.add_argument("--gemm-microbench", action="store_true", help="also time the stand-alone tensor-core GEMM of the prompt path")
     # reduced cases for profiler captures only (never for a reported number)
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
@@ -455,6 +457,10 @@ def run_ours(args):
                 "how": "CUDA events around every launch inside the timed region, on the launching stream"}
     if args.gemv_microbench:
         roofline["fused_gemv_alone"] = gemv_sweep(torch, asd, hbm_peak)
+    elif args.gemv_shape:
+        n_in, n_rows, rows, epi = args.gemv_shape.split(",")
+        epi = {"plain": asd.EPI_PLAIN, "swiglu": asd.EPI_SWIGLU, "residual": asd.EPI_RESIDUAL}[epi]
+        roofline["fused_gemv_alone"] = [gemv_roofline(torch, asd, int(n_in), int(n_rows), int(rows), epi, hbm_peak)]
     # the prompt pass is the tensor-core part of a step: dense products + causal attention, then one decode pass
     _, tf_sustained, tf_kind = tensor_peak()
     pf_ms = agg["ms_prefill"] / args.steps

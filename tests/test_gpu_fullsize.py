@@ -57,6 +57,11 @@ def test_full_width_verify_rows_match_oracle_and_decode():
         a_g, out_g = dec.verify(row)
         from helpers import assert_cos_close, assert_logits_close
         assert_logits_close(dec.get_last_logits(), orc.last()["logits"])
+        # top-2 logit gap of every row (what draft exiting looks at): exactly the gap of the logits the pass computed,
+        # across all CTAs' partial results, and the oracle's within the logit tolerance
+        gl = np.sort(dec.get_last_logits(), axis=-1)
+        np.testing.assert_array_equal(dec.get_last_margins(), gl[:, -1] - gl[:, -2])
+        assert np.all(np.abs(dec.get_last_margins() - m) <= 2 * 2e-2 * np.abs(orc.last()["logits"]).max(axis=-1))
         ca, cm = dec.get_last_cosines()
         assert_cos_close(ca, orc.last()["cos_attn"]); assert_cos_close(cm, orc.last()["cos_mlp"])
         if np.all(m > 1e-2):
@@ -92,7 +97,8 @@ def test_7b_shaped_model_properties_in_the_benchmark_configuration():
     ca, cm, n = dec.get_similarity()
     assert n == 512 and np.all(np.abs(ca) <= 1 + 1e-6) and np.all(np.abs(cm) <= 1 + 1e-6)
     assert ca[0] < 0.5 and np.median(ca) > 0.98          # the recipe's similarity profile (first layer far from 1)
-    for kw in (dict(alpha=0.9995, flags=asd.USE_CS | asd.USE_RULE2, draft_len=4),      # bench.py's default member
+    for kw in (dict(alpha=0.9997, flags=asd.USE_CS | asd.USE_RULE2, draft_len=4, draft_exit_margin=0.1),  # bench.py's default
+               dict(alpha=0.9995, flags=asd.USE_CS | asd.USE_RULE2, draft_len=4),
                dict(alpha=0.985, m=3, n=2, flags=asd.ADMG_ALL, draft_len=6)):           # Table 2's hyper-parameters
         sp, st = dec.generate(prompt, new, mode=asd.MODE_SPEC, **kw)
         assert sp.tolist() == ar.tolist()                 # lossless, bit for bit

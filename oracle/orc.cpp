@@ -75,28 +75,20 @@ inline float round_bf16(float f) {
 }
 
 // ---------------------------------------------------------------- dot product
-// sum_k w[k]*x[k], bf16 weights, float activations, double accumulation.
-// The product of two floats is exact in double, so the only rounding is in the
-// eight running sums (element k goes to sum k mod 8) and their final addition.
-__attribute__((target_clones("default", "arch=haswell", "arch=skylake-avx512")))
+// sum_k w[k]*x[k] in index order: bf16 weights, float activations, one double accumulator.
+// The product of two floats is exact in double, so the only rounding is in the running sum.
 double dot_bf16_f32(const uint16_t* w, const float* x, int64_t n) {
-    double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    int64_t k = 0;
-    for (; k + 8 <= n; k += 8)
-        for (int j = 0; j < 8; ++j) acc[j] += (double)bf16_bits_to_float(w[k + j]) * (double)x[k + j];
-    for (int j = 0; k < n; ++k, ++j) acc[j] += (double)bf16_bits_to_float(w[k]) * (double)x[k];
-    return ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+    double acc = 0;
+    for (int64_t k = 0; k < n; ++k) acc += (double)bf16_bits_to_float(w[k]) * (double)x[k];
+    return acc;
 }
 
 // out[m][r] = sum_k W[r][k] * x[m][k]     W: [n_out, n_in] bf16 row-major, x: [M, n_in]
+// (output rows are shared among threads; every element is one independent dot product)
 void matvec_rows(const uint16_t* W, int64_t n_out, int64_t n_in, const float* x, int M, double* out) {
-    const int MB = 32;  // rows of x handled per sweep over W (cache blocking only; each dot is independent)
-    for (int m0 = 0; m0 < M; m0 += MB) {
-        const int m1 = std::min(M, m0 + MB);
 #pragma omp parallel for schedule(static)
-        for (int64_t r = 0; r < n_out; ++r)
-            for (int m = m0; m < m1; ++m) out[(int64_t)m * n_out + r] = dot_bf16_f32(W + r * n_in, x + (int64_t)m * n_in, n_in);
-    }
+    for (int64_t r = 0; r < n_out; ++r)
+        for (int m = 0; m < M; ++m) out[(int64_t)m * n_out + r] = dot_bf16_f32(W + r * n_in, x + (int64_t)m * n_in, n_in);
 }
 
 }  // namespace

@@ -418,3 +418,73 @@ def test_error_codes(small):
     with pytest.raises(oracle.OracleError) as e:
         o.similarity()
     assert e.value.code == oracle.ERR_STATE
+
+
+# ------------------------------------------------------------------ the bf16 roundings inside a sublayer (R5, R7)
+# Both cases are built from one-hot embeddings (RMSNorm turns e_i into exactly 8 e_i at d = 64: 1/sqrt(1/64 + 1e-5)
+# = 7.9974, whose nearest bf16 value is 8) and a read-out row e_0 - e_1 in the output projection, so that the
+# sublayer's output is the DIFFERENCE of two intermediate values that agree after the rounding and differ by 0.25
+# before it. With the rounding the sublayer adds exactly nothing and its cosine is exactly 1; without it the
+# residual moves by 0.25 e_0 and the cosine is 1/sqrt(1 + 0.25^2).
+ONE_LAYER = synth.DecoderShape(n_layers=1, d_model=64, n_heads=4, head_dim=16, d_ffn=96, vocab=50)
+
+
+def _blank_one_layer_model():
+    s = ONE_LAYER
+    d, f, V = s.d_model, s.d_ffn, s.vocab
+    z = lambda *shape: np.zeros(shape, np.float32)
+    embed, lm = z(V, d), z(V, d)
+    embed[0, 0] = embed[1, 1] = 1.0          # token 0 -> e_0, token 1 -> e_1
+    lm[0, 0] = lm[1, 1] = 1.0                # logit 0 reads element 0 of the final normalised state, logit 1 element 1
+    ones = np.ones(d, np.float32)
+    return dict(embed=embed, lm_head=lm, final_norm=ones, attn_norm=ones[None].copy(), wq=z(1, d, d), wk=z(1, d, d),
+                wv=z(1, d, d), wo=z(1, d, d), mlp_norm=ones[None].copy(), wg=z(1, f, d), wu=z(1, f, d), wd=z(1, d, f))
+
+
+def _as_model(parts):
+    return synth.SynthModel(shape=ONE_LAYER, seed=0, **{k: bf(v) for k, v in parts.items()})
+
+
+def test_attention_output_is_rounded_to_bf16_before_the_output_projection():
+    # Wq = 0: uniform attention. Position 1 (token 1 after token 0) averages v_0 and v_1:
+    #   element 0: (256 + 1.5) / 2 = 128.75 -> bf16 129 (spacing 1 between 128 and 256);  element 1: (129 + 129) / 2 = 129
+    # W_o row 0 = e_0 - e_1: o_0 = 129 - 129 = 0 with the rounding R5, 128.75 - 129 = -0.25 without it.
+    p = _blank_one_layer_model()
+    p["wv"][0, 0, 0], p["wv"][0, 0, 1] = 32.0, 0.1875          # v[0] = 8 * 32 = 256 for token 0, 8 * 0.1875 = 1.5 for token 1
+    p["wv"][0, 1, 0] = p["wv"][0, 1, 1] = 16.125               # v[1] = 129 for both tokens
+    p["wo"][0, 0, 0], p["wo"][0, 0, 1] = 1.0, -1.0
+    o = oracle.Oracle(_as_model(p), max_seq=4)
+    o.prefill([0, 1])
+    np.testing.assert_array_equal(o.kv(0, 0)[1][:2], [256.0, 129.0])
+    np.testing.assert_array_equal(o.kv(0, 1)[1][:2], [1.5, 129.0])
+    last = o.last()
+    # position 0 attends to itself only: o_0 = 256 - 129 = 127 on top of x = e_0 -> y = 128 e_0, still parallel to x
+    assert last["cos_attn"][0, 0] == 1.0
+    # position 1: the rounded average makes o vanish, y = x = e_1 exactly
+    assert last["cos_attn"][0, 1] == 1.0
+    assert last["logits"][1, 0] == 0.0 and last["logits"][1, 1] == 8.0
+    # the same case without any bf16 rounding: y = e_1 - 0.25 e_0 (up to the un-rounded norm factor 7.9974 / 8)
+    u = oracle.Oracle(_as_model(p), max_seq=4, flags=oracle.FLAG_NO_ROUNDING)
+    u.prefill([0, 1])
+    assert u.last()["cos_attn"][0, 1] == pytest.approx(1 / math.sqrt(1 + 0.25 ** 2), abs=1e-4)
+    assert u.last()["logits"][1, 0] < -1.0
+
+
+def test_swiglu_product_is_rounded_to_bf16_before_the_down_projection():
+    # attention is the identity (W_o = 0); the MLP sees yn = 8 e_1 for token 1.
+    #   t_0 = silu(20) * 8.0625 = 161.25 -> bf16 161;  t_1 = silu(23) * 7 = 161   (silu(g) = g to float precision for g >= 20)
+    # W_d row 0 = e_0 - e_1: dn_0 = 161 - 161 = 0 with the rounding R7, 0.25 without it.
+    p = _blank_one_layer_model()
+    p["wg"][0, 0, 1], p["wu"][0, 0, 1] = 2.5, 1.0078125        # g_0 = 20, u_0 = 8.0625
+    p["wg"][0, 1, 1], p["wu"][0, 1, 1] = 2.875, 0.875          # g_1 = 23, u_1 = 7
+    p["wd"][0, 0, 0], p["wd"][0, 0, 1] = 1.0, -1.0
+    o = oracle.Oracle(_as_model(p), max_seq=4)
+    o.prefill([1])
+    last = o.last()
+    assert last["cos_attn"][0, 0] == 1.0
+    assert last["cos_mlp"][0, 0] == 1.0                         # z = y exactly
+    assert last["logits"][0, 0] == 0.0 and last["logits"][0, 1] == 8.0
+    u = oracle.Oracle(_as_model(p), max_seq=4, flags=oracle.FLAG_NO_ROUNDING)
+    u.prefill([1])
+    assert u.last()["cos_mlp"][0, 0] == pytest.approx(1 / math.sqrt(1 + 0.25 ** 2), abs=1e-4)
+    assert u.last()["logits"][0, 0] > 1.0

@@ -200,7 +200,17 @@ int asd_get_last_cosines(asd_ctx* ctx, int32_t* M, float* cos_attn, float* cos_m
 int asd_get_last_margins(asd_ctx* ctx, int32_t* M, float* margins);
 /* Logits [M][vocab] of the last pass; only recorded while bit 0 of asd_set_debug's flags is set. */
 int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
-/* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline. */
+/* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline.
+ * Two more bits exercise the error path of the bounded device waits without hanging anything.
+ * ASD_DEBUG_SHORT_WAITS: every wait of the pass kernel (ring slots, grid barrier) gives up after about a
+ * millisecond instead of about two seconds. ASD_DEBUG_MISSING_ARRIVAL: the grid barrier in front of the last
+ * stage of a pass waits for one arrival more than there are CTAs, so it can only end by its budget; the pass then
+ * still runs to its end, and the call that launched it returns ASD_ERR_DEVICE_TIMEOUT with the stage and the CTA in
+ * asd_last_error. The error stays set (every later pass returns it too) until asd_reset. */
+#define ASD_DEBUG_LOGITS 1
+#define ASD_DEBUG_TRACE 2
+#define ASD_DEBUG_SHORT_WAITS 4
+#define ASD_DEBUG_MISSING_ARRIVAL 8
 int asd_set_debug(asd_ctx* ctx, int32_t flags);
 /* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][12][n_ctas]. Entries 0-3 are device
  * timestamps in ns of every CTA: 0 = stage entered, 1 = inputs of the stage ready (previous stage finished on
@@ -260,7 +270,9 @@ int asd_fused_gemv(void* cuda_stream, int32_t M, int32_t n_in, int32_t n_rows, c
  *     with a long reduction dimension and many activation rows) is rejected with ASD_ERR_NOMEM and a message on
  *     stderr; use asd_fused_gemv with your own scratch for those.
  *   - The first call on each device looks up the array's device address (that device must be current) and
- *     configures the kernels; make that first call outside any stream capture.
+ *     configures the kernels; make that first call outside any stream capture. The address is kept per device
+ *     ordinal for the life of the process: it does not survive a cudaDeviceReset, after which this entry point
+ *     must not be used again in the same process. The set-up itself is serialised between host threads.
  *   - All calls on a device share the one array: two calls whose kernels can overlap on the GPU (different
  *     streams without ordering, or several host threads) race on it. Order them on one stream.
  *   - The call itself allocates nothing: no cudaMalloc, cudaFree or allocating library routine.

@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -19,6 +20,7 @@ namespace asd {
 constexpr int kPrefillRows = kPassMaxRows;  // prompt rows per pass of the chunked prefill
 constexpr size_t kAlign = 256;
 constexpr int kMaxGemvGrid = 1024;
+constexpr long long kShortWaitCycles = 2000000LL;  // ASD_DEBUG_SHORT_WAITS: about a millisecond per wait
 
 static size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
@@ -68,12 +70,14 @@ struct DeviceInfo {
     int num_sms = 0, max_smem = 0;
 };
 static DeviceInfo g_dev[64];
+static std::mutex g_dev_mutex;  // first calls from several host threads set the per-device records up one at a time
 
 static cudaError_t device_info(DeviceInfo** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     DeviceInfo& d = g_dev[dev];
     if (!d.ready) {
         if ((e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
@@ -303,6 +307,9 @@ struct asd_ctx {
     int64_t n_run_rows = 0;
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, last_had_lm_head = false, trace = false;
+    bool short_waits = false, inject_missing_arrival = false;  // test hooks of the bounded device waits (asd_set_debug)
+    bool dev_failed = false;     // a kernel gave up waiting: nothing more is launched until asd_reset
+    std::string dev_failed_msg;
     int last_n_stages = 0;
     int prefill_mode = ASD_PREFILL_AUTO;
     // tensor maps of the dense prompt path (host copies, passed to the kernels by value): activations with boxes of
@@ -519,6 +526,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     const Layout& ly = x->lay;
     const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
     cudaStream_t s = x->stream;
+    if (x->dev_failed) return fail(x, ASD_ERR_DEVICE_TIMEOUT, x->dev_failed_msg);  // the caches hold an abandoned pass
     if (M < 1 || (M > kMaxRows && M != kPassMaxRows)) return fail(x, ASD_ERR_ARG, "row count out of range");
     if ((long long)pos0 + M > c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "pass would exceed max_seq positions");
     PassPlan pl;
@@ -553,6 +561,8 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.grid_bar = words + 16;
     p.err = reinterpret_cast<int*>(words + 32);
     p.bar_base = x->bar_base;
+    p.wait_cycles = x->short_waits ? kShortWaitCycles : kWaitCycles;
+    p.bar_extra_last = x->inject_missing_arrival ? 1u : 0u;
     const int table = use_mask ? 1 : 0;
     p.stages = x->at<StageDesc>(ly.stage_tab) + (size_t)table * ly.max_stages;
     const int n_table = use_mask ? x->n_stages_draft : x->n_stages_full;
@@ -597,7 +607,9 @@ static int check_device_error(asd_ctx* x, const int32_t* w) {
     char buf[256];
     snprintf(buf, sizeof buf, "a kernel gave up waiting: %s (stage %d, item %d, slot %d, CTA %d, thread %d, tag %d, parity %d)",
              (w[0] >= 1 && w[0] <= 4) ? names[w[0]] : "unknown", w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
-    return fail(x, ASD_ERR_DEVICE_TIMEOUT, buf);
+    x->dev_failed = true;
+    x->dev_failed_msg = std::string(buf) + " (call asd_reset before going on)";
+    return fail(x, ASD_ERR_DEVICE_TIMEOUT, x->dev_failed_msg);
 }
 
 // copy n ints from the device and the pass kernel's error words to the pinned buffer, wait, and check them
@@ -886,6 +898,7 @@ extern "C" int asd_reset(asd_ctx* x) {
     std::fill(x->run_mlp.begin(), x->run_mlp.end(), 0.0);
     x->n_run_rows = 0;
     x->last_M = 0;
+    x->dev_failed = false;
     x->stats = asd_stats{};
     x->spans.clear();
     x->events_used = 0;
@@ -962,6 +975,7 @@ static int prefill_dense(asd_ctx* x, const int32_t* dev_tokens, int n, int pos0)
 
 static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int32_t* first_token, bool resolve) {
     if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
+    if (x->dev_failed) return fail(x, ASD_ERR_DEVICE_TIMEOUT, x->dev_failed_msg);
     if (n <= 0) return fail(x, ASD_ERR_ARG, "empty prompt");
     if ((long long)x->n_committed + n > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "prompt exceeds max_seq");
     size_t e0, e1;
@@ -1299,6 +1313,8 @@ extern "C" int asd_set_debug(asd_ctx* x, int32_t flags) {
     if (!x) return ASD_ERR_ARG;
     x->debug_logits = (flags & 1) != 0;
     x->trace = (flags & 2) != 0;
+    x->short_waits = (flags & ASD_DEBUG_SHORT_WAITS) != 0;
+    x->inject_missing_arrival = (flags & ASD_DEBUG_MISSING_ARRIVAL) != 0;
     return ASD_OK;
 }
 
@@ -1443,16 +1459,20 @@ extern "C" int asd_fused_gemv_static(void* cuda_stream, int32_t M, int32_t n_in,
     if (device_info(&dv) != cudaSuccess) return ASD_ERR_CUDA;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ASD_ERR_CUDA;
-    if (!g_static_scratch_addr[dev]) {  // first call on this device: resolve the array's device address
-        void* ptr = nullptr;
-        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-        if (e != cudaSuccess || !ptr) {
-            fprintf(stderr, "asd_fused_gemv_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
-            return ASD_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_dev_mutex);
+        if (!g_static_scratch_addr[dev]) {  // first call on this device: resolve the array's device address
+            void* ptr = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e != cudaSuccess || !ptr) {
+                fprintf(stderr, "asd_fused_gemv_static: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+                return ASD_ERR_CUDA;
+            }
+            g_static_scratch_addr[dev] = ptr;
         }
-        g_static_scratch_addr[dev] = ptr;
+        scratch = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
     }
-    unsigned char* scratch = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
     int grid, xin;
     size_t smem;
     if (!plan_gemv(*dv, M, n_rows, n_in, gain != nullptr, &grid, &xin, &smem)) return ASD_ERR_ARG;
@@ -1464,8 +1484,9 @@ extern "C" int asd_fused_gemv_static(void* cuda_stream, int32_t M, int32_t n_in,
         return ASD_ERR_NOMEM;
     }
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    // the array keeps whatever the previous call left: the arrival counter must start at zero
-    if (cudaMemsetAsync(scratch, 0, 256, s) != cudaSuccess) return ASD_ERR_CUDA;
+    // the array keeps whatever the previous call left: the arrival counter, which only the residual epilogue
+    // uses, must start at zero
+    if (epilogue == ASD_EPI_RESIDUAL && cudaMemsetAsync(scratch, 0, 256, s) != cudaSuccess) return ASD_ERR_CUDA;
     GemvParams p{};
     p.W = reinterpret_cast<const __nv_bfloat16*>(W);
     p.n_rows = n_rows;

@@ -13,7 +13,7 @@ constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kSeg = 1024;         // elements of the reduction dimension per warp work item
 constexpr int kAttnChunk = 128;    // keys per attention work item; chunks are aligned to absolute positions
 
-enum Epilogue : int { kEpiPlain = 0, kEpiSwiglu = 1, kEpiResidual = 2, kEpiQkv = 3, kEpiArgmax = 4 };
+enum Epilogue : int { kEpiPlain = 0, kEpiSwiglu = 1, kEpiResidual = 2 };
 
 // Parameter block of the fused RMSNorm -> GEMV -> epilogue kernel.
 struct GemvParams {
@@ -29,15 +29,6 @@ struct GemvParams {
     double* sumcos;   // residual: running sum over prompt rows, or null
     float* partials;  // [gridDim.x][kMaxRows][4] cross-CTA partial results
     unsigned* counter;  // zero before launch; reset by the last CTA
-    // qkv
-    __nv_bfloat16 *q_out, *k_cache, *v_cache;
-    const float *rope_cos, *rope_sin;
-    int pos0, d_model, kv_dim, head_dim;
-    // argmax
-    const int* row_tokens;  // tokens fed to the M rows (acceptance compares row_tokens[j+1] with argmax[j]); may be null
-    int* argmax_out;        // [M]
-    int* accept_out;        // [0] = a, [1 .. a+1] = accepted drafts then M's own token; may be null
-    float* logits_out;      // [M, n_rows] or null
 };
 
 struct PassParams;

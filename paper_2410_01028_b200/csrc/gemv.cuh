@@ -17,9 +17,6 @@
 //   residual : y = x + a in place; per-row <x,y>, |x|^2, |y|^2 by warp shuffles, one block-level finish per
 //              CTA, and the last CTA to arrive turns the per-CTA partials into the cosine similarity of the
 //              hidden state before and after the sublayer (summand of C_l, Section 3.2)
-//   qkv      : rotary embedding of q and k, bf16 rounding, K/V written straight into the cache
-//   argmax   : LM head; per-CTA (max, index) partials; the last CTA finishes the argmax of every row and
-//              the greedy acceptance of the drafted tokens (Section 1)
 #pragma once
 #include <limits.h>
 
@@ -31,36 +28,17 @@ struct WeightItem {
     uint4 a[4], b[4];
 };
 
-template <int EPI>
-__device__ __forceinline__ void pair_rows(const GemvParams& p, int pair, int& ra, int& rb) {
-    if (EPI == kEpiQkv) {
-        const int half = p.head_dim >> 1;
-        const int nq = p.d_model >> 1, nk = p.kv_dim >> 1;
-        int base, pp;
-        if (pair < nq) {
-            base = 0;
-            pp = pair;
-        } else if (pair < nq + nk) {
-            base = p.d_model;
-            pp = pair - nq;
-        } else {
-            base = p.d_model + p.kv_dim;
-            pp = pair - nq - nk;
-        }
-        const int head = pp / half, j = pp - head * half;
-        ra = base + head * p.head_dim + j;
-        rb = ra + half;
-    } else {
-        ra = 2 * pair;
-        rb = 2 * pair + 1;
-    }
+// the unit of work is a pair of neighbouring weight rows (gate_i and up_i for the SwiGLU epilogue)
+__device__ __forceinline__ void pair_rows(int pair, int& ra, int& rb) {
+    ra = 2 * pair;
+    rb = 2 * pair + 1;
 }
 
 template <int EPI>
 __device__ __forceinline__ void load_item(const GemvParams& p, int pair0, int n_seg, int it, int lane, WeightItem& w) {
     const int pl = it / n_seg, seg = it - pl * n_seg;
     int ra, rb;
-    pair_rows<EPI>(p, pair0 + pl, ra, rb);
+    pair_rows(pair0 + pl, ra, rb);
     rb = min(rb, p.n_rows - 1);  // an odd row count: the missing partner re-reads the last row and is discarded
     const __nv_bfloat16* Wa = p.W + (size_t)ra * p.n_in;
     const __nv_bfloat16* Wb = p.W + (size_t)rb * p.n_in;
@@ -231,17 +209,11 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvParams 
 
     // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
     float s_loc[M][3];
-    float best_v[M];
-    int best_i[M];
 #pragma unroll
-    for (int m = 0; m < M; ++m) {
-        s_loc[m][0] = s_loc[m][1] = s_loc[m][2] = 0.f;
-        best_v[m] = -INFINITY;
-        best_i[m] = INT_MAX;
-    }
+    for (int m = 0; m < M; ++m) s_loc[m][0] = s_loc[m][1] = s_loc[m][2] = 0.f;
     for (int pl = tid; pl < np; pl += kGemvThreads) {
         int ra, rb;
-        pair_rows<EPI>(p, pair0 + pl, ra, rb);
+        pair_rows(pair0 + pl, ra, rb);
         const bool has_b = rb < p.n_rows;
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -274,41 +246,6 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvParams 
                     s_loc[m][0] = fmaf(x1, y1, s_loc[m][0]);
                     s_loc[m][1] = fmaf(x1, x1, s_loc[m][1]);
                     s_loc[m][2] = fmaf(y1, y1, s_loc[m][2]);
-                }
-            } else if (EPI == kEpiQkv) {
-                const int pos = p.pos0 + m;
-                const int half = p.head_dim >> 1;
-                if (ra < p.d_model + p.kv_dim) {  // q or k: rotate the pair (j, j + head_dim/2) by pos * theta_j
-                    const int j = ra % p.head_dim;  // region bases are multiples of head_dim
-                    const float c = p.rope_cos[(size_t)pos * half + j], s = p.rope_sin[(size_t)pos * half + j];
-                    const float r0 = va * c - vb * s;
-                    const float r1 = vb * c + va * s;
-                    va = r0;
-                    vb = r1;
-                }
-                const __nv_bfloat16 ha = __float2bfloat16_rn(va), hb = __float2bfloat16_rn(vb);
-                if (ra < p.d_model) {
-                    p.q_out[(size_t)m * p.d_model + ra] = ha;
-                    p.q_out[(size_t)m * p.d_model + rb] = hb;
-                } else if (ra < p.d_model + p.kv_dim) {
-                    p.k_cache[(size_t)pos * p.kv_dim + (ra - p.d_model)] = ha;
-                    p.k_cache[(size_t)pos * p.kv_dim + (rb - p.d_model)] = hb;
-                } else {
-                    p.v_cache[(size_t)pos * p.kv_dim + (ra - p.d_model - p.kv_dim)] = ha;
-                    p.v_cache[(size_t)pos * p.kv_dim + (rb - p.d_model - p.kv_dim)] = hb;
-                }
-            } else if (EPI == kEpiArgmax) {
-                if (p.logits_out) {
-                    p.logits_out[(size_t)m * p.n_rows + ra] = va;
-                    if (has_b) p.logits_out[(size_t)m * p.n_rows + rb] = vb;
-                }
-                if (va > best_v[m]) {
-                    best_v[m] = va;
-                    best_i[m] = ra;
-                }
-                if (has_b && vb > best_v[m]) {
-                    best_v[m] = vb;
-                    best_i[m] = rb;
                 }
             }
         }
@@ -359,71 +296,6 @@ __global__ void __launch_bounds__(kGemvThreads, 1) gemv_kernel(const GemvParams 
                     double acc = *p.sumcos;
                     for (int m = 0; m < M; ++m) acc += (double)red[m];
                     *p.sumcos = acc;
-                }
-                *p.counter = 0u;
-            }
-        }
-    } else if (EPI == kEpiArgmax) {
-        // block-level argmax with ties resolved to the lowest index
-#pragma unroll
-        for (int m = 0; m < M; ++m) {
-            float v = best_v[m];
-            int i = best_i[m];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, i, o);
-                if (ov > v || (ov == v && oi < i)) {
-                    v = ov;
-                    i = oi;
-                }
-            }
-            if (lane == 0) {
-                red[warp * (kMaxRows * 4) + m * 4 + 0] = v;
-                red[warp * (kMaxRows * 4) + m * 4 + 1] = __int_as_float(i);
-            }
-        }
-        __syncthreads();
-        if (tid < M) {
-            float v = -INFINITY;
-            int i = INT_MAX;
-            for (int w = 0; w < kGemvWarps; ++w) {
-                const float ov = red[w * (kMaxRows * 4) + tid * 4 + 0];
-                const int oi = __float_as_int(red[w * (kMaxRows * 4) + tid * 4 + 1]);
-                if (ov > v || (ov == v && oi < i)) {
-                    v = ov;
-                    i = oi;
-                }
-            }
-            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 0] = v;
-            p.partials[((size_t)blockIdx.x * kMaxRows + tid) * 4 + 1] = __int_as_float(i);
-        }
-        if (last_cta_arrives(p.counter, flag)) {
-            int* g = reinterpret_cast<int*>(red);
-            if (tid < M) {
-                float v = -INFINITY;
-                int i = INT_MAX;
-                for (unsigned b = 0; b < gridDim.x; ++b) {
-                    const float ov = __ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 0);
-                    const int oi = __float_as_int(__ldcg(p.partials + ((size_t)b * kMaxRows + tid) * 4 + 1));
-                    if (ov > v || (ov == v && oi < i)) {
-                        v = ov;
-                        i = oi;
-                    }
-                }
-                if (i == INT_MAX) i = 0;
-                p.argmax_out[tid] = i;
-                g[tid] = i;
-            }
-            __syncthreads();
-            if (tid == 0) {
-                if (p.accept_out && p.row_tokens) {
-                    // greedy verification: drafted token j+1 is accepted while it equals M's argmax of row j
-                    int a = 0;
-                    while (a < M - 1 && p.row_tokens[a + 1] == g[a]) ++a;
-                    p.accept_out[0] = a;
-                    for (int j = 0; j < a; ++j) p.accept_out[1 + j] = p.row_tokens[j + 1];
-                    p.accept_out[1 + a] = g[a];
                 }
                 *p.counter = 0u;
             }

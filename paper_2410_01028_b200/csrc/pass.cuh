@@ -84,6 +84,8 @@ struct PassParams {
     unsigned* fin_counter;
     unsigned* grid_bar;
     unsigned bar_base;
+    unsigned bar_extra_last;  // test hook: arrivals the LAST stage's barrier waits for beyond the grid size (0 in normal use)
+    long long wait_cycles;    // cycle budget of every bounded wait of the pass
     int* err;
     const StageDesc* stages;
     int n_stages;
@@ -194,7 +196,7 @@ __device__ __forceinline__ bool ring_spin_consumed(const PassParams& p, const Pa
         if (sm.consumed[slot] >= gen) return true;
         if ((spin & 255u) != 0) continue;
         if (*err != kErrNone) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > p.wait_cycles) {
             if (atomicCAS(p.err, kErrNone, code) == kErrNone) {
                 p.err[1] = stage, p.err[2] = (int)g, p.err[3] = slot, p.err[4] = blockIdx.x, p.err[5] = threadIdx.x;
                 p.err[6] = tag, p.err[7] = -1;
@@ -210,7 +212,7 @@ __device__ __forceinline__ int ring_wait_full(const PassParams& p, const PassSme
     uint32_t gen;
     ring_locate(p, g, slot, gen);
     if (gen > 0 && !ring_spin_consumed(p, sm, slot, gen, kErrFullWait, stage, g, tag)) return slot;
-    mbar_wait(&sm.full[slot], gen & 1, p.err, kErrFullWait, stage, g, slot, tag);
+    mbar_wait(&sm.full[slot], gen & 1, p.err, kErrFullWait, stage, g, slot, tag, p.wait_cycles);
     return slot;
 }
 // consumer: one thread, after all readers of the slot are done (warp or group barrier before the call)
@@ -229,7 +231,7 @@ __device__ __forceinline__ int ring_acquire(const PassParams& p, const PassSmem&
     ring_locate(p, g, slot, gen);
     if (gen > 0) {
         if (!ring_spin_consumed(p, sm, slot, gen, kErrEmptyWait, stage, g, tag)) return slot;
-        mbar_wait(&sm.empty[slot], (gen - 1) & 1, p.err, kErrEmptyWait, stage, g, slot, tag);
+        mbar_wait(&sm.empty[slot], (gen - 1) & 1, p.err, kErrEmptyWait, stage, g, slot, tag, p.wait_cycles);
     }
     return slot;
 }
@@ -359,7 +361,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 if ((round & 255u) == 0) {  // the error word lives in global memory: look at it only now and then
                     if (*err != kErrNone) {
                         active = false;
-                    } else if (clock64() - t_progress > kWaitCycles) {
+                    } else if (clock64() - t_progress > p.wait_cycles) {
                         if (atomicCAS(p.err, kErrNone, kErrEmptyWait) == kErrNone) {
                             p.err[1] = c.s, p.err[2] = (int)g, p.err[3] = slot, p.err[4] = blockIdx.x, p.err[5] = threadIdx.x;
                             p.err[6] = M, p.err[7] = (int)((gen - 1) & 1);
@@ -406,7 +408,7 @@ __device__ __forceinline__ void grid_wait(const PassParams& p, unsigned target) 
         for (unsigned spin = 1; (int)(ld_acquire_gpu(p.grid_bar) - target) < 0; ++spin) {
             if ((spin & 63u) != 0) continue;
             if (*err != kErrNone) break;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > p.wait_cycles) {
                 if (atomicCAS(p.err, kErrNone, kErrGridWait) == kErrNone) {
                     p.err[1] = (int)((target - p.bar_base) / gridDim.x), p.err[2] = (int)ld_acquire_gpu(p.grid_bar);
                     p.err[3] = (int)target, p.err[4] = blockIdx.x;
@@ -435,7 +437,7 @@ __device__ __forceinline__ bool last_cta_consumers(unsigned* counter, int* flag_
 // Every stage starts by waiting for the previous stage of all CTAs. Whatever does not depend on activations (the
 // stage descriptor, index arithmetic, zeroing of partial sums, RMSNorm gains) is done before this wait.
 __device__ __forceinline__ void stage_begin(const PassParams& p, int s) {
-    if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x);
+    if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x + (s == p.n_stages - 1 ? p.bar_extra_last : 0u));
     trace_mark(p, s, 1);
 }
 

@@ -11,7 +11,7 @@
 namespace asd {
 
 constexpr int kSlotBytes = 8192;             // one ring slot: 8 weight rows x 512 bf16 inputs, or one 64-key K/V box
-constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
+constexpr long long kWaitCycles = 4000000000LL;  // default budget of one wait: ~2 s at 2 GHz
 
 enum DeviceError : int {
     kErrNone = 0,
@@ -47,14 +47,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Wait for a phase of an mbarrier. Returns false when the wait was abandoned (error word set).
 // The first wait to give up also records where it was: err[1..7] = stage, ring item, slot, CTA, thread, tag, parity.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err, int code, int stage = -1,
-                                          unsigned item = 0, int slot = -1, int tag = 0) {
+                                          unsigned item = 0, int slot = -1, int tag = 0, long long budget = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (unsigned spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 255u) != 0) continue;  // the error word lives in global memory: look at it only now and then
         if (*err != kErrNone) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > budget) {
             if (atomicCAS(const_cast<int*>(err), kErrNone, code) == kErrNone) {
                 err[1] = stage, err[2] = (int)item, err[3] = slot, err[4] = blockIdx.x, err[5] = threadIdx.x, err[6] = tag;
                 err[7] = (int)parity;

@@ -1,5 +1,11 @@
 """Comparison helpers shared by the GPU parity tests (tolerances of the parity contract)."""
+import collections
+
 import numpy as np
+
+# soft = token mismatches at steps whose top-2 logit gap in the oracle is at most MARGIN (allowed);
+# decided = steps whose gap exceeds MARGIN, where the GPU's token had to equal the oracle's (and did)
+Compare = collections.namedtuple("Compare", "soft decided")
 
 LOGIT_TOL = 2e-2     # |l_gpu - l_orc| <= LOGIT_TOL * max|l_orc| per row
 COS_TOL = 1e-3       # absolute, per sublayer and row
@@ -25,7 +31,8 @@ def teacher_forced_compare(dec, orc, prompt, max_new, check_logits=True):
     """Feed the oracle's greedy tokens through the GPU decoder step by step.
 
     At every step the GPU's argmax must equal the oracle's wherever the oracle's top-2 margin exceeds MARGIN;
-    logits and per-sublayer cosines are compared at every step.  Returns the number of low-margin mismatches.
+    logits and per-sublayer cosines are compared at every step.  Returns Compare(soft, decided); at least one step
+    must have been decided, so that the token comparison cannot pass vacuously.
     """
     ref, margins, _ = orc.generate(prompt, max_new)
     orc.reset()
@@ -34,12 +41,14 @@ def teacher_forced_compare(dec, orc, prompt, max_new, check_logits=True):
         dec.set_debug(True)
     t_o = orc.prefill(prompt)
     t_g = dec.prefill(prompt)
-    soft = 0
+    soft = decided = 0
 
     def check(tok_g, tok_o, margin, step):
-        nonlocal soft
-        if tok_g != tok_o:
-            assert margin <= MARGIN, f"token mismatch at step {step} with margin {margin}"
+        nonlocal soft, decided
+        if margin > MARGIN:
+            assert tok_g == tok_o, f"token mismatch at step {step} with margin {margin}"
+            decided += 1
+        elif tok_g != tok_o:
             soft += 1
 
     assert t_o == ref[0]
@@ -55,4 +64,31 @@ def teacher_forced_compare(dec, orc, prompt, max_new, check_logits=True):
         assert_cos_close(cm, last["cos_mlp"])
         if check_logits:
             assert_logits_close(dec.get_last_logits(), last["logits"])
-    return soft
+    assert decided > 0, "no step had a top-2 logit gap above the margin: the token comparison decided nothing"
+    return Compare(soft, decided)
+
+
+def verify_outcomes_agree(a_g, out_g, a_o, out_o, margins):
+    """Greedy acceptance of one verify pass, GPU against oracle.
+
+    The oracle's outcome (a_o accepted drafts, then M's own token) is decided by its rows 0..a_o. Where every one of
+    those rows has a top-2 logit gap above MARGIN the GPU must report the same acceptance and the same tokens; the
+    function then returns 1 (a decided comparison), otherwise 0.
+    """
+    if np.all(np.asarray(margins)[: a_o + 1] > MARGIN):
+        assert a_g == a_o and list(out_g) == list(out_o), (a_g, list(out_g), a_o, list(out_o))
+        return 1
+    return 0
+
+
+def argmax_rows_agree(gpu_logits, orc_last, rows=None):
+    """Token ids of the rows of one pass: the argmax of the GPU's logits must equal the oracle's argmax in every row
+    whose top-2 gap in the oracle exceeds MARGIN. Returns how many rows were decided that way."""
+    margin, am = np.asarray(orc_last["margin"]), np.asarray(orc_last["argmax"])
+    if rows is not None:
+        margin, am = margin[rows], am[rows]
+    got = np.argmax(gpu_logits, axis=-1)
+    assert got.shape == am.shape
+    decided = margin > MARGIN
+    assert np.array_equal(got[decided], am[decided]), (got, am, margin)
+    return int(decided.sum())

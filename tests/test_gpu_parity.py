@@ -6,7 +6,8 @@ import pytest
 
 import oracle
 import synth
-from helpers import COS_TOL, MARGIN, MASK_MARGIN, assert_cos_close, assert_logits_close, teacher_forced_compare
+from helpers import (COS_TOL, MARGIN, MASK_MARGIN, argmax_rows_agree, assert_cos_close, assert_logits_close,
+                     teacher_forced_compare, verify_outcomes_agree)
 
 pytestmark = pytest.mark.gpu
 
@@ -39,8 +40,6 @@ def test_tiny_prefill_similarity_logits_and_kv(tiny_pair, tiny_prompt):
     dec.set_debug(True)
     t_g, t_o = dec.prefill(tiny_prompt), orc.prefill(tiny_prompt)
     last = orc.last()
-    if last["margin"][-1] > MARGIN:
-        assert t_g == t_o
     ca_g, cm_g, n_g = dec.get_similarity()
     ca_o, cm_o, n_o = orc.similarity()
     assert n_g == n_o == 32
@@ -51,6 +50,9 @@ def test_tiny_prefill_similarity_logits_and_kv(tiny_pair, tiny_prompt):
     assert_cos_close(ca, last["cos_attn"][:, -rows:])
     assert_cos_close(cm, last["cos_mlp"][:, -rows:])
     assert_logits_close(dec.get_last_logits(), last["logits"][-rows:])
+    # token ids of those rows (the last one is t_1), wherever the oracle's top-2 gap decides them
+    assert argmax_rows_agree(dec.get_last_logits(), last, slice(-rows, None)) >= rows // 2
+    assert t_g == int(np.argmax(dec.get_last_logits()[-1]))
     # K/V cache, bf16. Layer 0 depends on the embedding, one RMSNorm and one product only: nearly every element is
     # identical, the rest are one-ulp rounding flips. Deeper layers inherit flips: one flipped element of K, V or of the
     # attention output moves the hidden state of every later row that attends to it by up to ~1e-3 of its scale and
@@ -69,8 +71,8 @@ def test_tiny_prefill_similarity_logits_and_kv(tiny_pair, tiny_prompt):
 
 def test_tiny_teacher_forced_decode(tiny_pair, tiny_prompt):
     dec, orc = tiny_pair
-    soft = teacher_forced_compare(dec, orc, tiny_prompt, 64)
-    assert soft <= 8
+    res = teacher_forced_compare(dec, orc, tiny_prompt, 64)
+    assert res.soft <= 8 and res.decided >= 32
 
 
 def test_tiny_generate_ar_spec_bit_exact_and_matches_oracle(tiny_pair, tiny_prompt):
@@ -81,7 +83,7 @@ def test_tiny_generate_ar_spec_bit_exact_and_matches_oracle(tiny_pair, tiny_prom
     assert st_ar["full_passes"] == 63
     # up to the first low-margin step the GPU must reproduce the oracle's tokens
     first_soft = next((i for i in range(64) if margins[i] <= MARGIN), 64)
-    assert ar[:first_soft].tolist() == ref[:first_soft].tolist()
+    assert first_soft >= 4 and ar[:first_soft].tolist() == ref[:first_soft].tolist()
     for (m, n) in [(3, 2), (2, 1), (1, 0)]:
         for k in (1, 4, 8):
             sp, st = dec.generate(tiny_prompt, 64, mode=asd.MODE_SPEC, draft_len=k, m=m, n=n)
@@ -112,6 +114,7 @@ def test_tiny_skip_masks_match_oracle(tiny_pair, tiny_prompt):
 
 def test_tiny_draft_and_verify_calls_match_oracle(tiny_pair, tiny_prompt):
     dec, orc = tiny_pair
+    decided_drafts = decided_verifies = 0
     for mask in ([0, 1, 0, 0], [0, 0, 1, 0]), ([1, 1, 1, 1], [1, 1, 1, 1]), ([0, 0, 0, 0], [0, 0, 0, 0]):
         dec.reset(); orc.reset()
         t = orc.prefill(tiny_prompt)
@@ -129,16 +132,17 @@ def test_tiny_draft_and_verify_calls_match_oracle(tiny_pair, tiny_prompt):
                     assert_cos_close(cm, orc.last()["cos_mlp"])
                     if m_o > MARGIN:
                         assert row_g[-1] == row_o[-1]
+                        decided_drafts += 1
             assert dec.positions() == orc.positions()
             a_o, out_o = orc.verify(row_o)
             margins = orc.last()["margin"]
             a_g, out_g = dec.verify(row_o)          # same drafted row into both
-            if np.all(margins > MARGIN):
-                assert a_g == a_o and out_g.tolist() == out_o.tolist()
+            decided_verifies += verify_outcomes_agree(a_g, out_g, a_o, out_o, margins)
             assert dec.positions()[0] == dec.positions()[1]
             if (a_g, out_g.tolist()) != (a_o, out_o.tolist()):
                 break
             t = int(out_o[-1])
+    assert decided_drafts >= 12 and decided_verifies >= 3     # the comparisons above did decide tokens
 
 
 # ------------------------------------------------------------------ other shapes: odd sizes, GQA, several tiles
@@ -312,3 +316,32 @@ def test_weights_from_file_equal_weights_from_host(tmp_path):
     with pytest.raises(asd.AsdError) as e:
         dec2.load_weights_file(str(path))
     assert e.value.code == -7
+
+
+def test_bounded_device_wait_runs_out_and_the_context_recovers(tiny_model, tiny_prompt):
+    """Every spin of the pass kernel has a cycle budget. Here the barrier in front of the last stage is told to wait
+    for one arrival that never comes, with the budget cut to about a millisecond: the pass must still end, the call
+    must report ASD_ERR_DEVICE_TIMEOUT with where it gave up, and after asd_reset the same context decodes as before."""
+    import paper_2410_01028_b200 as asd
+    dec = asd.Decoder(synth.TINY, max_seq=128, max_draft=8)
+    dec.load_weights_host(tiny_model)
+    want, _ = dec.generate(tiny_prompt, 24, mode=asd.MODE_AR)
+    dec.reset()
+    t = dec.prefill(tiny_prompt)
+    dec.set_debug(record_logits=False, short_waits=True)              # a short budget alone changes nothing
+    t2 = dec.decode_step(t)
+    assert t2 == want[1]
+    dec.set_debug(record_logits=False, short_waits=True, missing_arrival=True)
+    with pytest.raises(asd.AsdError) as e:
+        dec.decode_step(t2)
+    assert e.value.code == asd.binding.ERR_DEVICE_TIMEOUT
+    assert "grid barrier" in str(e.value) and "stage" in str(e.value)
+    with pytest.raises(asd.AsdError) as e:                           # the error is sticky until the context is reset
+        dec.set_debug(record_logits=False)
+        dec.decode_step(t2)
+    assert e.value.code == asd.binding.ERR_DEVICE_TIMEOUT
+    dec.reset()
+    got, _ = dec.generate(tiny_prompt, 24, mode=asd.MODE_AR)
+    assert got.tolist() == want.tolist()
+    sp, _ = dec.generate(tiny_prompt, 24, mode=asd.MODE_SPEC, draft_len=4, m=2, n=1)
+    assert sp.tolist() == want.tolist()

@@ -10,6 +10,7 @@ the first one left in the shared array).  It is collected last on purpose.
 import numpy as np
 import pytest
 
+import oracle
 import synth
 
 pytestmark = pytest.mark.gpu
@@ -49,6 +50,15 @@ def test_static_scratch_variant_matches_caller_scratch_variant_twice(M, n_in, n_
         assert float((got_t - want_t).abs().max()) <= 1e-5 * scale, call
         assert float((got_y - want_y).abs().max()) <= 1e-5 * max(scale, float(want_y.abs().max())), call
         assert float((got_cos - want_cos).abs().max()) <= 1e-5, call
+    # and directly against the CPU oracle (normalised input rounded to bf16 on both sides: a rounding flip moves one
+    # product by 2^-8, hence 2e-3 of the output scale; cosine within 1e-3)
+    xh, Wh, gh, rh = (x.cpu().numpy(), W.view(torch.int16).cpu().numpy().view(np.uint16),
+                      gain.view(torch.int16).cpu().numpy().view(np.uint16), res.cpu().numpy())
+    ref_t, _ = oracle.fused_matvec(xh, Wh, epilogue=0, gain=gh)
+    ref_y, ref_cos = oracle.fused_matvec(xh, Wh, epilogue=2, gain=gh, res=rh)
+    assert np.abs(got_t.cpu().numpy() - ref_t).max() <= 2e-3 * np.abs(ref_t).max()
+    assert np.abs(got_y.cpu().numpy() - ref_y).max() <= 2e-3 * np.abs(ref_y).max()
+    assert np.abs(got_cos.cpu().numpy() - ref_cos).max() <= 1e-3
 
 
 def test_static_scratch_variant_rejects_bad_arguments():

@@ -49,7 +49,8 @@ class AdmgParams(ctypes.Structure):
 
 class GenParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("draft_len", ctypes.c_int32), ("max_new", ctypes.c_int32),
-                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float)]
+                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float),
+                ("temperature", ctypes.c_float), ("seed", ctypes.c_uint64)]
 
 
 class Stats(ctypes.Structure):
@@ -71,6 +72,18 @@ def lib():
         L.orc_cosine.restype = ctypes.c_double
         L.orc_cosine.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]
         L.orc_last_error.restype = ctypes.c_char_p
+        L.orc_uniform.restype = ctypes.c_double
+        L.orc_uniform.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32]
+        L.orc_sample_cdf.restype = ctypes.c_int32
+        L.orc_sample_cdf.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_double]
+        L.orc_softmax_t.restype = None
+        L.orc_softmax_t.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p]
+        L.orc_spec_accept.restype = ctypes.c_int32
+        L.orc_spec_accept.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_uint64, ctypes.c_int32, ctypes.c_void_p]
+        L.orc_philox4x32_10.restype = None
+        L.orc_philox4x32_10.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.orc_set_sampling.argtypes = [ctypes.c_void_p, ctypes.c_float, ctypes.c_uint64]
         _lib = L
     return _lib
 
@@ -144,6 +157,49 @@ def fused_matvec(x, W, epilogue: int = 0, gain=None, eps: float = 1e-5, W2=None,
     return out, (cosv if epilogue == 2 else None)
 
 
+DRAW_DRAFT, DRAW_ACCEPT, DRAW_TARGET = 0, 1, 2
+
+
+def philox4x32_10(counter, key):
+    """The counter-based generator behind every random draw: four 32-bit words from a 128-bit counter and a 64-bit key."""
+    c = np.ascontiguousarray(counter, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.size == 4 and k.size == 2
+    out = np.zeros(4, np.uint32)
+    lib().orc_philox4x32_10(c.ctypes.data, k.ctypes.data, out.ctypes.data)
+    return out
+
+
+def uniform(seed: int, position: int, kind: int) -> float:
+    """The uniform number in (0, 1) of (seed, position of the token being chosen, kind of draw)."""
+    return float(lib().orc_uniform(seed, position, kind))
+
+
+def softmax_t(logits, T: float) -> np.ndarray:
+    l = _f32(logits)
+    out = np.empty(l.size, np.float64)
+    lib().orc_softmax_t(l.ctypes.data, l.size, float(T), out.ctypes.data)
+    return out
+
+
+def sample_cdf(w, u: float) -> int:
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    return int(lib().orc_sample_cdf(w.ctypes.data, w.size, float(u)))
+
+
+def spec_accept(p, q, drafts, seed: int, pos0: int):
+    """Sampling-based verification of k drafts: p [k+1, V], q [k, V] (float64), drafts [k]. Returns (a, tokens[a+1])."""
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    d = np.ascontiguousarray(drafts, dtype=np.int32)
+    k, V = d.size, p.shape[1]
+    assert p.shape == (k + 1, V) and (k == 0 or q.shape == (k, V))
+    out = np.zeros(k + 1, np.int32)
+    a = lib().orc_spec_accept(p.ctypes.data, q.ctypes.data if k else None, d.ctypes.data if k else None, k, V, seed, pos0,
+                              out.ctypes.data)
+    return int(a), out[: a + 1].copy()
+
+
 def num_threads() -> int:
     return int(lib().orc_num_threads())
 
@@ -210,6 +266,10 @@ class Oracle:
         _check(lib().orc_set_skip_mask(self._ctx, ctypes.c_void_p(a.ctypes.data), ctypes.c_void_p(b.ctypes.data)),
                "orc_set_skip_mask")
 
+    def set_sampling(self, temperature: float, seed: int = 0):
+        """temperature 0 = greedy (the default); above 0 every token is drawn, see ``orc_set_sampling``."""
+        _check(lib().orc_set_sampling(self._ctx, ctypes.c_float(temperature), ctypes.c_uint64(seed)), "orc_set_sampling")
+
     def set_running_similarity(self, on: bool):
         _check(lib().orc_set_running_similarity(self._ctx, ctypes.c_int32(1 if on else 0)), "orc_set_running_similarity")
 
@@ -241,10 +301,11 @@ class Oracle:
         return a.value, out[: a.value + 1].copy()
 
     def generate(self, prompt, max_new: int, mode: int = MODE_AR, draft_len: int = 4, alpha=0.985, m=3, n=2,
-                 flags=ADMG_ALL, eos_id: int = -1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
+                 flags=ADMG_ALL, eos_id: int = -1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0, temperature=0.0, seed=0):
         """Returns (tokens, margins, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin)
+        gp = GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin,
+                       temperature, seed)
         out = np.zeros(max_new, np.int32)
         margins = np.zeros(max_new, np.float32)
         n_out = ctypes.c_int32()

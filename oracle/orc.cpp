@@ -39,6 +39,17 @@
 // similarity (orc_admg_ext; pinned by brute force over all masks on L=2), and C_l kept running over the rows
 // committed after the prompt, with Algorithm 1 run again every few rounds (pinned: the running C_l after a
 // generation equals the C_l of one prefill over prompt + emitted tokens, for both decoding modes).
+//   * verification when sampling is used: drafted tokens are sampled from D's distribution q and accepted
+//     with probability min(1, p/q) under M's distribution p, a rejected token is resampled from the
+//     normalised max(0, p - q), so that every emitted token is distributed as if M had sampled it
+//                                                       -- Section 1 (third paragraph; the rule of the two
+//                                                          speculative-sampling papers cited there), used for
+//                                                          the T > 0 columns of Tables 3 and 4
+//     Random numbers come from one counter-based generator, Philox4x32-10 (Salmon et al., SC'11), keyed
+//     by the seed and indexed by (position of the token being chosen, kind of draw).  Pins: the generator's
+//     published known-answer vectors; softmax and inverse-CDF sampling against scipy / numpy; T -> 0 gives
+//     the greedy loop; q = p accepts everything; the emitted-token histogram over 10^5 rounds equals p for a
+//     deliberately wrong q (chi-square).
 // Parity unpinned: absolute token ids / logits of the random synthetic models
 // (the paper prints no worked example).
 #include <algorithm>
@@ -108,7 +119,7 @@ typedef struct {  // bf16 bit patterns, row-major [out,in], stacked over layers;
 } orc_weights;
 
 typedef struct { float alpha; int32_t m, n; uint32_t flags; float alpha_mlp; int32_t refresh; } orc_admg_params;
-typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; float draft_exit_margin; } orc_gen_params;
+typedef struct { int32_t mode, draft_len, max_new, eos_id; orc_admg_params admg; float draft_exit_margin; float temperature; uint64_t seed; } orc_gen_params;
 typedef struct {
     int64_t full_passes, draft_passes, verify_passes, rounds, drafted, accepted, prefill_rows;
     double ms_prefill, ms_full, ms_draft, ms_verify, ms_total;
@@ -169,6 +180,93 @@ int orc_admg_ext(const float* C_attn, const float* C_mlp, int32_t L, float alpha
     return ORC_OK;
 }
 
+// ---------------------------------------------------------------- random numbers (sampling-based verification)
+// Philox4x32-10: ten rounds of  (c0,c1,c2,c3) <- (hi(M1*c2) ^ c1 ^ k0, lo(M1*c2), hi(M0*c0) ^ c3 ^ k1, lo(M0*c0))
+// with the key bumped by the Weyl constants after every round (Salmon, Moraes, Dror, Shaw, SC'11).
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0, c1 = n1, c2 = n2, c3 = n3;
+        k0 += W0, k1 += W1;
+    }
+    out[0] = c0, out[1] = c1, out[2] = c2, out[3] = c3;
+}
+
+// kinds of draw at one position of the sequence
+enum { ORC_DRAW_DRAFT = 0, ORC_DRAW_ACCEPT = 1, ORC_DRAW_TARGET = 2 };
+
+// The uniform number in (0,1) for (seed, position of the token being chosen, kind of draw): first output word of
+// the generator with key = seed and counter = (position, kind, 0, 0), mapped to (x + 1/2) / 2^32.
+double orc_uniform(uint64_t seed, uint32_t position, uint32_t kind) {
+    const uint32_t ctr[4] = {position, kind, 0u, 0u}, key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return ((double)out[0] + 0.5) * (1.0 / 4294967296.0);
+}
+
+// p_i = exp(l_i / T) / sum_j exp(l_j / T), evaluated with the maximum subtracted
+void orc_softmax_t(const float* logits, int32_t V, double T, double* p) {
+    double mx = -INFINITY;
+    for (int32_t i = 0; i < V; ++i) mx = std::max(mx, (double)logits[i] / T);
+    double sum = 0;
+    for (int32_t i = 0; i < V; ++i) {
+        p[i] = std::exp((double)logits[i] / T - mx);
+        sum += p[i];
+    }
+    for (int32_t i = 0; i < V; ++i) p[i] /= sum;
+}
+
+// Inverse-CDF sampling from non-negative weights w (not necessarily normalised): the smallest i with
+// w_0 + ... + w_i > u * (w_0 + ... + w_{V-1}); if rounding leaves none, the last index with w_i > 0.
+int32_t orc_sample_cdf(const double* w, int32_t V, double u) {
+    double total = 0;
+    for (int32_t i = 0; i < V; ++i) total += w[i];
+    const double target = u * total;
+    double run = 0;
+    int32_t last = 0;
+    for (int32_t i = 0; i < V; ++i) {
+        if (w[i] > 0) last = i;
+        run += w[i];
+        if (run > target) return i;
+    }
+    return last;
+}
+
+// Verification of k drafted tokens when sampling is used (Section 1; speculative sampling).  p has k+1 rows (M's
+// distribution for the token after each verify row), q has k rows (D's distribution each draft was sampled from),
+// drafts[j] is the token at position pos0 + 1 + j.  Draft j is accepted when its ACCEPT draw is below
+// min(1, p_j(x)/q_j(x)); the first rejected one is replaced by a token sampled from max(0, p_j - q_j) (normalised)
+// with the TARGET draw of that position; if all k are accepted one more token is sampled from p_k.  out receives
+// the accepted drafts followed by that last token (a+1 tokens); returns a.
+int32_t orc_spec_accept(const double* p, const double* q, const int32_t* drafts, int32_t k, int32_t V, uint64_t seed,
+                        int32_t pos0, int32_t* out) {
+    std::vector<double> res(V);
+    for (int32_t j = 0; j < k; ++j) {
+        const int32_t x = drafts[j];
+        const double pj = p[(size_t)j * V + x], qj = q[(size_t)j * V + x];
+        const double r = orc_uniform(seed, (uint32_t)(pos0 + 1 + j), ORC_DRAW_ACCEPT);
+        if (r * qj < pj) {  // r < min(1, p/q), written without the division
+            out[j] = x;
+            continue;
+        }
+        double mass = 0;
+        for (int32_t i = 0; i < V; ++i) {
+            res[i] = std::max(0.0, p[(size_t)j * V + i] - q[(size_t)j * V + i]);
+            mass += res[i];
+        }
+        const double u = orc_uniform(seed, (uint32_t)(pos0 + 1 + j), ORC_DRAW_TARGET);
+        // (a rejection implies p != q, so the residual has mass; should rounding leave none, fall back to p)
+        out[j] = mass > 0 ? orc_sample_cdf(res.data(), V, u) : orc_sample_cdf(p + (size_t)j * V, V, u);
+        return j;
+    }
+    out[k] = orc_sample_cdf(p + (size_t)k * V, V, orc_uniform(seed, (uint32_t)(pos0 + 1 + k), ORC_DRAW_TARGET));
+    return k;
+}
+
 // ---------------------------------------------------------------- decoder state
 struct orc_ctx {
     orc_config c;
@@ -183,6 +281,11 @@ struct orc_ctx {
     std::vector<double> sumcos_attn, sumcos_mlp;  // running sums over prompt rows
     int64_t n_sim_rows = 0;
     bool running_c = false;          // fold the rows committed after the prompt into the sums as well (opt-in)
+    // sampling (temperature > 0): every token is drawn instead of taken as the argmax
+    double temperature = 0.0;
+    uint64_t seed = 0;
+    std::vector<double> q_rows;      // [drafts of this round][V]: D's distribution each drafted token was sampled from
+    std::vector<int32_t> drafted;    // the tokens sampled by the draft steps of this round
     // results of the last pass
     int32_t last_M = 0;
     std::vector<float> last_logits;              // [M][V]
@@ -245,6 +348,7 @@ int orc_reset(orc_ctx* x) {
     std::fill(x->sumcos_mlp.begin(), x->sumcos_mlp.end(), 0.0);
     x->n_sim_rows = 0;
     x->last_M = 0;
+    x->drafted.clear();
     x->stats = orc_stats{};
     return ORC_OK;
 }
@@ -428,6 +532,27 @@ int orc_set_running_similarity(orc_ctx* x, int32_t on) {
     return ORC_OK;
 }
 
+int orc_set_sampling(orc_ctx* x, float temperature, uint64_t seed) {
+    if (!x || !(temperature >= 0.f)) return ORC_ERR_ARG;
+    x->temperature = (double)temperature;
+    x->seed = seed;
+    return ORC_OK;
+}
+
+// The token that row m of the last pass chooses for position pos: M's (or D's) argmax when decoding greedily, else a
+// draw of the given kind from softmax(logits / T).  dist, when given, receives that distribution.
+static int32_t choose_token(orc_ctx* x, int m, int32_t pos, uint32_t kind, double* dist) {
+    if (x->temperature <= 0.0) return x->last_argmax[m];
+    const int V = x->c.vocab;
+    std::vector<double> local;
+    if (!dist) {
+        local.resize(V);
+        dist = local.data();
+    }
+    orc_softmax_t(x->last_logits.data() + (size_t)m * V, V, x->temperature, dist);
+    return orc_sample_cdf(dist, V, orc_uniform(x->seed, (uint32_t)pos, kind));
+}
+
 // Section 3.2: the whole input context goes through M, fills the KV cache, yields t_1 and the
 // per-layer similarity sums.  May be called repeatedly to feed the prompt in pieces.
 int orc_prefill(orc_ctx* x, const int32_t* tokens, int32_t n, int32_t* first_token) {
@@ -439,7 +564,8 @@ int orc_prefill(orc_ctx* x, const int32_t* tokens, int32_t n, int32_t* first_tok
     x->draft_cursor = x->n_committed;
     x->stats.prefill_rows += n;
     x->stats.ms_prefill += now_ms() - t0;
-    if (first_token) *first_token = x->last_argmax[n - 1];
+    x->drafted.clear();
+    if (first_token) *first_token = choose_token(x, n - 1, x->n_committed, ORC_DRAW_TARGET, nullptr);
     return ORC_OK;
 }
 
@@ -462,6 +588,7 @@ int orc_set_skip_mask(orc_ctx* x, const uint8_t* skip_attn, const uint8_t* skip_
         x->skip_mlp[l] = skip_mlp[l] ? 1 : 0;
     }
     x->draft_cursor = x->n_committed;
+    x->drafted.clear();
     return ORC_OK;
 }
 
@@ -491,7 +618,8 @@ int orc_decode_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
     if (x->running_c) fold_committed_rows(x, 1);
     x->stats.full_passes += 1;
     x->stats.ms_full += now_ms() - t0;
-    if (token_out) *token_out = x->last_argmax[0];
+    x->drafted.clear();
+    if (token_out) *token_out = choose_token(x, 0, x->n_committed, ORC_DRAW_TARGET, nullptr);
     return ORC_OK;
 }
 
@@ -504,7 +632,17 @@ int orc_draft_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
     x->draft_cursor += 1;
     x->stats.draft_passes += 1;
     x->stats.ms_draft += now_ms() - t0;
-    if (token_out) *token_out = x->last_argmax[0];
+    // when sampling, the drafted token is a DRAFT draw from D's distribution q, which the verification needs again
+    const size_t j = x->drafted.size(), V = x->c.vocab;
+    int32_t tok;
+    if (x->temperature > 0.0) {
+        x->q_rows.resize((j + 1) * V);
+        tok = choose_token(x, 0, x->draft_cursor, ORC_DRAW_DRAFT, x->q_rows.data() + j * V);
+    } else {
+        tok = x->last_argmax[0];
+    }
+    x->drafted.push_back(tok);
+    if (token_out) *token_out = tok;
     return ORC_OK;
 }
 
@@ -514,14 +652,29 @@ int orc_draft_step(orc_ctx* x, int32_t token_in, int32_t* token_out) {
 int orc_verify(orc_ctx* x, const int32_t* tokens, int32_t k, int32_t* n_accepted, int32_t* out_tokens) {
     if (!x || !tokens || k < 0) return ORC_ERR_ARG;
     const double t0 = now_ms();
+    if (x->temperature > 0.0) {
+        // the k tokens to verify must be the ones the last k draft steps sampled: their distributions q are needed
+        if ((int32_t)x->drafted.size() != k) return ORC_ERR_STATE;
+        for (int j = 0; j < k; ++j)
+            if (x->drafted[j] != tokens[j + 1]) return ORC_ERR_STATE;
+    }
     const int rc = forward_rows(x, tokens, k + 1, x->n_committed, false, false);
     if (rc) return rc;
     int a = 0;
-    while (a < k && tokens[a + 1] == x->last_argmax[a]) ++a;
-    if (out_tokens) {
-        for (int j = 0; j < a; ++j) out_tokens[j] = tokens[j + 1];
-        out_tokens[a] = x->last_argmax[a];
+    std::vector<int32_t> emitted(k + 1);
+    if (x->temperature > 0.0) {
+        const int V = x->c.vocab;
+        std::vector<double> p((size_t)(k + 1) * V);
+        for (int j = 0; j <= k; ++j) orc_softmax_t(x->last_logits.data() + (size_t)j * V, V, x->temperature, p.data() + (size_t)j * V);
+        a = orc_spec_accept(p.data(), x->q_rows.data(), tokens + 1, k, V, x->seed, x->n_committed, emitted.data());
+    } else {
+        while (a < k && tokens[a + 1] == x->last_argmax[a]) ++a;
+        for (int j = 0; j < a; ++j) emitted[j] = tokens[j + 1];
+        emitted[a] = x->last_argmax[a];
     }
+    x->drafted.clear();
+    if (out_tokens)
+        for (int j = 0; j <= a; ++j) out_tokens[j] = emitted[j];
     if (n_accepted) *n_accepted = a;
     x->n_committed += a + 1;
     x->draft_cursor = x->n_committed;
@@ -544,6 +697,9 @@ int orc_generate(orc_ctx* x, const int32_t* prompt, int32_t n_prompt, const orc_
     orc_reset(x);
     if (gp->mode == ORC_MODE_SPEC_MANUAL_MASK) orc_set_skip_mask(x, ka.data(), km.data());
     x->running_c = (gp->admg.flags & ORC_RUNNING_C) != 0;
+    if (!(gp->temperature >= 0.f)) return ORC_ERR_ARG;
+    x->temperature = (double)gp->temperature;
+    x->seed = gp->seed;
     const double t0 = now_ms();
     int32_t last;
     int rc = orc_prefill(x, prompt, n_prompt, &last);

@@ -135,13 +135,18 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const size_t psum = ((size_t)std::max<long long>(np_max, 120) * 2 * M * 4 + 15) & ~(size_t)15;
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
-    // activation window: whole rows (the longest reduction dimension, in segments) when they fit the budget, so that
-    // short passes leave more shared memory to the ring
+    // Activation window: the longest reduction dimension (in segments of 256 inputs) cut into as few windows as leave
+    // the ring 16 slots. Streaming does not get faster with more slots than that (measured), while every further
+    // window costs a stage of a multi-row pass a block-wide refill. One row always fits whole.
     const size_t seg_max = ((size_t)std::max(c.d_model, c.d_ffn) + kSegK - 1) / kSegK;
-    // otherwise at least whole rows of d_model inputs when that stays modest (every stage but W_d then needs one window)
-    const size_t seg_d = ((size_t)c.d_model + kSegK - 1) / kSegK;
-    const size_t full_f = (size_t)M * (seg_max * kSegK + kXsPad) * 2, full_d = (size_t)M * (seg_d * kSegK + kXsPad) * 2;
-    const int xs_bytes = (int)(full_f <= (size_t)kXsBudget ? full_f : (full_d <= 57344 ? std::max<size_t>(full_d, kXsBudget) : (size_t)kXsBudget));
+    const long long fixed = 1024 + (long long)(psum + misc) + 2 * 64 * 8;
+    size_t wseg_plan = seg_max;
+    for (size_t nw = 1; nw <= seg_max; ++nw) {
+        wseg_plan = (seg_max + nw - 1) / nw;
+        const size_t bytes = (size_t)M * (wseg_plan * kSegK + kXsPad) * 2;
+        if ((long long)dv.max_smem - fixed - (long long)((bytes + 15) & ~(size_t)15) >= 16LL * kSlotBytes) break;
+    }
+    const int xs_bytes = (int)((size_t)M * (wseg_plan * kSegK + kXsPad) * 2);
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M, xs_bytes) * kSegK + kXsPad) * 2;
     // up to three groups of four warps work on attention items, as many as their scratch fits the window's bytes
     const int groups_by_scratch = (int)std::max<size_t>(1, std::min<size_t>(3, (size_t)kXsBudget / attn_scratch));

@@ -46,7 +46,8 @@ namespace asd {
 constexpr int kPassConsumerWarps = 15;
 constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
-constexpr int kXsBudget = 40960;                    // most shared memory the activation window / attention scratch may take
+constexpr unsigned kProducerNapNs = 50;             // the producer warp's sleep after a round without a free slot
+constexpr int kXsBudget = 40960;                    // most shared memory the attention scratch of all warp groups may take
 
 enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead, kStFinish };
 
@@ -101,7 +102,7 @@ struct PassParams {
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
     int attn_groups;   // 1 to 3 groups of 4 warps work on attention items
     int off_bars, off_misc, off_psum, off_reg_a;
-    int xs_bytes;      // bytes of the activation window: whole rows when they fit kXsBudget (the rest goes to the ring)
+    int xs_bytes;      // bytes of the activation window (as few windows per stage as leave the ring 16 slots)
 };
 
 constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)
@@ -297,6 +298,41 @@ __device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& 
     }
 }
 
+// Where item c.idx of the lane's current stage lives: a K/V box (tensor map + coordinates) or a run of weight bytes.
+struct ItemSrc {
+    const CUtensorMap* map;  // non-null: K/V box at (x, y)
+    int x, y;
+    const unsigned char* ptr;
+    uint32_t bytes;
+};
+__device__ __forceinline__ ItemSrc item_source(const PassParams& p, const ProdState& c) {
+    ItemSrc s;
+    if (c.type == kStAttn) {
+        const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
+        const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
+        const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
+        const int j = c.idx / (2 * tile_slots), r = c.idx - j * 2 * tile_slots;
+        const int which = r / tile_slots, t = r - which * tile_slots;
+        const int rg = t / nhb, hb = t - rg * nhb;
+        const int item = c.first + j;
+        const int kvh = item / c.n_chunks, chunk = item - kvh * c.n_chunks;
+        s.map = which ? c.tm_v : c.tm_k;
+        s.x = kvh * p.head_dim + hb * 64;
+        s.y = chunk * kAttnChunk + rg * kBoxKeys;
+        s.ptr = nullptr;
+        s.bytes = (uint32_t)kBoxKeys * box_cols * 2u;
+    } else {
+        const int seg = c.idx / c.n_oct, o = c.idx - seg * c.n_oct;
+        const int nblk = min(kSegBlocks, c.row_blocks - seg * kSegBlocks);  // column blocks of this segment
+        const int rows = 2 * min(kGrpPairs, c.np - kGrpPairs * o);
+        s.map = nullptr;
+        s.x = s.y = 0;
+        s.ptr = c.slab + (size_t)seg * c.np * (kSegK * 4) + (size_t)o * nblk * (kGrpRows * 64);
+        s.bytes = (uint32_t)(nblk * rows * 64);
+    }
+    return s;
+}
+
 template <int M>
 __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     const int lane = threadIdx.x & 31;
@@ -311,6 +347,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     long long tp_first = (p.trace && lane == 0) ? global_ns() : 0, stall = 0, t_blocked = 0;
     bool blocked = false;
     for (unsigned round = 1; __any_sync(0xffffffffu, active); ++round) {
+        bool copied = false;
         if (active) {
             const uint32_t g = c.gi + (uint32_t)c.idx;
             int slot;
@@ -323,28 +360,12 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 if (p.trace && lane == 0 && blocked) stall += clock64() - t_blocked;
                 blocked = false;
                 unsigned char* dst = sm.ring + (size_t)slot * kSlotBytes;
-                if (c.type == kStAttn) {
-                    const int nhb = p.head_dim > 64 ? p.head_dim / 64 : 1;
-                    const int box_cols = p.head_dim > 64 ? 64 : p.head_dim;
-                    const int tile_slots = (kAttnChunk / kBoxKeys) * nhb;
-                    const int j = c.idx / (2 * tile_slots), r = c.idx - j * 2 * tile_slots;
-                    const int which = r / tile_slots, t = r - which * tile_slots;
-                    const int rg = t / nhb, hb = t - rg * nhb;
-                    const int item = c.first + j;
-                    const int kvh = item / c.n_chunks, chunk = item - kvh * c.n_chunks;
-                    mbar_expect_tx(&sm.full[slot], (uint32_t)kBoxKeys * box_cols * 2u);
-                    tma_load_2d(dst, which ? c.tm_v : c.tm_k, kvh * p.head_dim + hb * 64, chunk * kAttnChunk + rg * kBoxKeys,
-                                &sm.full[slot]);
-                } else {
-                    const int seg = c.idx / c.n_oct, o = c.idx - seg * c.n_oct;
-                    const int nblk = min(kSegBlocks, c.row_blocks - seg * kSegBlocks);  // column blocks of this segment
-                    const int rows = 2 * min(kGrpPairs, c.np - kGrpPairs * o);
-                    const uint32_t bytes = (uint32_t)(nblk * rows * 64);
-                    mbar_expect_tx(&sm.full[slot], bytes);
-                    tma_load_1d_hint(dst, c.slab + (size_t)seg * c.np * (kSegK * 4) + (size_t)o * nblk * (kGrpRows * 64), bytes, &sm.full[slot],
-                                     pol_stream);
-                }
+                const ItemSrc src = item_source(p, c);
+                mbar_expect_tx(&sm.full[slot], src.bytes);
+                if (src.map) tma_load_2d(dst, src.map, src.x, src.y, &sm.full[slot]);
+                else tma_load_1d_hint(dst, src.ptr, src.bytes, &sm.full[slot], pol_stream);
                 issued[1] = issued[0], issued[0] = g, ++n_issued;
+                copied = true;
                 t_progress = clock64();
                 c.idx += 32;
                 if (c.idx >= c.n_items) {
@@ -371,6 +392,10 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                 }
             }
         }
+        // A round in which no lane found a free slot: sleep a moment instead of polling again at once. The warp shares
+        // its scheduler with three consumer warps, and a refill that starts some tens of nanoseconds later costs
+        // nothing against a memory latency of microseconds.
+        if (!__any_sync(0xffffffffu, copied)) __nanosleep(kProducerNapNs);
         __syncwarp();
     }
     // If the pass was abandoned, copies may still be in flight into this CTA's shared memory: let this lane's
@@ -478,7 +503,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     constexpr bool kKeepX = (M <= 2);
     const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
     uint2 gpre[3] = {make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)};  // this thread's RMSNorm gains
-    if (keep) {
+    const bool short_rows = norm && n_in <= kPassConsumers * 12;  // a thread owns at most three 4-element chunks of a row
+    if (short_rows) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) {
             const int i = (tid + c * kPassConsumers) * 4;
@@ -535,8 +561,38 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     }
                 }
             }
+        } else if (M <= 3 && n_in <= kPassConsumers * 12) {
+            // up to three rows x three chunks per thread in flight together: one memory round trip per three rows
+#pragma unroll
+            for (int m0 = 0; m0 < M; m0 += 3) {
+                float4 v[3][3];
+#pragma unroll
+                for (int u = 0; u < 3; ++u)
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        const int i = (tid + c * kPassConsumers) * 4;
+                        v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (m0 + u < M && i < n_in) v[u][c] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
+                    }
+#pragma unroll
+                for (int u = 0; u < 3; ++u)
+                    if (m0 + u < M) {
+                        float s = ssq[m0 + u];
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) {
+                            const int i = (tid + c * kPassConsumers) * 4;
+                            if (i < n_in) {  // same order of additions as the one-row path: chunk by chunk, element by element
+                                s = fmaf(v[u][c].x, v[u][c].x, s);
+                                s = fmaf(v[u][c].y, v[u][c].y, s);
+                                s = fmaf(v[u][c].z, v[u][c].z, s);
+                                s = fmaf(v[u][c].w, v[u][c].w, s);
+                            }
+                        }
+                        ssq[m0 + u] = s;
+                    }
+            }
         } else {
-            // the loads of up to four rows are in flight together (one memory round trip per four rows and stride)
+            // long rows: the loads of up to four rows are in flight together (one memory round trip per four rows and stride)
             for (int i = tid * 4; i < n_in; i += kPassConsumers * 4) {
 #pragma unroll
                 for (int m0 = 0; m0 < M; m0 += 4) {
@@ -600,6 +656,44 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                             o.y = *reinterpret_cast<uint32_t*>(&hi);
                         }
                         *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                    }
+                }
+            }
+            for (int i = kPassConsumers * 12 + tid * 4; i < wlen; i += kPassConsumers * 4)  // zero padding past 5760
+                for (int m = 0; m < M; ++m) *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = make_uint2(0u, 0u);
+        } else if (M <= 3 && short_rows && w0 == 0 && wlen >= n_in) {
+            // the window holds whole rows: three rows x three chunks per thread in flight together, then normalised
+#pragma unroll
+            for (int m0 = 0; m0 < M; m0 += 3) {
+                float4 v[3][3];
+#pragma unroll
+                for (int u = 0; u < 3; ++u)
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        const int i = (tid + c * kPassConsumers) * 4;
+                        v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (m0 + u < M && i < n_in) v[u][c] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
+                    }
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const int i = (tid + c * kPassConsumers) * 4;
+                    if (i < wlen) {
+                        const bool in = i < n_in;
+                        const uint2 gv = gpre[c];
+                        const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
+#pragma unroll
+                        for (int u = 0; u < 3; ++u)
+                            if (m0 + u < M) {
+                                const int m = m0 + u;
+                                uint2 o = make_uint2(0u, 0u);
+                                if (in) {
+                                    __nv_bfloat162 lo = __floats2bfloat162_rn(v[u][c].x * inv[m] * g0, v[u][c].y * inv[m] * g1);
+                                    __nv_bfloat162 hi = __floats2bfloat162_rn(v[u][c].z * inv[m] * g2, v[u][c].w * inv[m] * g3);
+                                    o.x = *reinterpret_cast<uint32_t*>(&lo);
+                                    o.y = *reinterpret_cast<uint32_t*>(&hi);
+                                }
+                                *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                            }
                     }
                 }
             }

@@ -103,6 +103,11 @@ typedef struct {
      * the gap between D's largest and second-largest logit, is below this value; that token is still verified.
      * 0 = off (every round drafts draft_len tokens). Costs one host read-back per draft step. */
     float draft_exit_margin;
+    /* Sampling (Section 1; the T > 0 columns of Tables 3 and 4): 0 = greedy decoding as described above. Above 0 every
+     * token is drawn from softmax(logits / temperature) and the verification accepts drafts so that the output keeps
+     * the full model's distribution; see asd_set_sampling for the rule and the random numbers. */
+    float temperature;
+    uint64_t seed;
 } asd_gen_params;
 
 /* Counters and device times (CUDA events) accumulated since the last asd_reset / asd_generate start.
@@ -165,6 +170,21 @@ int asd_draft_step(asd_ctx* ctx, int32_t token_in, int32_t* token_out);
  * accepted drafts followed by g_a (a+1 tokens, a = *n_accepted); a+1 positions are committed and the draft
  * cursor returns to the committed length. 0 <= k <= max_draft. */
 int asd_verify(asd_ctx* ctx, const int32_t* tokens, int32_t k, int32_t* n_accepted, int32_t* out_tokens);
+
+/* Decoding with sampling instead of the argmax (Section 1 on verification "when sampling is used", which points to
+ * the rule of speculative sampling; the paper runs T = 0.2 and T = 0.6 in Tables 3 and 4). temperature = 0 restores
+ * greedy decoding. With temperature > 0:
+ *   - asd_prefill's first token and asd_decode_step's token are drawn from p = softmax(logits / temperature);
+ *   - asd_draft_step draws its token from the draft model's distribution q and keeps q on the device;
+ *   - asd_verify takes the tokens drawn by this round's draft steps (anything else: ASD_ERR_STATE) and accepts draft x
+ *     at a position when its uniform number r satisfies r < min(1, p(x)/q(x)); the first rejected draft is replaced
+ *     by a draw from max(0, p - q) normalised, and a round in which all drafts are accepted ends with one more draw
+ *     from p. Every emitted token is then distributed as if M had drawn it.
+ * Random numbers: the counter-based generator Philox4x32-10 with key = seed and counter = (position of the token being
+ * chosen, kind of draw: 0 draft, 1 acceptance test, 2 full model's draw, 0, 0); its first output word x gives the
+ * uniform number (x + 1/2) / 2^32. Probabilities and all comparisons are evaluated in double precision on the device.
+ * asd_generate takes both values from its parameter block instead. Errors: ARG (negative or NaN temperature). */
+int asd_set_sampling(asd_ctx* ctx, float temperature, uint64_t seed);
 
 /* The whole method: reset, prefill, t_1, (Algorithm 1), then rounds of draft_len draft steps and one verify
  * until max_new tokens (out[0] = t_1) or eos. out has room for max_new tokens. stats may be NULL. */

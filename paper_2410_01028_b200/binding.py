@@ -34,7 +34,8 @@ class AdmgParams(ctypes.Structure):
 
 class GenParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("draft_len", ctypes.c_int32), ("max_new", ctypes.c_int32),
-                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float)]
+                ("eos_id", ctypes.c_int32), ("admg", AdmgParams), ("draft_exit_margin", ctypes.c_float),
+                ("temperature", ctypes.c_float), ("seed", ctypes.c_uint64)]
 
 
 class Stats(ctypes.Structure):
@@ -54,7 +55,7 @@ EXPORTS = (
     "asd_load_weights_file", "asd_reset", "asd_prefill", "asd_prefill_device", "asd_get_similarity", "asd_admg_update",
     "asd_set_skip_mask", "asd_decode_step", "asd_draft_step", "asd_verify", "asd_generate", "asd_generate_device",
     "asd_get_last_cosines", "asd_get_last_margins", "asd_get_last_logits", "asd_set_debug", "asd_get_last_trace", "asd_get_kv", "asd_get_positions", "asd_get_stats",
-    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_admg_ext", "asd_set_running_similarity", "asd_set_prefill_mode", "asd_gemm_bf16",
+    "asd_fused_gemv_scratch_bytes", "asd_fused_gemv", "asd_fused_gemv_static", "asd_admg", "asd_admg_ext", "asd_set_running_similarity", "asd_set_prefill_mode", "asd_gemm_bf16", "asd_set_sampling",
 )
 
 _lib = None
@@ -243,6 +244,11 @@ class Decoder:
         flags = (1 if record_logits else 0) | (2 if trace else 0) | (4 if short_waits else 0) | (8 if missing_arrival else 0)
         self._check(lib().asd_set_debug(self._ctx, ctypes.c_int32(flags)), "asd_set_debug")
 
+    def set_sampling(self, temperature, seed=0):
+        """temperature 0 = greedy (default); above 0 every token is drawn and verification keeps M's distribution
+        (see asd_set_sampling)."""
+        self._check(lib().asd_set_sampling(self._ctx, ctypes.c_float(temperature), ctypes.c_uint64(seed)), "asd_set_sampling")
+
     def set_prefill_mode(self, mode):
         """PREFILL_AUTO (default), PREFILL_ROWS (row passes, bit-identical to one-row passes) or PREFILL_GEMM."""
         self._check(lib().asd_set_prefill_mode(self._ctx, ctypes.c_int32(mode)), "asd_set_prefill_mode")
@@ -309,14 +315,17 @@ class Decoder:
         self._check(lib().asd_verify(self._ctx, _vp(t), ctypes.c_int32(k), ctypes.byref(a), _vp(out)), "asd_verify")
         return a.value, out[: a.value + 1].copy()
 
-    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
-        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin)
+    def _gen_params(self, max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0,
+                    temperature=0.0, seed=0):
+        return GenParams(mode, draft_len, max_new, eos_id, AdmgParams(alpha, m, n, flags, alpha_mlp, refresh), draft_exit_margin,
+                         temperature, seed)
 
     def generate(self, prompt, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2, flags=ADMG_ALL, eos_id=-1,
-                 alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
+                 alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0, temperature=0.0, seed=0):
         """Host buffers in, host buffers out. Returns (tokens, stats dict)."""
         p = np.ascontiguousarray(prompt, dtype=np.int32)
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin,
+                              temperature, seed)
         out = np.zeros(max_new, np.int32)
         n_out = ctypes.c_int32()
         st = Stats()
@@ -325,9 +334,10 @@ class Decoder:
         return out[: n_out.value].copy(), st.as_dict()
 
     def generate_device(self, dev_prompt, dev_out, max_new, mode=MODE_AR, draft_len=4, alpha=0.985, m=3, n=2,
-                        flags=ADMG_ALL, eos_id=-1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0):
+                        flags=ADMG_ALL, eos_id=-1, alpha_mlp=1.0, refresh=0, draft_exit_margin=0.0, temperature=0.0, seed=0):
         """Prompt and output are int32 CUDA tensors. Returns (n_out, stats dict)."""
-        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin)
+        gp = self._gen_params(max_new, mode, draft_len, alpha, m, n, flags, eos_id, alpha_mlp, refresh, draft_exit_margin,
+                              temperature, seed)
         n_out = ctypes.c_int32()
         st = Stats()
         self._check(lib().asd_generate_device(self._ctx, _vp(dev_prompt), ctypes.c_int32(dev_prompt.numel()),

@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "pass.cuh"
 #include "prefill.h"
+#include "sample.h"
 
 namespace asd {
 
@@ -172,7 +173,7 @@ struct Layout {
     size_t l_attn_norm, l_wqkv, l_wo, l_mlp_norm, l_wgu, l_wd;  // offsets inside one layer block
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
     size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
-    size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits;
+    size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits, probs_p, probs_q;
     size_t stage_tab, tmaps, sync_words, trace, resid_tab;
     int max_stages;
     size_t total;
@@ -256,6 +257,8 @@ static Layout make_layout(const asd_config& c) {
     L.argmax = take(64 * 4);
     L.accept = take(64 * 4);
     L.logits = take((size_t)kPassMaxRows * V * 4);
+    L.probs_p = take((size_t)kMaxRows * V * 8);  // sampling: the full model's distributions of a verify pass
+    L.probs_q = take((size_t)kMaxRows * V * 8);  // sampling: the draft model's distributions of this round's draft steps
     L.max_stages = 5 * c.n_layers + 3;
     L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
@@ -313,6 +316,10 @@ struct asd_ctx {
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, last_had_lm_head = false, trace = false;
     bool short_waits = false, inject_missing_arrival = false;  // test hooks of the bounded device waits (asd_set_debug)
+    // sampling (temperature > 0): every token is drawn; the draft steps of a round keep their distributions for the verify
+    double temperature = 0.0;
+    uint64_t seed = 0;
+    std::vector<int32_t> drafted;  // tokens drawn by the single-step draft calls of this round (host copy)
     bool dev_failed = false;     // a kernel gave up waiting: nothing more is launched until asd_reset
     std::string dev_failed_msg;
     int last_n_stages = 0;
@@ -576,7 +583,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
     p.margin_out = reinterpret_cast<float*>(x->at<int>(ly.argmax) + 32);  // second half of the argmax block
     p.accept_out = accept ? x->at<int>(ly.accept) : nullptr;
-    p.logits_out = x->debug_logits ? x->at<float>(ly.logits) : nullptr;
+    p.logits_out = (x->debug_logits || x->temperature > 0.0) ? x->at<float>(ly.logits) : nullptr;
     p.acc_sim = acc_sim ? 1 : 0;
     p.trace = x->trace ? x->at<long long>(ly.trace) : nullptr;
     x->last_n_stages = p.n_stages;
@@ -623,6 +630,26 @@ static int read_back(asd_ctx* x, const int* dev_src, int n) {
     ASD_CUDA(x, cudaMemcpyAsync(x->pinned + 32, x->at<unsigned>(x->lay.sync_words) + 32, 32, cudaMemcpyDeviceToHost, x->stream));
     ASD_CUDA(x, cudaStreamSynchronize(x->stream));
     return check_device_error(x, x->pinned + 32);
+}
+
+// Sampling: row `row` of the pass that has just been launched chooses the token at `position`. Its distribution
+// softmax(logits / T) goes to probs (device, vocab doubles) and a draw of the given kind to token_out (and token_out2).
+static int sample_row(asd_ctx* x, int row, double* probs, int position, int kind, int* token_out, int* token_out2) {
+    const int V = x->c.vocab;
+    ASD_CUDA(x, launch_softmax_rows(x->at<float>(x->lay.logits) + (size_t)row * V, 1, V, x->temperature, probs, x->stream));
+    ASD_CUDA(x, launch_draw(probs, V, x->seed, position, kind, token_out, token_out2, x->stream));
+    x->stats.kernel_launches += 2;
+    return ASD_OK;
+}
+// Sampling: acceptance of the k drafts of the verify pass that has just been launched at position pos0 (rows in
+// dev_row_tokens); the result replaces the greedy one in the accept block.
+static int sample_accept(asd_ctx* x, int k, int pos0, const int* dev_row_tokens) {
+    const int V = x->c.vocab;
+    double* P = x->at<double>(x->lay.probs_p);
+    ASD_CUDA(x, launch_softmax_rows(x->at<float>(x->lay.logits), k + 1, V, x->temperature, P, x->stream));
+    ASD_CUDA(x, launch_accept(P, x->at<double>(x->lay.probs_q), dev_row_tokens, k, V, x->seed, pos0, x->at<int>(x->lay.accept), x->stream));
+    x->stats.kernel_launches += 2;
+    return ASD_OK;
 }
 
 // Running similarities: request the per-row cosines of the pass that has just been launched (before the caller's
@@ -903,6 +930,7 @@ extern "C" int asd_reset(asd_ctx* x) {
     std::fill(x->run_mlp.begin(), x->run_mlp.end(), 0.0);
     x->n_run_rows = 0;
     x->last_M = 0;
+    x->drafted.clear();
     x->dev_failed = false;
     x->stats = asd_stats{};
     x->spans.clear();
@@ -1012,6 +1040,11 @@ static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int3
     x->draft_cursor = x->n_committed;
     x->n_sim_rows += n;
     x->stats.prefill_rows += n;
+    x->drafted.clear();
+    if (x->temperature > 0.0) {  // t_1 is the full model's own draw for position n_committed; it takes the argmax's place
+        int* slot = x->at<int>(x->lay.argmax) + (last_rows - 1);
+        if ((rc = sample_row(x, last_rows - 1, x->at<double>(x->lay.probs_p), x->n_committed, kDrawTarget, slot, nullptr))) return rc;
+    }
     if (first_token) {
         if ((rc = read_back(x, x->at<int>(x->lay.argmax) + (last_rows - 1), 1))) return rc;
         *first_token = x->pinned[0];
@@ -1067,6 +1100,7 @@ extern "C" int asd_set_skip_mask(asd_ctx* x, const uint8_t* skip_attn, const uin
         x->skip_mlp[l] = skip_mlp[l] ? 1 : 0;
     }
     x->draft_cursor = x->n_committed;
+    x->drafted.clear();
     return build_stage_tables(x);
 }
 
@@ -1119,11 +1153,15 @@ extern "C" int asd_decode_step(asd_ctx* x, int32_t token_in, int32_t* token_out)
     if (rc) return rc;
     rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, x->at<int>(x->lay.tok_in), false, nullptr, false);
     if (rc) return rc;
+    if (x->temperature > 0.0 &&
+        (rc = sample_row(x, 0, x->at<double>(x->lay.probs_p), x->n_committed + 1, kDrawTarget, x->at<int>(x->lay.argmax), nullptr)))
+        return rc;
     if ((rc = request_cosines(x))) return rc;
     if ((rc = read_back(x, x->at<int>(x->lay.argmax), 1))) return rc;
     fold_committed_rows(x, 1);
     x->n_committed += 1;
     x->draft_cursor = x->n_committed;
+    x->drafted.clear();
     if (token_out) *token_out = x->pinned[0];
     return resolve_spans(x);
 }
@@ -1134,10 +1172,17 @@ extern "C" int asd_draft_step(asd_ctx* x, int32_t token_in, int32_t* token_out) 
     if (x->draft_cursor + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
     int rc = stage_tokens(x, &token_in, 1, x->at<int>(x->lay.tok_in));
     if (rc) return rc;
+    const size_t j = x->drafted.size();
+    if (x->temperature > 0.0 && (int)j >= kMaxRows - 1) return fail(x, ASD_ERR_STATE, "more draft steps in one round than a verify pass has rows");
     rc = timed_pass(x, SPAN_DRAFT, 1, x->draft_cursor, x->at<int>(x->lay.tok_in), true, nullptr, false);
     if (rc) return rc;
+    // when sampling, the drafted token is a draw from the draft model's distribution q, which the verification needs again
+    if (x->temperature > 0.0 && (rc = sample_row(x, 0, x->at<double>(x->lay.probs_q) + j * (size_t)x->c.vocab, x->draft_cursor + 1,
+                                                 kDrawDraft, x->at<int>(x->lay.argmax), nullptr)))
+        return rc;
     if ((rc = read_back(x, x->at<int>(x->lay.argmax), 1))) return rc;
     x->draft_cursor += 1;
+    x->drafted.push_back(x->pinned[0]);
     if (token_out) *token_out = x->pinned[0];
     return resolve_spans(x);
 }
@@ -1147,10 +1192,18 @@ extern "C" int asd_verify(asd_ctx* x, const int32_t* tokens, int32_t k, int32_t*
     if (!x->have_weights) return fail(x, ASD_ERR_STATE, "weights not loaded");
     if (k < 0 || k > x->c.max_draft) return fail(x, ASD_ERR_ARG, "draft length out of range");
     if ((long long)x->n_committed + k + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "verify would exceed max_seq");
+    if (x->temperature > 0.0) {
+        // the k tokens to verify must be the ones the last k draft steps drew: their distributions q are needed
+        bool same = (int32_t)x->drafted.size() == k;
+        for (int j = 0; same && j < k; ++j) same = x->drafted[j] == tokens[j + 1];
+        if (!same) return fail(x, ASD_ERR_STATE, "sampling-based verification needs exactly the tokens drawn by this round's draft steps");
+    }
     int rc = stage_tokens(x, tokens, k + 1, x->at<int>(x->lay.draft_toks));
     if (rc) return rc;
     rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, x->at<int>(x->lay.draft_toks), false, nullptr, true);
     if (rc) return rc;
+    if (x->temperature > 0.0 && (rc = sample_accept(x, k, x->n_committed, x->at<int>(x->lay.draft_toks)))) return rc;
+    x->drafted.clear();
     if ((rc = request_cosines(x))) return rc;
     if ((rc = read_back(x, x->at<int>(x->lay.accept), k + 2))) return rc;
     const int a = x->pinned[0];
@@ -1178,6 +1231,11 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
     if (rc) return rc;
     if (gp->mode == ASD_MODE_SPEC_MANUAL_MASK) asd_set_skip_mask(x, ka.data(), km.data());
     x->running_c = (gp->admg.flags & ASD_RUNNING_C) != 0;
+    if (!(gp->temperature >= 0.f)) return fail(x, ASD_ERR_ARG, "bad generation parameters");
+    x->temperature = (double)gp->temperature;
+    x->seed = gp->seed;
+    const bool sampling = x->temperature > 0.0;
+    int* scratch_tok = x->at<int>(x->lay.argmax);  // where a pass leaves its own argmax when the token is drawn instead
     cudaStream_t s = x->stream;
     size_t ev_begin, ev_end;
     if ((rc = new_event(x, &ev_begin))) return rc;
@@ -1202,9 +1260,10 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
         // token i is read from dev_out[i-1] and written to dev_out[i]: no host round trip between steps
         while (produced < gp->max_new && !stop) {
             if (x->n_committed + 1 > x->c.max_seq) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
-            rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, dev_out + produced - 1, false, dev_out + produced, false);
+            rc = timed_pass(x, SPAN_FULL, 1, x->n_committed, dev_out + produced - 1, false, sampling ? scratch_tok : dev_out + produced, false);
             if (rc) return rc;
             x->n_committed += 1;
+            if (sampling && (rc = sample_row(x, 0, x->at<double>(x->lay.probs_p), x->n_committed, kDrawTarget, dev_out + produced, nullptr))) return rc;
             if (need_host_token || x->running_c) {  // running similarities: one host read-back per step
                 if ((rc = request_cosines(x))) return rc;
                 if ((rc = read_back(x, dev_out + produced, 1))) return rc;
@@ -1222,8 +1281,11 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             if (k < 0) return fail(x, ASD_ERR_OVERFLOW, "KV cache is full");
             ASD_CUDA(x, cudaMemcpyAsync(draft, last_src, 4, cudaMemcpyDeviceToDevice, s));
             for (int j = 0; j < k; ++j) {  // k steps of the draft model, chained on the device
-                rc = timed_pass(x, SPAN_DRAFT, 1, x->n_committed + j, draft + j, true, draft + j + 1, false);
+                rc = timed_pass(x, SPAN_DRAFT, 1, x->n_committed + j, draft + j, true, sampling ? scratch_tok : draft + j + 1, false);
                 if (rc) return rc;
+                if (sampling && (rc = sample_row(x, 0, x->at<double>(x->lay.probs_q) + (size_t)j * x->c.vocab, x->n_committed + j + 1, kDrawDraft,
+                                                 draft + j + 1, nullptr)))
+                    return rc;
                 // draft exiting: a draft token whose top-2 logit margin in D falls below the threshold ends the run
                 // (the token itself is still verified); costs one host read-back per draft step
                 if (gp->draft_exit_margin > 0.f && j + 1 < k) {
@@ -1235,6 +1297,7 @@ static int generate_device(asd_ctx* x, const int32_t* dev_prompt, int32_t n_prom
             }
             rc = timed_pass(x, SPAN_VERIFY, k + 1, x->n_committed, draft, false, nullptr, true);
             if (rc) return rc;
+            if (sampling && (rc = sample_accept(x, k, x->n_committed, draft))) return rc;
             if ((rc = request_cosines(x))) return rc;
             if ((rc = read_back(x, accept, k + 2))) return rc;
             const int a = x->pinned[0];
@@ -1320,6 +1383,14 @@ extern "C" int asd_set_debug(asd_ctx* x, int32_t flags) {
     x->trace = (flags & 2) != 0;
     x->short_waits = (flags & ASD_DEBUG_SHORT_WAITS) != 0;
     x->inject_missing_arrival = (flags & ASD_DEBUG_MISSING_ARRIVAL) != 0;
+    return ASD_OK;
+}
+
+extern "C" int asd_set_sampling(asd_ctx* x, float temperature, uint64_t seed) {
+    if (!x || !(temperature >= 0.f)) return ASD_ERR_ARG;
+    x->temperature = (double)temperature;
+    x->seed = seed;
+    x->drafted.clear();
     return ASD_OK;
 }
 

@@ -57,6 +57,9 @@ def parse_args():
     ap.add_argument("--draft-exit", type=float, default=0.1, help="draft exiting: stop a round's drafting below this top-2 "
                     "logit gap of the draft model (0 = every round drafts --draft-len tokens)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the extra blocks of the line (headline variants, sampling, "
+                    "the 8192-token and 13B-shaped workloads)")
+    ap.add_argument("--no-13b", action="store_true", help="skip the 13B-shaped workload of the extra blocks (26 GB of weights)")
     ap.add_argument("--gemv-microbench", action="store_true", help="also time the stand-alone fused GEMV kernel")
     ap.add_argument("--ablation", action="store_true", help="also time the rule subsets of the paper's ablation (Table 5) and "
                     "the two extensions (MLP similarity threshold, running similarities) end to end")
@@ -201,9 +204,17 @@ def oracle_sample(args, model, shape, prompt, steps, warmup):
         if i >= warmup:
             times.append(dt)
     per_step = sum(times) / len(times)
+    # the oracle's time per pass (its own clocks around each pass), at this sample's context length
+    pass_ms = {"draft": st["ms_draft"] / max(st["draft_passes"], 1), "verify": st["ms_verify"] / max(st["verify_passes"], 1),
+               "verify_rows": 1 + st["drafted"] / max(st["verify_passes"], 1)}
+    t0 = time.perf_counter()
+    orc.decode_step(int(toks[-1]))
+    pass_ms["full"] = (time.perf_counter() - t0) * 1e3
     return {"value": max_new / per_step, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": "first %d prompt tokens, %d generated tokens, same ADMG and draft settings; %.1f s per step"
-                      % (n_prompt, max_new, per_step)}, per_step
+                      % (n_prompt, max_new, per_step),
+            "pass_ms": pass_ms, "pass_ms_at": "%d to %d cached positions (the oracle's cost per row is dominated by the "
+                                             "weights, not by the context)" % (n_prompt, n_prompt + max_new)}, per_step
 
 
 def run_reference(args):
@@ -333,6 +344,82 @@ def ablation(torch, asd, dec, dev_prompt, dev_out, new, args, ar_tokens):
                     "acceptance": st["accepted"] / max(st["drafted"], 1), "removed_attn": int(ra.sum()), "removed_mlp": int(rm.sum()),
                     "draft_ms": st["ms_draft"] / max(st["draft_passes"], 1), "spec_equals_ar": same})
     return out
+
+
+def headline_variants(asd, dec, dev_prompt, dev_out, new, args, ar_tokens):
+    """The same workload under three settings of the draft-model generator, so that the headline's dependence on the
+    tuned threshold and on draft exiting (an extension the paper only points to) is visible: Table 2's
+    hyper-parameters with all three rules; the threshold of the command line without draft exiting; and with it."""
+    rows = [("Algorithm 1 with Table 2's hyper-parameters (alpha 0.985, m 3, n 2), no draft exiting",
+             dict(draft_len=args.draft_len, alpha=0.985, m=3, n=2, flags=asd.ADMG_ALL, draft_exit_margin=0.0)),
+            ("command-line setting without draft exiting", dict(admg_kwargs(args), draft_exit_margin=0.0)),
+            ("command-line setting (the headline)", admg_kwargs(args))]
+    out = []
+    for name, kw in rows:
+        dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        _, st = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        ra, rm = dec.admg_update(kw["alpha"], kw["m"], kw["n"], kw["flags"])
+        out.append({"setting": name, "tokens_per_s": new / (st["ms_total"] * 1e-3), "acceptance": st["accepted"] / max(st["drafted"], 1),
+                    "removed_attn": int(ra.sum()), "removed_mlp": int(rm.sum()),
+                    "draft_ms": st["ms_draft"] / max(st["draft_passes"], 1), "verify_ms": st["ms_verify"] / max(st["verify_passes"], 1),
+                    "spec_equals_ar": bool((dev_out.cpu().numpy() == ar_tokens).all())})
+    return out
+
+
+def sampling_rows(asd, dec, dev_prompt, dev_out, new, args):
+    """Sampling-based decoding at the paper's temperatures (Tables 3 and 4): plain sampled decoding and speculative
+    decoding with distribution-preserving acceptance, same seed."""
+    out = []
+    for T in (0.2, 0.6):
+        dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_AR, temperature=T, seed=1)
+        _, st_a = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_AR, temperature=T, seed=1)
+        kw = dict(admg_kwargs(args), temperature=T, seed=1)
+        dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        _, st_s = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+        out.append({"temperature": T, "sampled_ar_tokens_per_s": new / (st_a["ms_total"] * 1e-3),
+                    "sampled_spec_tokens_per_s": new / (st_s["ms_total"] * 1e-3),
+                    "acceptance": st_s["accepted"] / max(st_s["drafted"], 1)})
+    return out
+
+
+def other_workload(torch, asd, name, args, hbm_peak, peak_kind, model=None):
+    """One more workload of the benchmark family in the same line (one warm-up and one timed generation each of plain
+    greedy and speculative decoding): per-pass times, roofline fractions, tokens/s."""
+    shape, S, new, desc = WORKLOADS[name]
+    t0 = time.perf_counter()
+    if model is None:
+        model = synth.make_model(shape, seed=0)
+    dec = asd.Decoder(shape, max_seq=S + new + 16, max_draft=8)
+    dec.load_weights_host(model)
+    dev_prompt = torch.from_numpy(synth.make_prompt(shape.vocab, S, seed=1)).cuda()
+    dev_out = torch.zeros(new, dtype=torch.int32, device="cuda")
+    kw = dict(admg_kwargs(args), draft_len=6 if name == "13b" else args.draft_len)
+    dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_AR)
+    _, st_ar = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_AR)
+    ar = dev_out.cpu().numpy().copy()
+    dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+    _, st = dec.generate_device(dev_prompt, dev_out, new, mode=asd.MODE_SPEC, **kw)
+    same = bool((dev_out.cpu().numpy() == ar).all())
+
+    def pp(kind, s):
+        n = s[kind + "_passes"]
+        if not n:
+            return None
+        gbs = s["bytes_" + kind] / s["ms_" + kind] / 1e6
+        return {"ms": s["ms_" + kind] / n, "GBps": gbs, "frac_of_%s_peak" % peak_kind: gbs / hbm_peak, "frac_of_8TBps": gbs / 8000.0}
+
+    _, tf_sustained, _ = tensor_peak()
+    pf_tf = prefill_flops(shape, S) / (st["ms_prefill"] * 1e-3) / 1e12
+    res = {"workload": desc, "draft_len": kw["draft_len"], "spec_tokens_per_s": new / (st["ms_total"] * 1e-3),
+           "ar_tokens_per_s": new / (st_ar["ms_total"] * 1e-3), "acceptance": st["accepted"] / max(st["drafted"], 1),
+           "spec_equals_ar": same, "passes": {"full": pp("full", st_ar), "draft": pp("draft", st), "verify": pp("verify", st)},
+           "prefill_ms": st["ms_prefill"], "prefill_TFLOPs": pf_tf, "prefill_frac_of_sustained_tensor_peak": pf_tf / tf_sustained,
+           "wall_s": None}
+    dec.close()
+    del dec
+    torch.cuda.empty_cache()
+    res["wall_s"] = time.perf_counter() - t0
+    return res
 
 
 def rank_env():
@@ -490,6 +577,19 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         cb, _ = oracle_sample(args, model, shape, synth.make_prompt(shape.vocab, S, seed=1), 1, 0)
         line["cpu_baseline"] = cb
+    if not args.no_extras and world == 1 and not (args.layers or args.prompt_len or args.max_new):
+        line["headline_variants"] = headline_variants(asd, dec, dev_prompt, dev_out, new, args, ar_tokens)
+        line["sampling"] = sampling_rows(asd, dec, dev_prompt, dev_out, new, args)
+        if args.workload == "7b":
+            # the long-context workload shares the 7B-shaped weights; the 13B-shaped one generates its own
+            dec.close()
+            del dec
+            torch.cuda.empty_cache()
+            others = [other_workload(torch, asd, "7b_long", args, hbm_peak, peak_kind, model=model)]
+            if not args.no_13b:
+                del model
+                others.append(other_workload(torch, asd, "13b", args, hbm_peak, peak_kind))
+            line["other_workloads"] = others
     print(json.dumps(line))
 
 

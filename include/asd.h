@@ -223,14 +223,15 @@ int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
 /* Debug flags: bit 0 = record the logits of every pass; bit 1 = record a per-stage device timeline.
  * Two more bits exercise the error path of the bounded device waits without hanging anything.
  * ASD_DEBUG_SHORT_WAITS: every wait of the pass kernel (ring slots, grid barrier) gives up after about a
- * millisecond instead of about two seconds. ASD_DEBUG_MISSING_ARRIVAL: the grid barrier in front of the last
- * stage of a pass waits for one arrival more than there are CTAs, so it can only end by its budget; the pass then
- * still runs to its end, and the call that launched it returns ASD_ERR_DEVICE_TIMEOUT with the stage and the CTA in
+ * millisecond instead of about two seconds. ASD_DEBUG_MISSING_ARRIVAL: the grid barrier in front of the stage
+ * that finishes the cosine similarities of a pass waits for one arrival more than there are CTAs, so it can only
+ * end by its budget; the pass then still runs to its end, and the call that launched it returns ASD_ERR_DEVICE_TIMEOUT with the stage and the CTA in
  * asd_last_error. The error stays set (every later pass returns it too) until asd_reset. */
 #define ASD_DEBUG_LOGITS 1
 #define ASD_DEBUG_TRACE 2
 #define ASD_DEBUG_SHORT_WAITS 4
 #define ASD_DEBUG_MISSING_ARRIVAL 8
+#define ASD_DEBUG_NO_TAGGED_HANDOFF 16 /* one- and two-row passes synchronise at the grid barrier like the others (for comparison) */
 int asd_set_debug(asd_ctx* ctx, int32_t flags);
 /* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][12][n_ctas]. Entries 0-3 are device
  * timestamps in ns of every CTA: 0 = stage entered, 1 = inputs of the stage ready (previous stage finished on

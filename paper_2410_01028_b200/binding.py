@@ -238,10 +238,11 @@ class Decoder:
         self._check(lib().asd_get_positions(self._ctx, ctypes.byref(a), ctypes.byref(b)), "asd_get_positions")
         return a.value, b.value
 
-    def set_debug(self, record_logits=True, trace=False, short_waits=False, missing_arrival=False):
+    def set_debug(self, record_logits=True, trace=False, short_waits=False, missing_arrival=False, no_tagged_handoff=False):
         """record_logits / trace: see asd_set_debug. short_waits and missing_arrival exercise the bounded device waits:
         with both set, the next pass ends with ASD_ERR_DEVICE_TIMEOUT after about a millisecond (see include/asd.h)."""
-        flags = (1 if record_logits else 0) | (2 if trace else 0) | (4 if short_waits else 0) | (8 if missing_arrival else 0)
+        flags = ((1 if record_logits else 0) | (2 if trace else 0) | (4 if short_waits else 0) | (8 if missing_arrival else 0)
+                 | (16 if no_tagged_handoff else 0))
         self._check(lib().asd_set_debug(self._ctx, ctypes.c_int32(flags)), "asd_set_debug")
 
     def set_sampling(self, temperature, seed=0):

@@ -130,7 +130,7 @@ struct PassPlan {
 static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan* pl) {
     const int kvd = c.n_kv_heads * c.head_dim;
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
-    const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 1;
+    const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 2;
     // per-pair partial sums; when a CTA has fewer than 8 groups of 8 pairs up to 15 warps keep copies (at most 15 / groups
     // copies of at most 8 * groups pairs: 120 pairs in all)
     const size_t psum = ((size_t)std::max<long long>(np_max, 120) * 2 * M * 4 + 15) & ~(size_t)15;
@@ -172,7 +172,7 @@ struct Layout {
     size_t embed, lm_head, final_norm, layers, layer_stride;
     size_t l_attn_norm, l_wqkv, l_wo, l_mlp_norm, l_wgu, l_wd;  // offsets inside one layer block
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
-    size_t x, q, a, t, part_acc, part_ml, partials, counters, cosv, sumcos;
+    size_t x, q, a, t, xl, al, tl, part_acc, part_ml, partials, counters, cosv, sumcos;
     size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits, probs_p, probs_q;
     size_t stage_tab, tmaps, sync_words, trace, resid_tab;
     int max_stages;
@@ -243,6 +243,10 @@ static Layout make_layout(const asd_config& c) {
     L.q = take(kPassMaxRows * d * 2);
     L.a = take(kPassMaxRows * d * 2);
     L.t = take(kPassMaxRows * f * 2);
+    // the same three activations as (value, tag) words for the one- and two-row passes (see pass.cuh, "tagged handoff")
+    L.xl = take((size_t)2 * d * 8);
+    L.al = take((size_t)2 * (d / 2) * 8);
+    L.tl = take((size_t)2 * (f / 2) * 8);
     L.chunk_stride = (int)((S + kAttnChunk - 1) / kAttnChunk);
     L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * c.head_dim * 4);
     L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * 2 * 4);
@@ -316,6 +320,7 @@ struct asd_ctx {
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, last_had_lm_head = false, trace = false;
     bool short_waits = false, inject_missing_arrival = false;  // test hooks of the bounded device waits (asd_set_debug)
+    bool no_tagged_handoff = false;  // asd_set_debug: one- and two-row passes use the grid barrier like the others
     // sampling (temperature > 0): every token is drawn; the draft steps of a round keep their distributions for the verify
     double temperature = 0.0;
     uint64_t seed = 0;
@@ -331,6 +336,7 @@ struct asd_ctx {
     asd_stats stats{};
     int32_t* pinned = nullptr;  // small host staging buffer
     uint32_t bar_base = 0;      // value of the grid-barrier counter at the start of the next pass
+    uint32_t pass_tag = 0x1000; // tag of stage 0 of the next pass in the tagged handoff buffers (never 0: the workspace starts zeroed)
     int n_stages_full = 0, n_stages_draft = 0, n_resid_full = 0, n_resid_draft = 0;
     std::vector<cudaEvent_t> events;
     size_t events_used = 0;
@@ -473,6 +479,7 @@ static int build_stage_tables(asd_ctx* x) {
     for (int which = 0; which < 2; ++which) {
         StageDesc* t = tab.data() + (size_t)which * ly.max_stages;
         int n = 0, nr = 0;
+        int x_writer = 0;  // index of the stage that wrote the current hidden state (stage 0 = embedding)
         ResidOut* ro = resid.data() + (size_t)which * max_resid;
         t[n] = StageDesc{};
         t[n++].type = kStEmbed;
@@ -486,6 +493,7 @@ static int build_stage_tables(asd_ctx* x) {
                 q.W = lw + ly.l_wqkv;
                 q.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_attn_norm);
                 q.k_cache = kc, q.v_cache = vc;
+                q.src_stage = x_writer;
                 t[n++] = q;
                 StageDesc a{};
                 a.type = kStAttn, a.layer = l;
@@ -496,7 +504,9 @@ static int build_stage_tables(asd_ctx* x) {
                 o.type = kStOproj, o.layer = l, o.n_rows = d, o.n_in = d;
                 o.W = lw + ly.l_wo;
                 o.resid_slot = nr;
+                o.src_stage = x_writer;
                 ro[nr++] = ResidOut{cosv + (size_t)(0 * L + l) * kPassMaxRows, x->at<double>(ly.sumcos) + l};
+                x_writer = n;
                 t[n++] = o;
             }
             if (!(which && x->skip_mlp[l])) {
@@ -504,12 +514,15 @@ static int build_stage_tables(asd_ctx* x) {
                 g.type = kStGateUp, g.layer = l, g.n_rows = 2 * f, g.n_in = d;
                 g.W = lw + ly.l_wgu;
                 g.gain = reinterpret_cast<const __nv_bfloat16*>(lw + ly.l_mlp_norm);
+                g.src_stage = x_writer;
                 t[n++] = g;
                 StageDesc w{};
                 w.type = kStDown, w.layer = l, w.n_rows = d, w.n_in = f;
                 w.W = lw + ly.l_wd;
                 w.resid_slot = nr;
+                w.src_stage = x_writer;
                 ro[nr++] = ResidOut{cosv + (size_t)(1 * L + l) * kPassMaxRows, x->at<double>(ly.sumcos) + L + l};
+                x_writer = n;
                 t[n++] = w;
             }
         }
@@ -520,6 +533,7 @@ static int build_stage_tables(asd_ctx* x) {
         h.type = kStLmHead, h.layer = L, h.n_rows = c.vocab, h.n_in = d;
         h.W = x->ws + ly.lm_head;
         h.gain = x->at<__nv_bfloat16>(ly.final_norm);
+        h.src_stage = x_writer;
         t[n++] = h;
         (which ? x->n_stages_draft : x->n_stages_full) = n;
         (which ? x->n_resid_draft : x->n_resid_full) = nr;
@@ -562,6 +576,8 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.q = x->at<__nv_bfloat16>(ly.q);
     p.a = x->at<__nv_bfloat16>(ly.a);
     p.t = x->at<__nv_bfloat16>(ly.t);
+    p.xl = x->at<uint2>(ly.xl), p.al = x->at<uint2>(ly.al), p.tl = x->at<uint2>(ly.tl);
+    p.pass_tag = x->pass_tag;
     p.part_acc = x->at<float>(ly.part_acc);
     p.part_ml = x->at<float>(ly.part_ml);
     p.attn_counters = x->at<unsigned>(ly.counters) + 64;
@@ -591,9 +607,14 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.ns_magic = (unsigned)((1ull << 32) / (unsigned)pl.ns + 1);
     p.off_bars = pl.off_bars, p.off_misc = pl.off_misc, p.off_psum = pl.off_psum, p.off_reg_a = pl.off_reg_a;
     p.xs_bytes = pl.xs_bytes;
+    // tagged handoff: one- and two-row passes whose activation window holds whole rows (always so on the benchmark shapes)
+    p.use_ll = (!x->no_tagged_handoff && M <= 2 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
+                (long long)pass_wseg(M, pl.xs_bytes) * kSegK >= std::max(d, f)) ? 1 : 0;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));
     x->bar_base += (uint32_t)p.n_stages * (uint32_t)grid;
+    x->pass_tag += (uint32_t)ly.max_stages + 1u;
+    if (x->pass_tag < 0x1000u) x->pass_tag = 0x1000u;  // wrapped around
     x->stats.kernel_launches += 1;
 
     // algorithmic bytes of the pass: weights of the stages that ran, plus K/V read by the kept attention sublayers
@@ -784,14 +805,18 @@ extern "C" const char* asd_last_error(asd_ctx* x) { return x ? x->err.c_str() : 
 // block R rows x 64 bytes (8 blocks, fewer in the last segment). Inputs past n_in are zero.
 template <class RowFn, class PairFn>
 static int upload_packed(asd_ctx* x, unsigned char* dev_dst, size_t n_rows, size_t n_in, RowFn row, PairFn pair_rows_of,
-                         std::vector<unsigned char>& staging) {
+                         std::vector<unsigned char>& staging, size_t pair_align = 1) {
     const size_t n_pairs = (n_rows + 1) / 2, row_blocks = (n_in + 31) / 32, n_seg = (n_in + kSegK - 1) / kSegK;
     const size_t total = n_pairs * row_blocks * 128;
     const int G = x->dev->num_sms;
     staging.assign(total, 0);
 #pragma omp parallel for schedule(static)
     for (int b = 0; b < G; ++b) {
-        const size_t pair0 = (size_t)b * n_pairs / G, pair1 = (size_t)(b + 1) * n_pairs / G, np = pair1 - pair0;
+        // (the same split as cta_pairs() of the pass kernel; W_gu's boundaries are even so that two neighbouring SwiGLU
+        // outputs, which share one tagged word, always belong to the same CTA)
+        const size_t units = n_pairs / pair_align;
+        const size_t pair0 = (size_t)b * units / G * pair_align, pair1 = (b + 1 == G) ? n_pairs : (size_t)(b + 1) * units / G * pair_align;
+        const size_t np = pair1 - pair0;
         unsigned char* slab = staging.data() + pair0 * row_blocks * 128;
         for (size_t sg = 0; sg < n_seg; ++sg) {
             const size_t nblk = std::min<size_t>(kSegBlocks, row_blocks - sg * kSegBlocks);
@@ -863,7 +888,7 @@ static int upload_weights(asd_ctx* x, const asd_host_weights& w) {
         // gate_i and up_i form a pair, so that one warp holds both operands of SwiGLU
         const uint16_t *wg = w.wg + (size_t)l * f * d, *wu = w.wu + (size_t)l * f * d;
         if ((rc = upload_packed(x, lw + ly.l_wgu, 2 * f, d, [&](size_t r) { return (r & 1) ? wu + (r / 2) * d : wg + (r / 2) * d; },
-                                plain_pair, staging)))
+                                plain_pair, staging, 2)))
             return rc;
         const uint16_t* wd = w.wd + (size_t)l * d * f;
         if ((rc = upload_packed(x, lw + ly.l_wd, d, f, [&](size_t r) { return wd + r * f; }, plain_pair, staging))) return rc;
@@ -1383,6 +1408,7 @@ extern "C" int asd_set_debug(asd_ctx* x, int32_t flags) {
     x->trace = (flags & 2) != 0;
     x->short_waits = (flags & ASD_DEBUG_SHORT_WAITS) != 0;
     x->inject_missing_arrival = (flags & ASD_DEBUG_MISSING_ARRIVAL) != 0;
+    x->no_tagged_handoff = (flags & ASD_DEBUG_NO_TAGGED_HANDOFF) != 0;
     return ASD_OK;
 }
 

@@ -59,6 +59,7 @@ struct StageDesc {
     __nv_bfloat16 *k_cache, *v_cache;   // this layer's cache [max_seq, kv_dim]
     const CUtensorMap *tm_k, *tm_v;     // tensor maps over the same
     int resid_slot;                     // residual stages: which block of per-CTA partial sums they write
+    int src_stage;                      // index of the stage that wrote the hidden state this stage reads (tagged handoff)
 };
 
 // where the cosine similarity of one residual stage goes (filled in by the finish stage of the pass)
@@ -76,6 +77,9 @@ struct PassParams {
     const float *rope_cos, *rope_sin;
     float* x;
     __nv_bfloat16 *q, *a, *t;
+    uint2 *xl, *al, *tl;  // tagged handoff (one- and two-row passes): hidden state [M][d], attention output [M][d/2], SwiGLU output [M][f/2]
+    uint32_t pass_tag;     // tag of stage 0 of this pass; stage s writes pass_tag + s
+    int use_ll;            // 1: this pass hands its activations over through the tagged buffers (host: M <= 2, d_model <= 5760)
     float *part_acc, *part_ml;
     unsigned* attn_counters;
     int chunk_stride;
@@ -85,7 +89,7 @@ struct PassParams {
     unsigned* fin_counter;
     unsigned* grid_bar;
     unsigned bar_base;
-    unsigned bar_extra_last;  // test hook: arrivals the LAST stage's barrier waits for beyond the grid size (0 in normal use)
+    unsigned bar_extra_last;  // test hook: arrivals the finish stage's barrier waits for beyond the grid size (0 in normal use)
     long long wait_cycles;    // cycle budget of every bounded wait of the pass
     int* err;
     const StageDesc* stages;
@@ -161,10 +165,14 @@ __device__ __forceinline__ void stage_pair_rows(int type, const PassParams& p, i
     }
 }
 
-__device__ __forceinline__ void cta_pairs(int n_rows, int& pair0, int& np) {
+// CTA b owns pairs [pair0, pair0 + np) of a matrix. W_gu is split at even pair indices (align = 2): two neighbouring
+// SwiGLU outputs share one tagged word of the handoff buffer and must come from the same CTA.
+__device__ __forceinline__ void cta_pairs(int n_rows, int type, int& pair0, int& np) {
     const int n_pairs = (n_rows + 1) >> 1;
-    pair0 = (int)((long long)blockIdx.x * n_pairs / gridDim.x);
-    const int pair1 = (int)((long long)(blockIdx.x + 1) * n_pairs / gridDim.x);
+    const int align = (type == kStGateUp) ? 2 : 1;
+    const int units = n_pairs / align;
+    pair0 = (int)((long long)blockIdx.x * units / gridDim.x) * align;
+    const int pair1 = (blockIdx.x + 1 == gridDim.x) ? n_pairs : (int)((long long)(blockIdx.x + 1) * units / gridDim.x) * align;
     np = pair1 - pair0;
 }
 
@@ -287,7 +295,7 @@ __device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& 
             c.tm_k = st.tm_k, c.tm_v = st.tm_v;
         } else {
             int pair0;
-            cta_pairs(st.n_rows, pair0, c.np);
+            cta_pairs(st.n_rows, st.type, pair0, c.np);
             c.n_oct = (c.np + kGrpPairs - 1) / kGrpPairs;
             c.n_items = c.n_oct * ((st.n_in + kSegK - 1) / kSegK);
             c.row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
@@ -420,10 +428,15 @@ __device__ __forceinline__ void trace_mark(const PassParams& p, int stage, int k
 // ============================================================================================ grid barrier
 __device__ __forceinline__ void consumers_sync() { bar_sync(1, kPassConsumers); }
 
-__device__ __forceinline__ void grid_arrive(const PassParams& p) {
+// release = false: the arrival only counts (nobody will wait for this stage before a later, releasing arrival of the
+// same CTA, whose release is cumulative); the CTA does not wait for its stores to be acknowledged.
+__device__ __forceinline__ void grid_arrive(const PassParams& p, bool release = true) {
     consumers_sync();
     // one release at GPU scope: cumulative over the writes of the whole CTA, which the barrier above ordered before it
-    if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p.grid_bar), "r"(1u) : "memory");
+    if (threadIdx.x == 0) {
+        if (release) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p.grid_bar), "r"(1u) : "memory");
+        else asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p.grid_bar), "r"(1u) : "memory");
+    }
 }
 __device__ __forceinline__ void grid_wait(const PassParams& p, unsigned target) {
     if (threadIdx.x == 0) {
@@ -461,8 +474,8 @@ __device__ __forceinline__ bool last_cta_consumers(unsigned* counter, int* flag_
 
 // Every stage starts by waiting for the previous stage of all CTAs. Whatever does not depend on activations (the
 // stage descriptor, index arithmetic, zeroing of partial sums, RMSNorm gains) is done before this wait.
-__device__ __forceinline__ void stage_begin(const PassParams& p, int s) {
-    if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x + (s == p.n_stages - 1 ? p.bar_extra_last : 0u));
+__device__ __forceinline__ void stage_begin(const PassParams& p, int s, unsigned extra = 0u) {
+    if (s > 0) grid_wait(p, p.bar_base + (unsigned)s * gridDim.x + extra);
     trace_mark(p, s, 1);
 }
 
@@ -475,6 +488,44 @@ __device__ __forceinline__ void top2_merge(float& v, int& i, float& s, float ov,
     }
 }
 
+// ============================================================================================ tagged handoff
+// One- and two-row passes (decode, draft, the commonest verify) spend a third of their time between weight streams,
+// and most of that in round trips to L2: a stage's last output is stored, a fence and an atomic arrive at the grid
+// barrier, every CTA polls the barrier word, and only then loads the activations. Here the activations carry their
+// own "ready" mark instead: every 4-byte value (one fp32 of the hidden state, or two bf16 of the attention / SwiGLU
+// output) is stored together with a 4-byte tag as ONE 8-byte word (8-byte scalar stores are single-copy atomic), the
+// tag naming the pass and the stage that wrote it. A consumer simply loads the words it needs and repeats the load
+// until every tag is the one it expects: one round trip after the slowest producer's store, no fence, no barrier.
+// A buffer is only overwritten by a stage that itself needed ALL outputs of a later stage than every reader's, so no
+// reader can still be waiting for the old contents (same ordering a barrier would give, carried by the data).
+__device__ __forceinline__ void ll_store(uint2* dst, uint32_t data, uint32_t tag) {
+    const unsigned long long v = ((unsigned long long)tag << 32) | (unsigned long long)data;
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(dst), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ll_load1(const uint2* src) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(src) : "memory");
+    return v;
+}
+__device__ __forceinline__ void ll_load2(const uint2* src, unsigned long long& a, unsigned long long& b) {  // 16-byte aligned
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(src) : "memory");
+}
+__device__ __forceinline__ bool ll_ready(unsigned long long v, uint32_t tag) { return (uint32_t)(v >> 32) == tag; }
+// after a load that found a stale tag: go on waiting? (bounded like every other wait of the kernel)
+__device__ __forceinline__ bool ll_keep_waiting(const PassParams& p, unsigned& spins, long long& t0, int stage) {
+    if (spins == 0) t0 = clock64();
+    if ((++spins & 31u) != 0) return true;
+    volatile int* err = p.err;
+    if (*err != kErrNone) return false;
+    if (clock64() - t0 > p.wait_cycles) {
+        if (atomicCAS(p.err, kErrNone, kErrGridWait) == kErrNone) {
+            p.err[1] = stage, p.err[2] = -1, p.err[3] = -1, p.err[4] = blockIdx.x, p.err[5] = threadIdx.x, p.err[6] = 77, p.err[7] = 0;
+        }
+        return false;
+    }
+    return true;
+}
+
 // ============================================================================================ GEMV stage
 template <int M>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
@@ -483,7 +534,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     const bool norm = (type == kStQkv || type == kStGateUp || type == kStLmHead);
     const int n_in = st.n_in, n_rows = st.n_rows;
     int pair0, np;
-    cta_pairs(n_rows, pair0, np);
+    cta_pairs(n_rows, type, pair0, np);
     const int n_seg = (n_in + kSegK - 1) / kSegK;
     const int n_oct = (np + kGrpPairs - 1) / kGrpPairs;  // groups of 16 rows (8 pairs; the last group may hold fewer)
     const int wseg = pass_wseg(M, p.xs_bytes);
@@ -494,6 +545,13 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
+    constexpr bool kLLCap = (M <= 2);
+    const bool ll = kLLCap && p.use_ll != 0;                      // activations come and go through the tagged buffers
+    const uint32_t tag_x = p.pass_tag + (uint32_t)st.src_stage;   // tag of the hidden state this stage reads
+    const uint32_t tag_in = p.pass_tag + (uint32_t)(stage - 1);   // tag of the attention / SwiGLU output (previous stage)
+    const uint32_t tag_out = p.pass_tag + (uint32_t)stage;        // tag of what this stage writes
+    unsigned ll_spins = 0;
+    long long ll_t0 = 0;
     // Fewer groups than warps (the d x d matrices leave ~28 rows to a CTA): several warps share a group, warp set ks
     // taking the segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are
     // added in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
@@ -528,10 +586,25 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             }
         }
     }
-    stage_begin(p, stage);
+    if (ll) trace_mark(p, stage, 1);  // no barrier: the loads below wait for exactly the words they need
+    else stage_begin(p, stage);
     if (kPre && (type == kStOproj || type == kStDown) && tid < np * 2 && 2 * pair0 + tid < n_rows) {
+        if (ll) {
+            unsigned long long raw[kPre ? M : 1] = {};
+            bool ok;
+            do {
+                ok = true;
 #pragma unroll
-        for (int m = 0; m < (kPre ? M : 0); ++m) pre[m] = __ldcg(p.x + (size_t)m * n_rows + 2 * pair0 + tid);
+                for (int m = 0; m < (kPre ? M : 0); ++m) raw[m] = ll_load1(p.xl + (size_t)m * n_rows + 2 * pair0 + tid);
+#pragma unroll
+                for (int m = 0; m < (kPre ? M : 0); ++m) ok = ok && ll_ready(raw[m], tag_x);
+            } while (!ok && ll_keep_waiting(p, ll_spins, ll_t0, stage));
+#pragma unroll
+            for (int m = 0; m < (kPre ? M : 0); ++m) pre[m] = __uint_as_float((uint32_t)raw[m]);
+        } else {
+#pragma unroll
+            for (int m = 0; m < (kPre ? M : 0); ++m) pre[m] = __ldcg(p.x + (size_t)m * n_rows + 2 * pair0 + tid);
+        }
     }
 
     // ---- RMSNorm statistics (same arithmetic for every row count). With one or two rows the hidden state read
@@ -543,13 +616,52 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 #pragma unroll
         for (int m = 0; m < M; ++m) ssq[m] = 0.f;
         if (keep) {
+            if (ll) {
+                // all of this thread's words of all rows in flight together; then only the 16-byte halves whose tags are
+                // still stale are loaded again, with a growing pause in between (a CTA that is early would otherwise
+                // re-read 32 KB per row and round and crowd the other CTAs' weight streams out of L2's ports)
+                unsigned long long raw[kKeepX ? M : 1][3][4] = {};
+                unsigned stale = 0u;  // bit (m * 3 + c) * 2 + h
+#pragma unroll
+                for (int m = 0; m < (kKeepX ? M : 0); ++m)
+#pragma unroll
+                    for (int c = 0; c < 3; ++c)
+                        if ((tid + c * kPassConsumers) * 4 < n_in) stale |= 3u << ((m * 3 + c) * 2);
+                for (;;) {
+#pragma unroll
+                    for (int m = 0; m < (kKeepX ? M : 0); ++m)
+#pragma unroll
+                        for (int c = 0; c < 3; ++c)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                if (stale & (1u << ((m * 3 + c) * 2 + h)))
+                                    ll_load2(p.xl + (size_t)m * n_in + (tid + c * kPassConsumers) * 4 + 2 * h, raw[m][c][2 * h], raw[m][c][2 * h + 1]);
+#pragma unroll
+                    for (int m = 0; m < (kKeepX ? M : 0); ++m)
+#pragma unroll
+                        for (int c = 0; c < 3; ++c)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                if ((stale & (1u << ((m * 3 + c) * 2 + h))) && ll_ready(raw[m][c][2 * h], tag_x) && ll_ready(raw[m][c][2 * h + 1], tag_x))
+                                    stale &= ~(1u << ((m * 3 + c) * 2 + h));
+                    if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
+                    __nanosleep(ll_spins < 4 ? 100u : 300u);
+                }
+#pragma unroll
+                for (int m = 0; m < (kKeepX ? M : 0); ++m)
+#pragma unroll
+                    for (int c = 0; c < 3; ++c)
+                        xr[m][c] = make_float4(__uint_as_float((uint32_t)raw[m][c][0]), __uint_as_float((uint32_t)raw[m][c][1]),
+                                               __uint_as_float((uint32_t)raw[m][c][2]), __uint_as_float((uint32_t)raw[m][c][3]));
+            }
 #pragma unroll
             for (int m = 0; m < M; ++m) {
 #pragma unroll
                 for (int c = 0; c < 3; ++c) {
                     const int i = (tid + c * kPassConsumers) * 4;
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (i < n_in) v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
+                    if (ll) v = xr[kKeepX ? m : 0][c];
+                    else if (i < n_in) v = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)m * n_in + i));
                     xr[kKeepX ? m : 0][c] = v;
                     if (i < n_in) {
                         float s = ssq[m];
@@ -726,6 +838,50 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                         }
                 }
             }
+        } else if (ll) {
+            // bf16 inputs as tagged words (two bf16 each): the window holds whole rows; two 8-element chunks per row and
+            // thread in flight together, repeated until every tag is the expected one
+            const uint2* src = (type == kStOproj) ? p.al : p.tl;
+            for (int i0 = tid * 8; i0 < wlen; i0 += 2 * kPassConsumers * 8) {
+                unsigned long long raw[kLLCap ? M : 1][2][4] = {};
+                unsigned stale = 0u;  // bit (m * 2 + u) * 2 + h
+#pragma unroll
+                for (int m = 0; m < (kLLCap ? M : 0); ++m)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+                        if (i0 + u * kPassConsumers * 8 < n_in) stale |= 3u << ((m * 2 + u) * 2);
+                for (;;) {
+#pragma unroll
+                    for (int m = 0; m < (kLLCap ? M : 0); ++m)
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                if (stale & (1u << ((m * 2 + u) * 2 + h)))
+                                    ll_load2(src + (((size_t)m * n_in + i0 + u * kPassConsumers * 8) >> 1) + 2 * h, raw[m][u][2 * h], raw[m][u][2 * h + 1]);
+#pragma unroll
+                    for (int m = 0; m < (kLLCap ? M : 0); ++m)
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                if ((stale & (1u << ((m * 2 + u) * 2 + h))) && ll_ready(raw[m][u][2 * h], tag_in) && ll_ready(raw[m][u][2 * h + 1], tag_in))
+                                    stale &= ~(1u << ((m * 2 + u) * 2 + h));
+                    if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
+                    __nanosleep(ll_spins < 4 ? 100u : 300u);
+                }
+#pragma unroll
+                for (int m = 0; m < (kLLCap ? M : 0); ++m)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int i = i0 + u * kPassConsumers * 8;
+                        if (i < wlen) {
+                            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                            if (i < n_in) v = make_uint4((uint32_t)raw[m][u][0], (uint32_t)raw[m][u][1], (uint32_t)raw[m][u][2], (uint32_t)raw[m][u][3]);
+                            *reinterpret_cast<uint4*>(xs + (size_t)m * xstride + i) = v;
+                        }
+                    }
+            }
         } else {
             for (int i = tid * 8; i < wlen; i += kPassConsumers * 8) {
                 const bool in = k0 + i < n_in;
@@ -849,20 +1005,53 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             if (row >= n_rows) continue;
             float xv[M];
 #pragma unroll
-            for (int m = 0; m < M; ++m) xv[m] = (kPre && e == tid) ? pre[kPre ? m : 0] : __ldcg(out + (size_t)m * n_rows + row);
+            for (int m = 0; m < M; ++m) {
+                if (kPre && e == tid) {
+                    xv[m] = pre[kPre ? m : 0];
+                } else if (ll) {  // (a CTA with more rows than threads: not on the benchmark shapes)
+                    unsigned long long raw;
+                    do raw = ll_load1(p.xl + (size_t)m * n_rows + row);
+                    while (!ll_ready(raw, tag_x) && ll_keep_waiting(p, ll_spins, ll_t0, stage));
+                    xv[m] = __uint_as_float((uint32_t)raw);
+                } else {
+                    xv[m] = __ldcg(out + (size_t)m * n_rows + row);
+                }
+            }
 #pragma unroll
             for (int m = 0; m < M; ++m) {
                 float v = psum[e * M + m];
                 for (int k = 1; k < S; ++k) v += psum[(size_t)k * copy_stride + e * M + m];
                 const float y = xv[m] + v;
-                out[(size_t)m * n_rows + row] = y;
+                if (ll) ll_store(p.xl + (size_t)m * n_rows + row, __float_as_uint(y), tag_out);
+                else out[(size_t)m * n_rows + row] = y;
                 s_loc[m][0] = fmaf(xv[m], y, s_loc[m][0]);
                 s_loc[m][1] = fmaf(xv[m], xv[m], s_loc[m][1]);
                 s_loc[m][2] = fmaf(y, y, s_loc[m][2]);
             }
         }
     }
-    for (int pl = resid ? np : tid; pl < np; pl += kPassConsumers) {
+    if (ll && type == kStGateUp) {
+        // pair0 and np are even: outputs pair0 + 2j and pair0 + 2j + 1 form one tagged word
+        for (int pj = tid; 2 * pj < np; pj += kPassConsumers) {
+#pragma unroll
+            for (int m = 0; m < M; ++m) {
+                uint32_t word = 0u;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int pl = 2 * pj + h;
+                    float va = psum[(pl * 2 + 0) * M + m], vb = psum[(pl * 2 + 1) * M + m];
+                    for (int k = 1; k < S; ++k) {
+                        va += psum[(size_t)k * copy_stride + (pl * 2 + 0) * M + m];
+                        vb += psum[(size_t)k * copy_stride + (pl * 2 + 1) * M + m];
+                    }
+                    const float t = va / (1.0f + expf(-va)) * vb;
+                    word |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(t)) << (16 * h);
+                }
+                ll_store(p.tl + (((size_t)m * (n_rows >> 1) + pair0) >> 1) + pj, word, tag_out);
+            }
+        }
+    }
+    for (int pl = (resid || (ll && type == kStGateUp)) ? np : tid; pl < np; pl += kPassConsumers) {
         int ra, rb;
         stage_pair_rows(type, p, pair0 + pl, ra, rb);
         const bool has_b = rb < n_rows;
@@ -1396,7 +1585,13 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                         uint2 o;
                         o.x = *reinterpret_cast<const uint32_t*>(&o01);
                         o.y = *reinterpret_cast<const uint32_t*>(&o23);
-                        *reinterpret_cast<uint2*>(p.a + (size_t)m * p.d_model + (size_t)head * hd + e4) = o;
+                        if (M <= 2 && p.use_ll) {
+                            uint2* dst = p.al + (((size_t)m * p.d_model + (size_t)head * hd + e4) >> 1);
+                            ll_store(dst, o.x, p.pass_tag + (uint32_t)stage);
+                            ll_store(dst + 1, o.y, p.pass_tag + (uint32_t)stage);
+                        } else {
+                            *reinterpret_cast<uint2*>(p.a + (size_t)m * p.d_model + (size_t)head * hd + e4) = o;
+                        }
                     }
                 }
             }
@@ -1454,10 +1649,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
                 const int m = i / d, e = i - m * d;
                 int t = __ldcg(p.tokens + m);
                 t = min(max(t, 0), p.vocab - 1);
-                p.x[i] = __bfloat162float(p.embed[(size_t)t * d + e]);
+                const float v = __bfloat162float(p.embed[(size_t)t * d + e]);
+                if (M <= 2 && p.use_ll) ll_store(p.xl + i, __float_as_uint(v), p.pass_tag);
+                else p.x[i] = v;
             }
         } else if (st.type == kStFinish) {
-            stage_begin(p, s);
+            stage_begin(p, s, p.bar_extra_last);  // (test hook: extra arrivals that never come)
             finish_stage<M>(p, sm);
         } else if (st.type == kStAttn) {
             attn_stage<M>(p, st, sm, gi, s);
@@ -1465,7 +1662,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
             gemv_stage<M>(p, st, sm, gi, s);
         }
         trace_mark(p, s, 3);
-        grid_arrive(p);
+        // With the tagged handoff only the attention and the finish stage still wait at the grid barrier: the arrival in
+        // front of one of them publishes everything this CTA has written so far, the others just count.
+        bool release = true;
+        if (M <= 2 && p.use_ll && s + 1 < p.n_stages) {
+            const int next = p.stages[s + 1].type;
+            release = (next == kStAttn || next == kStFinish);
+        }
+        grid_arrive(p, release);
     }
 }
 

@@ -231,7 +231,7 @@ int asd_get_last_logits(asd_ctx* ctx, int32_t* M, float* logits);
 #define ASD_DEBUG_TRACE 2
 #define ASD_DEBUG_SHORT_WAITS 4
 #define ASD_DEBUG_MISSING_ARRIVAL 8
-#define ASD_DEBUG_NO_TAGGED_HANDOFF 16 /* one- and two-row passes synchronise at the grid barrier like the others (for comparison) */
+#define ASD_DEBUG_NO_TAGGED_HANDOFF 16 /* one-row passes synchronise at the grid barrier like the others (for comparison) */
 int asd_set_debug(asd_ctx* ctx, int32_t flags);
 /* Timeline of the last pass (bit 1 of asd_set_debug): ns_out[n_stages][12][n_ctas]. Entries 0-3 are device
  * timestamps in ns of every CTA: 0 = stage entered, 1 = inputs of the stage ready (previous stage finished on

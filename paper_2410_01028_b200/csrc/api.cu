@@ -607,8 +607,9 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.ns_magic = (unsigned)((1ull << 32) / (unsigned)pl.ns + 1);
     p.off_bars = pl.off_bars, p.off_misc = pl.off_misc, p.off_psum = pl.off_psum, p.off_reg_a = pl.off_reg_a;
     p.xs_bytes = pl.xs_bytes;
-    // tagged handoff: one- and two-row passes whose activation window holds whole rows (always so on the benchmark shapes)
-    p.use_ll = (!x->no_tagged_handoff && M <= 2 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
+    // tagged handoff: one-row passes whose activation window holds whole rows (always so on the benchmark shapes). Measured
+    // against the barrier variant of the same kernel: 1 % faster at one row, 2 % slower at two rows (twice the words to poll).
+    p.use_ll = (!x->no_tagged_handoff && M == 1 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
                 (long long)pass_wseg(M, pl.xs_bytes) * kSegK >= std::max(d, f)) ? 1 : 0;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));

@@ -29,10 +29,17 @@ cudaError_t ASD_CAT(launch_gemv_m, ASD_M)(int epi, bool norm, const GemvParams& 
 }
 #endif
 
+// the one-row pass exists in two variants: activations handed over through tagged words (p.use_ll) or through
+// plain buffers behind the grid barrier
 cudaError_t ASD_CAT(launch_pass_m, ASD_M)(const PassParams& p, int grid, size_t smem, cudaStream_t s) {
     void* args[] = {const_cast<PassParams*>(&p)};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&pass_kernel<ASD_M>), dim3(grid), dim3(kPassThreads),
-                                       args, smem, s);
+    const void* fn = reinterpret_cast<const void*>(&pass_kernel<ASD_M, false>);
+#if ASD_M == 1
+    if (p.use_ll) fn = reinterpret_cast<const void*>(&pass_kernel<ASD_M, true>);
+#else
+    if (p.use_ll) return cudaErrorInvalidValue;
+#endif
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kPassThreads), args, smem, s);
 }
 
 // opt every instantiation in to large dynamic shared memory
@@ -49,7 +56,10 @@ cudaError_t ASD_CAT(configure_m, ASD_M)(int max_smem) {
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, true>))
     ASD_SET((gemv_kernel<ASD_M, kEpiResidual, false>))
 #endif
-    ASD_SET((pass_kernel<ASD_M>))
+    ASD_SET((pass_kernel<ASD_M, false>))
+#if ASD_M == 1
+    ASD_SET((pass_kernel<ASD_M, true>))
+#endif
 #undef ASD_SET
     return cudaSuccess;
 }

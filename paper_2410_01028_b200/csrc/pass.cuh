@@ -77,9 +77,9 @@ struct PassParams {
     const float *rope_cos, *rope_sin;
     float* x;
     __nv_bfloat16 *q, *a, *t;
-    uint2 *xl, *al, *tl;  // tagged handoff (one- and two-row passes): hidden state [M][d], attention output [M][d/2], SwiGLU output [M][f/2]
+    uint2 *xl, *al, *tl;  // tagged handoff (one-row passes): hidden state [d], attention output [d/2], SwiGLU output [f/2] as (value, tag) words
     uint32_t pass_tag;     // tag of stage 0 of this pass; stage s writes pass_tag + s
-    int use_ll;            // 1: this pass hands its activations over through the tagged buffers (host: M <= 2, d_model <= 5760)
+    int use_ll;            // 1: launch the kernel variant that hands activations over through the tagged buffers (host: one row, d_model <= 5760)
     float *part_acc, *part_ml;
     unsigned* attn_counters;
     int chunk_stride;
@@ -489,7 +489,7 @@ __device__ __forceinline__ void top2_merge(float& v, int& i, float& s, float ov,
 }
 
 // ============================================================================================ tagged handoff
-// One- and two-row passes (decode, draft, the commonest verify) spend a third of their time between weight streams,
+// One-row passes (decode, draft) spend a third of their time between weight streams,
 // and most of that in round trips to L2: a stage's last output is stored, a fence and an atomic arrive at the grid
 // barrier, every CTA polls the barrier word, and only then loads the activations. Here the activations carry their
 // own "ready" mark instead: every 4-byte value (one fp32 of the hidden state, or two bf16 of the attention / SwiGLU
@@ -527,7 +527,7 @@ __device__ __forceinline__ bool ll_keep_waiting(const PassParams& p, unsigned& s
 }
 
 // ============================================================================================ GEMV stage
-template <int M>
+template <int M, bool LL>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int type = st.type;
@@ -545,8 +545,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
 
     const float* xf = p.x;
     const __nv_bfloat16* xb = (type == kStOproj) ? p.a : p.t;
-    constexpr bool kLLCap = (M <= 2);
-    const bool ll = kLLCap && p.use_ll != 0;                      // activations come and go through the tagged buffers
+    constexpr bool kLLCap = LL;
+    constexpr bool ll = LL;                                       // activations come and go through the tagged buffers
     const uint32_t tag_x = p.pass_tag + (uint32_t)st.src_stage;   // tag of the hidden state this stage reads
     const uint32_t tag_in = p.pass_tag + (uint32_t)(stage - 1);   // tag of the attention / SwiGLU output (previous stage)
     const uint32_t tag_out = p.pass_tag + (uint32_t)stage;        // tag of what this stage writes
@@ -1262,7 +1262,7 @@ struct TileAddr {
     }
 };
 
-template <int M>
+template <int M, bool LL>
 __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, warp = tid >> 5;
     const int hd = p.head_dim;
@@ -1585,7 +1585,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                         uint2 o;
                         o.x = *reinterpret_cast<const uint32_t*>(&o01);
                         o.y = *reinterpret_cast<const uint32_t*>(&o23);
-                        if (M <= 2 && p.use_ll) {
+                        if (LL) {
                             uint2* dst = p.al + (((size_t)m * p.d_model + (size_t)head * hd + e4) >> 1);
                             ll_store(dst, o.x, p.pass_tag + (uint32_t)stage);
                             ll_store(dst + 1, o.y, p.pass_tag + (uint32_t)stage);
@@ -1601,7 +1601,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
 }
 
 // ============================================================================================ the kernel
-template <int M>
+template <int M, bool LL>
 __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_constant__ PassParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -1650,22 +1650,22 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
                 int t = __ldcg(p.tokens + m);
                 t = min(max(t, 0), p.vocab - 1);
                 const float v = __bfloat162float(p.embed[(size_t)t * d + e]);
-                if (M <= 2 && p.use_ll) ll_store(p.xl + i, __float_as_uint(v), p.pass_tag);
+                if (LL) ll_store(p.xl + i, __float_as_uint(v), p.pass_tag);
                 else p.x[i] = v;
             }
         } else if (st.type == kStFinish) {
             stage_begin(p, s, p.bar_extra_last);  // (test hook: extra arrivals that never come)
             finish_stage<M>(p, sm);
         } else if (st.type == kStAttn) {
-            attn_stage<M>(p, st, sm, gi, s);
+            attn_stage<M, LL>(p, st, sm, gi, s);
         } else {
-            gemv_stage<M>(p, st, sm, gi, s);
+            gemv_stage<M, LL>(p, st, sm, gi, s);
         }
         trace_mark(p, s, 3);
         // With the tagged handoff only the attention and the finish stage still wait at the grid barrier: the arrival in
         // front of one of them publishes everything this CTA has written so far, the others just count.
         bool release = true;
-        if (M <= 2 && p.use_ll && s + 1 < p.n_stages) {
+        if (LL && s + 1 < p.n_stages) {
             const int next = p.stages[s + 1].type;
             release = (next == kStAttn || next == kStFinish);
         }

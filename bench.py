@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the extra blocks of the line (headline variants, sampling, "
                     "the 8192-token and 13B-shaped workloads)")
+    ap.add_argument("--stage-timeline", action="store_true", help="also report the sublayer products of the kernel micro-benchmark "
+                    "configuration (d_model 2048..8192) as stages of the pass kernel, from its device timeline")
     ap.add_argument("--no-13b", action="store_true", help="skip the 13B-shaped workload of the extra blocks (26 GB of weights)")
     ap.add_argument("--gemv-microbench", action="store_true", help="also time the stand-alone fused GEMV kernel")
     ap.add_argument("--ablation", action="store_true", help="also time the rule subsets of the paper's ablation (Table 5) and "
@@ -422,6 +424,50 @@ def other_workload(torch, asd, name, args, hbm_peak, peak_kind, model=None):
     return res
 
 
+def stage_timeline(torch, asd, d, hbm_peak):
+    """The sublayer products of BASELINE config 2 (in = d -> out = d / 3d / 2 x 2.6875d, and in = 2.6875d -> out = d) as the
+    stages of the pass kernel: a 2-layer decoder of width d, the device timeline of one decode pass (1 row) and one verify
+    pass (5 rows), per stage the time from the end of the previous stage to the end of this one (everything a stage
+    costs: waiting for its inputs, RMSNorm prologue, weight stream, epilogue) and the weight bytes per that time."""
+    f = int(2.6875 * d)
+    shape = synth.DecoderShape(n_layers=2, d_model=d, n_heads=d // 128, head_dim=128, d_ffn=f, vocab=32000)
+    model = synth.make_model(shape, seed=3)
+    dec = asd.Decoder(shape, max_seq=160, max_draft=8)
+    dec.load_weights_host(model)
+    prompt = synth.make_prompt(shape.vocab, 64, seed=1)
+    t = dec.prefill(prompt)
+    dec.set_debug(record_logits=False, trace=True)
+    names = {1: ("qkv", "in d -> out 3d, rotary + K/V append", 2.0 * 3 * d * d), 3: ("o_proj", "in d -> out d, residual + cosine", 2.0 * d * d),
+             4: ("gate_up", "in d -> out 2 x 2.6875d, SwiGLU", 2.0 * 2 * f * d), 5: ("down", "in 2.6875d -> out d, residual + cosine", 2.0 * d * f)}
+    types = [0, 1, 2, 3, 4, 5, 1, 2, 3, 4, 5, 7, 6]
+    out = []
+    for rows in (1, 5):
+        best = {}
+        for rep in range(4):
+            if rows == 1:
+                t = dec.decode_step(t)
+            else:
+                a, o = dec.verify([t] + [1] * (rows - 1))
+                t = int(o[-1])
+            tr = dec.get_last_trace()
+            for s in range(6, 11):                       # the second layer: its first stage follows a full stage, not the embedding
+                if types[s] in names:
+                    period = float(np.median(tr[s, 3] - tr[s - 1, 3])) / 1e3
+                    stream = float(np.median(tr[s, 2] - tr[s, 7])) / 1e3
+                    key = types[s]
+                    if key not in best or period < best[key][0]:
+                        best[key] = (period, stream)
+        for key, (period, stream) in sorted(best.items()):
+            nm, what, nbytes = names[key]
+            out.append({"d": d, "rows": rows, "stage": nm, "shape": what, "MB": round(nbytes / 1e6, 1), "us": round(period, 2),
+                        "GBps": round(nbytes / period / 1e3, 1), "frac": round(nbytes / period / 1e3 / hbm_peak, 3),
+                        "stream_only_us": round(stream, 2)})
+    dec.close()
+    del dec
+    torch.cuda.empty_cache()
+    return out
+
+
 def rank_env():
     """(world size, rank, local rank) from the environment torch.distributed.run sets up; (1, 0, 0) without it."""
     return int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
@@ -544,7 +590,9 @@ def run_ours(args):
                 "how": "CUDA events around every launch inside the timed region, on the launching stream"}
     if args.gemv_microbench:
         roofline["fused_gemv_alone"] = gemv_sweep(torch, asd, hbm_peak)
-    elif args.gemv_shape:
+    if args.stage_timeline:
+        roofline["stage_timeline"] = [r for dd in (2048, 4096, 5120, 8192) for r in stage_timeline(torch, asd, dd, hbm_peak)]
+    if args.gemv_shape:
         n_in, n_rows, rows, epi = args.gemv_shape.split(",")
         epi = {"plain": asd.EPI_PLAIN, "swiglu": asd.EPI_SWIGLU, "residual": asd.EPI_RESIDUAL}[epi]
         roofline["fused_gemv_alone"] = [gemv_roofline(torch, asd, int(n_in), int(n_rows), int(rows), epi, hbm_peak)]

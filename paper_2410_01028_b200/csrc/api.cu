@@ -137,15 +137,16 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     // Activation window: the longest reduction dimension (in segments of 256 inputs) cut into as few windows as leave
-    // the ring 16 slots. Streaming does not get faster with more slots than that (measured), while every further
-    // window costs a stage of a multi-row pass a block-wide refill. One row always fits whole.
+    // the ring 20 slots. Every further window costs a stage of a multi-row pass a block-wide refill, every slot less
+    // costs bandwidth (one row, 7B shape: 24 slots 0.402 ms per 4 layers, 21: 0.409, 16: 0.422, 12: 0.481); 20 was the
+    // best trade for three and four rows. One row always fits whole.
     const size_t seg_max = ((size_t)std::max(c.d_model, c.d_ffn) + kSegK - 1) / kSegK;
     const long long fixed = 1024 + (long long)(psum + misc) + 2 * 64 * 8;
     size_t wseg_plan = seg_max;
     for (size_t nw = 1; nw <= seg_max; ++nw) {
         wseg_plan = (seg_max + nw - 1) / nw;
         const size_t bytes = (size_t)M * (wseg_plan * kSegK + kXsPad) * 2;
-        if ((long long)dv.max_smem - fixed - (long long)((bytes + 15) & ~(size_t)15) >= 16LL * kSlotBytes) break;
+        if ((long long)dv.max_smem - fixed - (long long)((bytes + 15) & ~(size_t)15) >= 20LL * kSlotBytes) break;
     }
     const int xs_bytes = (int)((size_t)M * (wseg_plan * kSegK + kXsPad) * 2);
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M, xs_bytes) * kSegK + kXsPad) * 2;

@@ -106,7 +106,7 @@ struct PassParams {
     unsigned ns_magic; // 2^32 / ns + 1, for exact division of ring item numbers by ns
     int attn_groups;   // 1 to 3 groups of 4 warps work on attention items
     int off_bars, off_misc, off_psum, off_reg_a;
-    int xs_bytes;      // bytes of the activation window (as few windows per stage as leave the ring 16 slots)
+    int xs_bytes;      // bytes of the activation window (as few windows per stage as leave the ring 20 slots)
 };
 
 constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)

@@ -121,7 +121,12 @@ typedef struct {
 
 typedef struct asd_ctx asd_ctx;
 
-/* Size of the device workspace a context of this shape needs (weights + KV cache + scratch); 0 on a bad config. */
+/* Size of the device workspace a context of this shape needs (weights + KV cache + scratch); 0 on a bad config.
+ * Where the tensor-core prompt path is available (head_dim 64 or 128) every sublayer matrix is kept twice, once in the
+ * packed order the decode passes stream and once row-major for the prompt GEMMs: about twice the bf16 weights, e.g.
+ * ~27 GB for the 7B shape and ~52 GB for the 13B shape before the KV cache, whatever asd_set_prefill_mode selects
+ * later. The packed copy is cut into one slab per SM of the device that is current when the weights are loaded, so
+ * a workspace image is not portable between devices with different SM counts. */
 size_t asd_workspace_bytes(const asd_config* cfg);
 
 /* Create a context inside dev_workspace (DEVICE, 256-byte aligned, >= asd_workspace_bytes(cfg)).

@@ -602,7 +602,7 @@ def run_ours(args):
     pf_tf = prefill_flops(shape, S) / (pf_ms * 1e-3) / 1e12
     prefill = {"ms": pf_ms, "bound": "tensor", "achieved": pf_tf, "peak": tf_sustained, "unit": "TFLOP/s",
                "frac": pf_tf / tf_sustained, "peak_kind": tf_kind + " sustained",
-               "what": "whole prompt pass (GEMMs on tcgen05, flash attention, row kernels, one decode pass for the last row)"}
+               "what": "whole prompt pass (GEMMs on tcgen05, flash attention, row kernels, the LM head stage of the pass kernel on the last row)"}
     if args.gemm_microbench:
         prefill["gemm_alone"] = gemm_roofline(torch, asd, shape)
     line = {

@@ -265,7 +265,7 @@ static Layout make_layout(const asd_config& c) {
     L.probs_p = take((size_t)kMaxRows * V * 8);  // sampling: the full model's distributions of a verify pass
     L.probs_q = take((size_t)kMaxRows * V * 8);  // sampling: the draft model's distributions of this round's draft steps
     L.max_stages = 5 * c.n_layers + 3;
-    L.stage_tab = take((size_t)2 * L.max_stages * sizeof(StageDesc));
+    L.stage_tab = take((size_t)3 * L.max_stages * sizeof(StageDesc));
     L.tmaps = take((size_t)2 * std::max(c.n_layers, 1) * sizeof(CUtensorMap));
     L.sync_words = take(256);
     L.resid_tab = take((size_t)2 * (2 * std::max(c.n_layers, 1)) * sizeof(ResidOut));
@@ -467,14 +467,15 @@ static int make_tensor_maps(asd_ctx* x) {
 }
 
 // Stage tables of the persistent pass kernel: table 0 = the full model M, table 1 = the draft model D (M
-// without the sublayers in the skip mask: they get no stage, so nothing is streamed or touched for them).
+// without the sublayers in the skip mask: they get no stage, so nothing is streamed or touched for them),
+// table 2 = the LM head alone on a hidden state that is already in place (last row of a dense prompt pass).
 static int build_stage_tables(asd_ctx* x) {
     const asd_config& c = x->c;
     const Layout& ly = x->lay;
     const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
     float* cosv = x->at<float>(ly.cosv);
     const CUtensorMap* maps = x->at<CUtensorMap>(ly.tmaps);
-    std::vector<StageDesc> tab((size_t)2 * ly.max_stages);
+    std::vector<StageDesc> tab((size_t)3 * ly.max_stages);
     const int max_resid = 2 * std::max(L, 1);
     std::vector<ResidOut> resid((size_t)2 * max_resid);
     for (int which = 0; which < 2; ++which) {
@@ -538,6 +539,12 @@ static int build_stage_tables(asd_ctx* x) {
         t[n++] = h;
         (which ? x->n_stages_draft : x->n_stages_full) = n;
         (which ? x->n_resid_draft : x->n_resid_full) = nr;
+        if (which == 0) {  // table 2: a finish stage without residual stages (nothing to do), then the LM head
+            StageDesc* t2 = tab.data() + (size_t)2 * ly.max_stages;
+            t2[0] = fin;
+            t2[1] = h;
+            t2[1].src_stage = 0;
+        }
     }
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.stage_tab, tab.data(), tab.size() * sizeof(StageDesc), cudaMemcpyHostToDevice, x->stream));
     ASD_CUDA(x, cudaMemcpyAsync(x->ws + ly.resid_tab, resid.data(), resid.size() * sizeof(ResidOut), cudaMemcpyHostToDevice, x->stream));
@@ -548,7 +555,7 @@ static int build_stage_tables(asd_ctx* x) {
 // tokens (DEVICE) feed rows at positions pos0..pos0+M-1. use_mask selects the draft model D. acc_sim adds the
 // rows' cosines to the prompt sums behind C_l. One cooperative launch of the persistent pass kernel.
 static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use_mask, bool acc_sim, bool lm_head,
-                    int* dev_argmax_out, bool accept, double* bytes_out) {
+                    int* dev_argmax_out, bool accept, double* bytes_out, bool head_only = false) {
     const asd_config& c = x->c;
     const Layout& ly = x->lay;
     const int d = c.d_model, f = c.d_ffn, kvd = x->kv_dim, L = c.n_layers;
@@ -585,16 +592,16 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.chunk_stride = ly.chunk_stride;
     p.partials = x->at<float>(ly.partials);
     p.resid = x->at<ResidOut>(ly.resid_tab) + (size_t)(use_mask ? 1 : 0) * (2 * std::max(L, 1));
-    p.n_resid = use_mask ? x->n_resid_draft : x->n_resid_full;
+    p.n_resid = head_only ? 0 : (use_mask ? x->n_resid_draft : x->n_resid_full);
     p.fin_counter = words + 0;
     p.grid_bar = words + 16;
     p.err = reinterpret_cast<int*>(words + 32);
     p.bar_base = x->bar_base;
     p.wait_cycles = x->short_waits ? kShortWaitCycles : kWaitCycles;
     p.bar_extra_last = x->inject_missing_arrival ? 1u : 0u;
-    const int table = use_mask ? 1 : 0;
+    const int table = head_only ? 2 : (use_mask ? 1 : 0);
     p.stages = x->at<StageDesc>(ly.stage_tab) + (size_t)table * ly.max_stages;
-    const int n_table = use_mask ? x->n_stages_draft : x->n_stages_full;
+    const int n_table = head_only ? 2 : (use_mask ? x->n_stages_draft : x->n_stages_full);
     p.n_stages = lm_head ? n_table : n_table - 1;
     p.row_tokens = accept ? dev_tokens : nullptr;
     p.argmax_out = dev_argmax_out ? dev_argmax_out : x->at<int>(ly.argmax);
@@ -610,7 +617,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.xs_bytes = pl.xs_bytes;
     // tagged handoff: one-row passes whose activation window holds whole rows (always so on the benchmark shapes). Measured
     // against the barrier variant of the same kernel: 1 % faster at one row, 2 % slower at two rows (twice the words to poll).
-    p.use_ll = (!x->no_tagged_handoff && M == 1 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
+    p.use_ll = (!x->no_tagged_handoff && !head_only && M == 1 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
                 (long long)pass_wseg(M, pl.xs_bytes) * kSegK >= std::max(d, f)) ? 1 : 0;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));
@@ -621,7 +628,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
 
     // algorithmic bytes of the pass: weights of the stages that ran, plus K/V read by the kept attention sublayers
     double bytes = 0;
-    for (int l = 0; l < L; ++l) {
+    for (int l = 0; l < L && !head_only; ++l) {
         if (!(use_mask && x->skip_attn[l]))
             bytes += 2.0 * ((double)(d + 2 * kvd) * d + (double)d * d) + 2.0 * 2.0 * kvd * (double)(pos0 + M);
         if (!(use_mask && x->skip_mlp[l])) bytes += 2.0 * 3.0 * (double)d * f;
@@ -979,8 +986,8 @@ static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which,
 }
 
 // Prompt rows [0, n) at positions pos0 + r through every layer of M as dense products: K/V appended to the cache,
-// each row's cosine similarity of every sublayer added to the sums behind C_l. No LM head: the caller feeds the
-// last prompt row through a one-row pass.
+// each row's cosine similarity of every sublayer added to the sums behind C_l. No LM head: the caller runs it on
+// the last row's hidden state, which stays in the residual buffer of the last chunk.
 static int prefill_dense(asd_ctx* x, const int32_t* dev_tokens, int n, int pos0) {
     const asd_config& c = x->c;
     const Layout& ly = x->lay;
@@ -1042,15 +1049,26 @@ static int prefill_device(asd_ctx* x, const int32_t* dev_tokens, int32_t n, int3
     int rc = new_event(x, &e0);
     if (rc) return rc;
     int last_rows = 0;
-    // Long prompts: all rows but the last as dense products on the tensor cores; the last row then takes a one-row
-    // pass, which also runs the LM head. Short prompts (and ASD_PREFILL_ROWS): row passes only.
+    // Long prompts: all rows as dense products on the tensor cores; the LM head then runs on the last row's hidden
+    // state as a pass of its own. Short prompts (and ASD_PREFILL_ROWS): row passes only.
     int n_dense = 0;
     if (x->prefill_mode == ASD_PREFILL_GEMM && x->lay.pf_rows == 0)
         return fail(x, ASD_ERR_ARG, "the dense prompt path needs head_dim 64 or 128 and at least one layer");
     if (x->lay.pf_rows > 0 && x->prefill_mode != ASD_PREFILL_ROWS && n > 1 &&
         (x->prefill_mode == ASD_PREFILL_GEMM || n - 1 >= kPrefillGemmMinRows))
-        n_dense = n - 1;
-    if (n_dense > 0 && (rc = prefill_dense(x, dev_tokens, n_dense, x->n_committed))) return rc;
+        n_dense = n;
+    if (n_dense > 0) {
+        if ((rc = prefill_dense(x, dev_tokens, n_dense, x->n_committed))) return rc;
+        // the last row's hidden state leaves the dense path's buffer for the pass kernel's, whose LM head stage alone runs
+        const int last_in_chunk = (n_dense - 1) % x->lay.pf_rows;
+        ASD_CUDA(x, cudaMemcpyAsync(x->at<float>(x->lay.x), x->at<float>(x->lay.pf_x) + (size_t)last_in_chunk * x->c.d_model,
+                                    (size_t)x->c.d_model * 4, cudaMemcpyDeviceToDevice, x->stream));
+        if ((rc = run_pass(x, 1, x->n_committed + n - 1, dev_tokens + n - 1, false, false, true, nullptr, false, nullptr, true))) return rc;
+        // "the last pass" reports the last prompt row: its cosines, which the dense path has computed, go where a pass leaves them
+        ASD_CUDA(x, cudaMemcpy2DAsync(x->at<float>(x->lay.cosv), (size_t)kPassMaxRows * 4, x->at<float>(x->lay.pf_cos) + last_in_chunk,
+                                      (size_t)x->lay.pf_rows * 4, 4, (size_t)2 * x->c.n_layers, cudaMemcpyDeviceToDevice, x->stream));
+        last_rows = 1;
+    }
     for (int c0 = n_dense, M = 0; c0 < n; c0 += M) {
         // row counts the pass kernel is built for: 16, or 1..9
         const int left = n - c0;

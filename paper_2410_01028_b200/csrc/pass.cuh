@@ -47,6 +47,9 @@ constexpr int kPassConsumerWarps = 15;
 constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
 constexpr unsigned kProducerNapNs = 50;             // the producer warp's sleep after a round without a free slot
+#ifndef ASD_FUSED_NORM_MIN
+#define ASD_FUSED_NORM_MIN 3
+#endif
 constexpr int kXsBudget = 40960;                    // most shared memory the attention scratch of all warp groups may take
 
 enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead, kStFinish };
@@ -527,6 +530,81 @@ __device__ __forceinline__ bool ll_keep_waiting(const PassParams& p, unsigned& s
 }
 
 // ============================================================================================ GEMV stage
+// RMSNorm of M whole rows into the activation window (three or more rows; rows of at most 12 x 480 elements), as a
+// function of its own so that its registers are its own: the rows are taken in batches of up to six, all loads of a
+// batch in flight together, and what was loaded for the statistics is normalised from registers, so a batch costs one
+// memory round trip. The arithmetic of a row is the one of the other paths: thread t adds the squares of its chunks
+// t, t + 480, t + 960 element by element, lanes by butterfly, warps in index order.
+template <int M>
+__device__ __noinline__ void norm_rows_into_window(const float* xf, const __nv_bfloat16* gain, int n_in, int wlen, int xstride, float eps,
+                                                   __nv_bfloat16* xs, float* red) {
+    constexpr int kBatches = (M + 5) / 6, kRB = (M + kBatches - 1) / kBatches;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint2 gv[3];
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        const int i = (tid + c * kPassConsumers) * 4;
+        gv[c] = make_uint2(0u, 0u);
+        if (i < n_in) gv[c] = *reinterpret_cast<const uint2*>(gain + i);
+    }
+#pragma unroll
+    for (int m0 = 0; m0 < M; m0 += kRB) {
+        float4 v[kRB][3];
+#pragma unroll
+        for (int u = 0; u < kRB; ++u)
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const int i = (tid + c * kPassConsumers) * 4;
+                v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (m0 + u < M && i < n_in) v[u][c] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
+            }
+#pragma unroll
+        for (int u = 0; u < kRB; ++u)
+            if (m0 + u < M) {
+                float s = 0.f;
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const int i = (tid + c * kPassConsumers) * 4;
+                    if (i < n_in) {
+                        s = fmaf(v[u][c].x, v[u][c].x, s);
+                        s = fmaf(v[u][c].y, v[u][c].y, s);
+                        s = fmaf(v[u][c].z, v[u][c].z, s);
+                        s = fmaf(v[u][c].w, v[u][c].w, s);
+                    }
+                }
+                s = warp_sum(s);
+                if (lane == 0) red[warp * (kPassMaxRows * 4) + m0 + u] = s;
+            }
+        bar_sync(1, kPassConsumers);
+#pragma unroll
+        for (int u = 0; u < kRB; ++u)
+            if (m0 + u < M) {
+                const int m = m0 + u;
+                float s = 0.f;
+#pragma unroll
+                for (int w = 0; w < kPassConsumerWarps; ++w) s += red[w * (kPassMaxRows * 4) + m];
+                const float inv = 1.0f / sqrtf(s / (float)n_in + eps);
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    const int i = (tid + c * kPassConsumers) * 4;
+                    if (i < wlen) {
+                        uint2 o = make_uint2(0u, 0u);
+                        if (i < n_in) {
+                            const float g0 = bf_lo(gv[c].x), g1 = bf_hi(gv[c].x), g2 = bf_lo(gv[c].y), g3 = bf_hi(gv[c].y);
+                            __nv_bfloat162 lo = __floats2bfloat162_rn(v[u][c].x * inv * g0, v[u][c].y * inv * g1);
+                            __nv_bfloat162 hi = __floats2bfloat162_rn(v[u][c].z * inv * g2, v[u][c].w * inv * g3);
+                            o.x = *reinterpret_cast<uint32_t*>(&lo);
+                            o.y = *reinterpret_cast<uint32_t*>(&hi);
+                        }
+                        *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
+                    }
+                }
+            }
+    }
+    for (int i = kPassConsumers * 12 + tid * 4; i < wlen; i += kPassConsumers * 4)  // zero padding past 5760
+        for (int m = 0; m < M; ++m) *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = make_uint2(0u, 0u);
+}
+
 template <int M, bool LL>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -611,7 +689,9 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     //      here stays in registers for the window fill below (one L2 round trip less per stage).
     float4 xr[kKeepX ? M : 1][3];
     float inv[M];
-    if (norm) {
+    constexpr bool kFusedNorm = (M >= ASD_FUSED_NORM_MIN);
+    const bool fused = kFusedNorm && short_rows && n_seg <= wseg;  // whole rows in one window: statistics and fill in one go below
+    if (norm && !fused) {
         float ssq[M];  // this thread's share of every row's sum of squares; per row the additions run in index order
 #pragma unroll
         for (int m = 0; m < M; ++m) ssq[m] = 0.f;
@@ -749,7 +829,9 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         const int k0 = w0 * kSegK;
         const int wlen = ws * kSegK;  // inputs in this window, including the zero padding past n_in
         consumers_sync();  // previous window fully consumed; psum zeroed; red free
-        if (keep) {  // a single window (n_in <= 5760): normalise the rows held in registers
+        if (fused) {
+            norm_rows_into_window<M>(xf, st.gain, n_in, wlen, xstride, p.eps, xs, red);
+        } else if (keep) {  // a single window (n_in <= 5760): normalise the rows held in registers
 #pragma unroll
             for (int c = 0; c < 3; ++c) {
                 const int i = (tid + c * kPassConsumers) * 4;

@@ -93,7 +93,7 @@ def test_tiny_prompt_through_the_dense_path_matches_oracle(tiny_model, tiny_prom
     ca_o, cm_o, n_o = orc.similarity()
     assert n_g == n_o == 32
     assert np.abs(ca_g - ca_o).max() <= COS_TOL and np.abs(cm_g - cm_o).max() <= COS_TOL
-    # the last prompt row went through a one-row pass on top of the cache the dense path wrote
+    # the last prompt row: cosines from the dense path, logits from the LM-head stage of the pass kernel on its hidden state
     ca, cm = dec.get_last_cosines()
     assert ca.shape[1] == 1
     assert_cos_close(ca, last["cos_attn"][:, -1:])

@@ -47,9 +47,6 @@ constexpr int kPassConsumerWarps = 15;
 constexpr int kPassConsumers = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumers + 32;  // + one producer warp
 constexpr unsigned kProducerNapNs = 50;             // the producer warp's sleep after a round without a free slot
-#ifndef ASD_FUSED_NORM_MIN
-#define ASD_FUSED_NORM_MIN 3
-#endif
 constexpr int kXsBudget = 40960;                    // most shared memory the attention scratch of all warp groups may take
 
 enum StageType : int { kStEmbed = 0, kStQkv, kStAttn, kStOproj, kStGateUp, kStDown, kStLmHead, kStFinish };
@@ -530,7 +527,7 @@ __device__ __forceinline__ bool ll_keep_waiting(const PassParams& p, unsigned& s
 }
 
 // ============================================================================================ GEMV stage
-// RMSNorm of M whole rows into the activation window (three or more rows; rows of at most 12 x 480 elements), as a
+// RMSNorm of M whole rows into the activation window (two or more rows; rows of at most 12 x 480 elements), as a
 // function of its own so that its registers are its own: the rows are taken in batches of up to six, all loads of a
 // batch in flight together, and what was loaded for the statistics is normalised from registers, so a batch costs one
 // memory round trip. The arithmetic of a row is the one of the other paths: thread t adds the squares of its chunks
@@ -636,7 +633,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
     const int copy_stride = np * 2 * M;
     for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
-    constexpr bool kKeepX = (M <= 2);
+    constexpr bool kKeepX = (M == 1);
     const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
     uint2 gpre[3] = {make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)};  // this thread's RMSNorm gains
     const bool short_rows = norm && n_in <= kPassConsumers * 12;  // a thread owns at most three 4-element chunks of a row
@@ -685,11 +682,12 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         }
     }
 
-    // ---- RMSNorm statistics (same arithmetic for every row count). With one or two rows the hidden state read
-    //      here stays in registers for the window fill below (one L2 round trip less per stage).
+    // ---- RMSNorm statistics (same arithmetic for every row count). With one row the hidden state read here stays in
+    //      registers for the window fill below (one L2 round trip less per stage); two and more rows whose window
+    //      holds them whole take norm_rows_into_window() instead.
     float4 xr[kKeepX ? M : 1][3];
     float inv[M];
-    constexpr bool kFusedNorm = (M >= ASD_FUSED_NORM_MIN);
+    constexpr bool kFusedNorm = (M >= 2);
     const bool fused = kFusedNorm && short_rows && n_seg <= wseg;  // whole rows in one window: statistics and fill in one go below
     if (norm && !fused) {
         float ssq[M];  // this thread's share of every row's sum of squares; per row the additions run in index order
@@ -752,36 +750,6 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                         ssq[m] = s;
                     }
                 }
-            }
-        } else if (M <= 3 && n_in <= kPassConsumers * 12) {
-            // up to three rows x three chunks per thread in flight together: one memory round trip per three rows
-#pragma unroll
-            for (int m0 = 0; m0 < M; m0 += 3) {
-                float4 v[3][3];
-#pragma unroll
-                for (int u = 0; u < 3; ++u)
-#pragma unroll
-                    for (int c = 0; c < 3; ++c) {
-                        const int i = (tid + c * kPassConsumers) * 4;
-                        v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (m0 + u < M && i < n_in) v[u][c] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
-                    }
-#pragma unroll
-                for (int u = 0; u < 3; ++u)
-                    if (m0 + u < M) {
-                        float s = ssq[m0 + u];
-#pragma unroll
-                        for (int c = 0; c < 3; ++c) {
-                            const int i = (tid + c * kPassConsumers) * 4;
-                            if (i < n_in) {  // same order of additions as the one-row path: chunk by chunk, element by element
-                                s = fmaf(v[u][c].x, v[u][c].x, s);
-                                s = fmaf(v[u][c].y, v[u][c].y, s);
-                                s = fmaf(v[u][c].z, v[u][c].z, s);
-                                s = fmaf(v[u][c].w, v[u][c].w, s);
-                            }
-                        }
-                        ssq[m0 + u] = s;
-                    }
             }
         } else {
             // long rows: the loads of up to four rows are in flight together (one memory round trip per four rows and stride)
@@ -850,44 +818,6 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                             o.y = *reinterpret_cast<uint32_t*>(&hi);
                         }
                         *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
-                    }
-                }
-            }
-            for (int i = kPassConsumers * 12 + tid * 4; i < wlen; i += kPassConsumers * 4)  // zero padding past 5760
-                for (int m = 0; m < M; ++m) *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = make_uint2(0u, 0u);
-        } else if (M <= 3 && short_rows && w0 == 0 && wlen >= n_in) {
-            // the window holds whole rows: three rows x three chunks per thread in flight together, then normalised
-#pragma unroll
-            for (int m0 = 0; m0 < M; m0 += 3) {
-                float4 v[3][3];
-#pragma unroll
-                for (int u = 0; u < 3; ++u)
-#pragma unroll
-                    for (int c = 0; c < 3; ++c) {
-                        const int i = (tid + c * kPassConsumers) * 4;
-                        v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (m0 + u < M && i < n_in) v[u][c] = __ldcg(reinterpret_cast<const float4*>(xf + (size_t)(m0 + u) * n_in + i));
-                    }
-#pragma unroll
-                for (int c = 0; c < 3; ++c) {
-                    const int i = (tid + c * kPassConsumers) * 4;
-                    if (i < wlen) {
-                        const bool in = i < n_in;
-                        const uint2 gv = gpre[c];
-                        const float g0 = bf_lo(gv.x), g1 = bf_hi(gv.x), g2 = bf_lo(gv.y), g3 = bf_hi(gv.y);
-#pragma unroll
-                        for (int u = 0; u < 3; ++u)
-                            if (m0 + u < M) {
-                                const int m = m0 + u;
-                                uint2 o = make_uint2(0u, 0u);
-                                if (in) {
-                                    __nv_bfloat162 lo = __floats2bfloat162_rn(v[u][c].x * inv[m] * g0, v[u][c].y * inv[m] * g1);
-                                    __nv_bfloat162 hi = __floats2bfloat162_rn(v[u][c].z * inv[m] * g2, v[u][c].w * inv[m] * g3);
-                                    o.x = *reinterpret_cast<uint32_t*>(&lo);
-                                    o.y = *reinterpret_cast<uint32_t*>(&hi);
-                                }
-                                *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = o;
-                            }
                     }
                 }
             }

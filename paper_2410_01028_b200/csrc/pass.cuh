@@ -527,14 +527,14 @@ __device__ __forceinline__ bool ll_keep_waiting(const PassParams& p, unsigned& s
 }
 
 // ============================================================================================ GEMV stage
-// RMSNorm of M whole rows into the activation window (two or more rows; rows of at most 12 x 480 elements), as a
-// function of its own so that its registers are its own: the rows are taken in batches of up to six, all loads of a
+// RMSNorm of M whole rows into the activation window (two or more rows; rows of at most 12 x 480 elements), for most
+// row counts a function of its own so that its registers are its own: the rows are taken in batches of up to six, all loads of a
 // batch in flight together, and what was loaded for the statistics is normalised from registers, so a batch costs one
 // memory round trip. The arithmetic of a row is the one of the other paths: thread t adds the squares of its chunks
 // t, t + 480, t + 960 element by element, lanes by butterfly, warps in index order.
 template <int M>
-__device__ __noinline__ void norm_rows_into_window(const float* xf, const __nv_bfloat16* gain, int n_in, int wlen, int xstride, float eps,
-                                                   __nv_bfloat16* xs, float* red) {
+__device__ __forceinline__ void norm_rows_body(const float* xf, const __nv_bfloat16* gain, int n_in, int wlen, int xstride, float eps,
+                                               __nv_bfloat16* xs, float* red) {
     constexpr int kBatches = (M + 5) / 6, kRB = (M + kBatches - 1) / kBatches;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint2 gv[3];
@@ -602,6 +602,176 @@ __device__ __noinline__ void norm_rows_into_window(const float* xf, const __nv_b
         for (int m = 0; m < M; ++m) *reinterpret_cast<uint2*>(xs + (size_t)m * xstride + i) = make_uint2(0u, 0u);
 }
 
+// Called as a function by most row counts; with five and six rows the call itself (measured) costs more than the
+// registers it frees.
+template <int M>
+__device__ __noinline__ void norm_rows_call(const float* xf, const __nv_bfloat16* gain, int n_in, int wlen, int xstride, float eps,
+                                            __nv_bfloat16* xs, float* red) {
+    norm_rows_body<M>(xf, gain, n_in, wlen, xstride, eps, xs, red);
+}
+template <int M>
+__device__ __forceinline__ void norm_rows_into_window(const float* xf, const __nv_bfloat16* gain, int n_in, int wlen, int xstride, float eps,
+                                                      __nv_bfloat16* xs, float* red) {
+    if constexpr (M == 5 || M == 6) norm_rows_body<M>(xf, gain, n_in, wlen, xstride, eps, xs, red);
+    else norm_rows_call<M>(xf, gain, n_in, wlen, xstride, eps, xs, red);
+}
+
+// Epilogues of a GEMV stage with four or more activation rows, as functions of their own (their registers are their
+// own; everything they need comes as scalar arguments, so nothing is re-read from the parameter block or the stage
+// table). The (weight row or pair, activation row) items of the CTA are spread over all consumer threads instead of
+// giving a thread all M rows of its pair. Every item is computed exactly as the one-row path computes it, and the
+// sums that cross threads keep that path's shape (the cosine sums of activation row m: the lanes of a warp hold 32
+// consecutive weight rows and are added by the same butterfly, the warps' sums are added in ascending order of the
+// weight rows), so row m of an M-row pass stays bit-identical to a one-row pass. pre0 / pre1: what the first item of
+// the thread (W_qkv: rotary factors) or of the warp (residual stages: old hidden state) needs from global memory,
+// requested by the caller ahead of the weight stream.
+__device__ __forceinline__ float psum_total(const float* psum, int idx, int S, int copy_stride) {
+    float v = psum[idx];  // the copies of a partial sum (warp sets that shared a group) in the order 0, 1, ...
+    for (int k = 1; k < S; ++k) v += psum[(size_t)k * copy_stride + idx];
+    return v;
+}
+
+// residual add + cosine sums: item (m, j) = activation row m, weight rows 32 j .. 32 j + 31 of this CTA, one warp each
+template <int M>
+__device__ __noinline__ void epi_resid_rows(float* out, const float* psum, float* red, float* partials_dst, int n_rows, int pair0, int np,
+                                            int S, float pre0) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int copy_stride = np * 2 * M;
+    const int W = (np * 2 + 31) >> 5;
+    for (int it = warp; it < M * W; it += kPassConsumerWarps) {
+        const int m = it / W, j = it - m * W, e = j * 32 + lane, row = 2 * pair0 + e;
+        float sxy = 0.f, sxx = 0.f, syy = 0.f;
+        if (e < np * 2 && row < n_rows) {
+            const float xv = (it == warp) ? pre0 : __ldcg(out + (size_t)m * n_rows + row);
+            const float y = xv + psum_total(psum, e * M + m, S, copy_stride);
+            out[(size_t)m * n_rows + row] = y;
+            sxy = fmaf(xv, y, 0.f);
+            sxx = fmaf(xv, xv, 0.f);
+            syy = fmaf(y, y, 0.f);
+        }
+        sxy = warp_sum(sxy);
+        sxx = warp_sum(sxx);
+        syy = warp_sum(syy);
+        if (lane == 0) red[it * 4 + 0] = sxy, red[it * 4 + 1] = sxx, red[it * 4 + 2] = syy;
+    }
+    bar_sync(1, kPassConsumers);
+    if (tid < M * 3) {
+        const int m = tid / 3, q = tid - m * 3;
+        float tot = 0.f;
+        for (int j = 0; j < W; ++j) tot += red[(m * W + j) * 4 + q];
+        partials_dst[m * 4 + q] = tot;
+    }
+}
+
+// W_qkv: rotary embedding of the q and k pairs, bf16 rounding, q to its buffer and k, v to the cache rows pos0 + m
+template <int M>
+__device__ __noinline__ void epi_qkv_rows(const float* psum, int pair0, int np, int S, int pos0, int d_model, int kv_dim, int head_dim,
+                                          const float* rope_cos, const float* rope_sin, __nv_bfloat16* q, __nv_bfloat16* kc,
+                                          __nv_bfloat16* vc, float pre0, float pre1) {
+    const int tid = threadIdx.x;
+    const int copy_stride = np * 2 * M;
+    const int half = head_dim >> 1, nq = d_model >> 1, nk = kv_dim >> 1;
+    for (int it = tid; it < np * M; it += kPassConsumers) {
+        const int m = it / np, pl = it - m * np, pair = pair0 + pl;
+        const int base = pair < nq ? 0 : (pair < nq + nk ? d_model : d_model + kv_dim);
+        const int pp = pair < nq ? pair : (pair < nq + nk ? pair - nq : pair - nq - nk);
+        const int head = pp / half, jr = pp - head * half;
+        const int ra = base + head * head_dim + jr, rb = ra + half;
+        float va = psum_total(psum, (pl * 2 + 0) * M + m, S, copy_stride), vb = psum_total(psum, (pl * 2 + 1) * M + m, S, copy_stride);
+        const int pos = pos0 + m;
+        if (ra < d_model + kv_dim) {  // q or k: rotate the pair (j, j + head_dim/2) by pos * theta_j
+            const float c = (it == tid) ? pre0 : rope_cos[(size_t)pos * half + jr];
+            const float sn = (it == tid) ? pre1 : rope_sin[(size_t)pos * half + jr];
+            const float r0 = __fmaf_rn(va, c, -__fmul_rn(vb, sn));
+            const float r1 = __fmaf_rn(vb, c, __fmul_rn(va, sn));
+            va = r0;
+            vb = r1;
+        }
+        const __nv_bfloat16 ha = __float2bfloat16_rn(va), hb = __float2bfloat16_rn(vb);
+        if (ra < d_model) {
+            q[(size_t)m * d_model + ra] = ha;
+            q[(size_t)m * d_model + rb] = hb;
+        } else if (ra < d_model + kv_dim) {
+            kc[(size_t)pos * kv_dim + (ra - d_model)] = ha;
+            kc[(size_t)pos * kv_dim + (rb - d_model)] = hb;
+        } else {
+            vc[(size_t)pos * kv_dim + (ra - d_model - kv_dim)] = ha;
+            vc[(size_t)pos * kv_dim + (rb - d_model - kv_dim)] = hb;
+        }
+    }
+}
+
+// W_gu: SwiGLU of every (pair, row), bf16 rounding
+template <int M>
+__device__ __noinline__ void epi_gateup_rows(const float* psum, int pair0, int np, int S, __nv_bfloat16* t_out, int t_stride) {
+    const int copy_stride = np * 2 * M;
+    for (int it = threadIdx.x; it < np * M; it += kPassConsumers) {
+        const int m = it / np, pl = it - m * np;
+        const float va = psum_total(psum, (pl * 2 + 0) * M + m, S, copy_stride), vb = psum_total(psum, (pl * 2 + 1) * M + m, S, copy_stride);
+        const float t = va / (1.0f + expf(-va)) * vb;
+        t_out[(size_t)m * t_stride + (pair0 + pl)] = __float2bfloat16_rn(t);
+    }
+}
+
+// LM head: the warps are dealt to the activation rows (warp w serves rows w mod G, w mod G + G, ...); a row's (largest
+// logit, its lowest index, second-largest logit) does not depend on the order of the comparisons. lmp: this CTA's
+// block of the per-CTA results.
+template <int M>
+__device__ __noinline__ void epi_lmhead_rows(const float* psum, float* red, int pair0, int np, int S, int n_rows, float* logits_out, float* lmp) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int copy_stride = np * 2 * M;
+    constexpr int G = M < kPassConsumerWarps ? M : kPassConsumerWarps;
+    const int g = warp % G, wi = warp / G, nw = (kPassConsumerWarps - g + G - 1) / G;
+    for (int m = g; m < M; m += G) {
+        float bv = -INFINITY, sv = -INFINITY;
+        int bi = INT_MAX;
+        for (int pl = wi * 32 + lane; pl < np; pl += nw * 32) {
+            const int ra = 2 * (pair0 + pl), rb = ra + 1;
+            const bool has_b = rb < n_rows;
+            const float va = psum_total(psum, (pl * 2 + 0) * M + m, S, copy_stride), vb = psum_total(psum, (pl * 2 + 1) * M + m, S, copy_stride);
+            if (logits_out) {
+                logits_out[(size_t)m * n_rows + ra] = va;
+                if (has_b) logits_out[(size_t)m * n_rows + rb] = vb;
+            }
+            if (va > bv) {  // rows come in ascending order: an equal logit keeps the lower index
+                sv = bv, bv = va, bi = ra;
+            } else {
+                sv = fmaxf(sv, va);
+            }
+            if (has_b) {
+                if (vb > bv) {
+                    sv = bv, bv = vb, bi = rb;
+                } else {
+                    sv = fmaxf(sv, vb);
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            const float os = __shfl_xor_sync(0xffffffffu, sv, o);
+            top2_merge(bv, bi, sv, ov, oi, os);
+        }
+        if (lane == 0) {
+            red[warp * (kPassMaxRows * 4) + m * 4 + 0] = bv;
+            red[warp * (kPassMaxRows * 4) + m * 4 + 1] = __int_as_float(bi);
+            red[warp * (kPassMaxRows * 4) + m * 4 + 2] = sv;
+        }
+    }
+    bar_sync(1, kPassConsumers);
+    if (tid < M) {
+        float v = -INFINITY, sc = -INFINITY;
+        int i = INT_MAX;
+        for (int w = tid % G; w < kPassConsumerWarps; w += G)
+            top2_merge(v, i, sc, red[w * (kPassMaxRows * 4) + tid * 4 + 0], __float_as_int(red[w * (kPassMaxRows * 4) + tid * 4 + 1]),
+                       red[w * (kPassMaxRows * 4) + tid * 4 + 2]);
+        lmp[tid * 4 + 0] = v;
+        lmp[tid * 4 + 1] = __int_as_float(i);
+        lmp[tid * 4 + 2] = sc;
+    }
+}
+
 template <int M, bool LL>
 __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassSmem& sm, uint32_t& gi, int stage) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -647,8 +817,20 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     // One or two rows: what the epilogue will need from global memory is requested ahead of the weight stream
     // (the rotary factors of this thread's pair before the barrier, the old hidden state of its row after it),
     // so the epilogue does not wait for a memory round trip.
+    constexpr bool kSpreadEpi = (M >= 4);  // measured: spreading the epilogue's items over the threads pays from four rows on
     constexpr bool kPre = (M <= 2);
     float pre[kPre ? 2 * M : 1];
+    float pre0 = 0.f, pre1 = 0.f;  // spread epilogue: what the first item of this thread / warp needs (see the epi_*_rows functions)
+    if (kSpreadEpi && type == kStQkv && tid < np * M) {
+        const int m = tid / np;
+        int ra, rb;
+        stage_pair_rows(type, p, pair0 + (tid - m * np), ra, rb);
+        if (ra < p.d_model + p.kv_dim) {
+            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+            pre0 = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
+            pre1 = p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
+        }
+    }
     if (kPre && type == kStQkv && tid < np) {
         int ra, rb;
         stage_pair_rows(type, p, pair0 + tid, ra, rb);
@@ -663,6 +845,13 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     }
     if (ll) trace_mark(p, stage, 1);  // no barrier: the loads below wait for exactly the words they need
     else stage_begin(p, stage);
+    if (kSpreadEpi && (type == kStOproj || type == kStDown)) {
+        const int W = (np * 2 + 31) >> 5;
+        if (warp < M * W) {
+            const int m = warp / W, e = (warp - m * W) * 32 + lane;
+            if (e < np * 2 && 2 * pair0 + e < n_rows) pre0 = __ldcg(p.x + (size_t)m * n_rows + 2 * pair0 + e);
+        }
+    }
     if (kPre && (type == kStOproj || type == kStDown) && tid < np * 2 && 2 * pair0 + tid < n_rows) {
         if (ll) {
             unsigned long long raw[kPre ? M : 1] = {};
@@ -998,7 +1187,8 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         p.trace[((size_t)stage * kTraceEntries + 5) * gridDim.x + blockIdx.x] = cyc_work;
     }
 
-    // ---- epilogue: thread t owns pairs t, t+512, ... of this CTA and all M rows of them
+    if constexpr (!kSpreadEpi) {
+    // ---- epilogue of a pass of up to three rows: thread t owns pairs t, t+480, ... of this CTA and all M rows of them
     float s_loc[M][3];
     float best_v[M], sec_v[M];
     int best_i[M];
@@ -1182,6 +1372,21 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
             lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 1] = __int_as_float(i);
             lmp[((size_t)blockIdx.x * kPassMaxRows + tid) * 4 + 2] = sc;
         }
+    }
+    } else {
+        if (type == kStOproj || type == kStDown)
+            epi_resid_rows<M>(p.x, psum, red, p.partials + ((size_t)st.resid_slot * gridDim.x + blockIdx.x) * kPassMaxRows * 4, n_rows, pair0, np, S,
+                              pre0);
+        else if (type == kStQkv)
+            epi_qkv_rows<M>(psum, pair0, np, S, p.pos0, p.d_model, p.kv_dim, p.head_dim, p.rope_cos, p.rope_sin, p.q, st.k_cache, st.v_cache, pre0,
+                            pre1);
+        else if (type == kStGateUp)
+            epi_gateup_rows<M>(psum, pair0, np, S, p.t, n_rows >> 1);
+        else
+            epi_lmhead_rows<M>(psum, red, pair0, np, S, n_rows, p.logits_out,
+                               p.partials + ((size_t)p.n_resid * gridDim.x + blockIdx.x) * kPassMaxRows * 4);
+    }
+    if (type == kStLmHead) {
         if (last_cta_consumers(p.fin_counter, sm.flag)) {
             int* g = reinterpret_cast<int*>(red);
             for (int m = warp; m < M; m += kPassConsumerWarps) {  // a warp per row: lanes scan the per-CTA partials, then a butterfly; ties -> lowest index

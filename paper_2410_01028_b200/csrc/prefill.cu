@@ -394,6 +394,62 @@ __global__ void __launch_bounds__(kRowThreads) resid_norm_kernel(int d, float* x
     }
 }
 
+// The same with the row held in registers (rows of at most kRowThreads * 4 * NV elements, a multiple of 4): x and the
+// sublayer output are read once, 16 bytes per load, and the sums, the new hidden state and the normalised row all
+// come from those registers.
+template <int NV>
+__global__ void __launch_bounds__(kRowThreads) resid_norm_vec_kernel(int d, float* x, const float* c, const __nv_bfloat16* gain, float eps,
+                                                                    __nv_bfloat16* xn, float* cos_out) {
+    __shared__ float red[24];
+    const int r = blockIdx.x, nvec = d >> 2;
+    float4* xr = reinterpret_cast<float4*>(x + (size_t)r * d);
+    const float4* cr = reinterpret_cast<const float4*>(c + (size_t)r * d);
+    float4 y[NV], cv[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int i = threadIdx.x + v * kRowThreads;
+        y[v] = cv[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < nvec) y[v] = xr[i], cv[v] = cr[i];
+    }
+    float s[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int i = threadIdx.x + v * kRowThreads;
+        if (i < nvec) {
+            const float4 xv = y[v];
+            float4 o;
+            o.x = xv.x + cv[v].x, o.y = xv.y + cv[v].y, o.z = xv.z + cv[v].z, o.w = xv.w + cv[v].w;
+            s[0] = fmaf(xv.x, o.x, s[0]), s[1] = fmaf(xv.x, xv.x, s[1]), s[2] = fmaf(o.x, o.x, s[2]);
+            s[0] = fmaf(xv.y, o.y, s[0]), s[1] = fmaf(xv.y, xv.y, s[1]), s[2] = fmaf(o.y, o.y, s[2]);
+            s[0] = fmaf(xv.z, o.z, s[0]), s[1] = fmaf(xv.z, xv.z, s[1]), s[2] = fmaf(o.z, o.z, s[2]);
+            s[0] = fmaf(xv.w, o.w, s[0]), s[1] = fmaf(xv.w, xv.w, s[1]), s[2] = fmaf(o.w, o.w, s[2]);
+            xr[i] = o;
+            y[v] = o;
+        }
+    }
+    block_sum<3>(s, red);
+    if (threadIdx.x == 0) {
+        const double den = fmax(sqrt((double)s[1]) * sqrt((double)s[2]), 1e-30);
+        cos_out[r] = (float)((double)s[0] / den);
+    }
+    if (gain) {
+        const float inv = 1.0f / sqrtf(s[2] / (float)d + eps);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int i = threadIdx.x + v * kRowThreads;
+            if (i < nvec) {
+                const uint2 g = *reinterpret_cast<const uint2*>(gain + (size_t)i * 4);
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(y[v].x * inv * bf_lo(g.x), y[v].y * inv * bf_hi(g.x));
+                const __nv_bfloat162 hi = __floats2bfloat162_rn(y[v].z * inv * bf_lo(g.y), y[v].w * inv * bf_hi(g.y));
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t*>(&lo);
+                o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(xn + (size_t)r * d + (size_t)i * 4) = o;
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(32) sumcos_kernel(const float* cos_rows, int stride, int n_rows, double* sumcos) {
     const float* c = cos_rows + (size_t)blockIdx.x * stride;
     double acc = 0.0;
@@ -410,7 +466,13 @@ cudaError_t launch_embed_norm(const int* tokens, int n_rows, int d, int vocab, c
 }
 cudaError_t launch_resid_norm(int n_rows, int d, float* x, const float* c, const __nv_bfloat16* gain, float eps, __nv_bfloat16* xn,
                               float* cos_out, cudaStream_t s) {
-    resid_norm_kernel<<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    const int nv = (d + kRowThreads * 4 - 1) / (kRowThreads * 4);
+    if (d % 4 != 0 || nv > 8) resid_norm_kernel<<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    else if (nv <= 1) resid_norm_vec_kernel<1><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    else if (nv <= 2) resid_norm_vec_kernel<2><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    else if (nv <= 4) resid_norm_vec_kernel<4><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    else if (nv <= 5) resid_norm_vec_kernel<5><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    else resid_norm_vec_kernel<8><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
     return cudaGetLastError();
 }
 cudaError_t launch_sumcos(const float* cos_rows, int stride, int n_rows, int n_sub, double* sumcos, cudaStream_t s) {

@@ -173,7 +173,7 @@ struct Layout {
     size_t embed, lm_head, final_norm, layers, layer_stride;
     size_t l_attn_norm, l_wqkv, l_wo, l_mlp_norm, l_wgu, l_wd;  // offsets inside one layer block
     size_t rope_cos, rope_sin, kcache, vcache, kv_layer_stride;
-    size_t x, q, a, t, xl, al, tl, part_acc, part_ml, partials, counters, cosv, sumcos;
+    size_t x, q, a, t, xl, al, tl, ql, kl, vl, pl_acc, pl_ml, part_acc, part_ml, partials, counters, cosv, sumcos;
     size_t tok_in, draft_toks, gen_toks, prompt_toks, argmax, accept, logits, probs_p, probs_q;
     size_t stage_tab, tmaps, sync_words, trace, resid_tab;
     int max_stages;
@@ -244,11 +244,16 @@ static Layout make_layout(const asd_config& c) {
     L.q = take(kPassMaxRows * d * 2);
     L.a = take(kPassMaxRows * d * 2);
     L.t = take(kPassMaxRows * f * 2);
-    // the same three activations as (value, tag) words for the one- and two-row passes (see pass.cuh, "tagged handoff")
+    // the same activations as (value, tag) words for the one-row passes (see pass.cuh, "tagged handoff")
     L.xl = take((size_t)2 * d * 8);
     L.al = take((size_t)2 * (d / 2) * 8);
     L.tl = take((size_t)2 * (f / 2) * 8);
     L.chunk_stride = (int)((S + kAttnChunk - 1) / kAttnChunk);
+    L.ql = take((size_t)d * 8);
+    L.kl = take((size_t)kvd * 8);
+    L.vl = take((size_t)kvd * 8);
+    L.pl_acc = take((size_t)c.n_heads * L.chunk_stride * c.head_dim * 8);
+    L.pl_ml = take((size_t)c.n_heads * L.chunk_stride * 2 * 8);
     L.part_acc = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * c.head_dim * 4);
     L.part_ml = take((size_t)c.n_heads * L.chunk_stride * kPassMaxRows * 2 * 4);
     L.partials = take((size_t)(2 * c.n_layers + 1) * kMaxGemvGrid * kPassMaxRows * 4 * 4);
@@ -585,6 +590,8 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.a = x->at<__nv_bfloat16>(ly.a);
     p.t = x->at<__nv_bfloat16>(ly.t);
     p.xl = x->at<uint2>(ly.xl), p.al = x->at<uint2>(ly.al), p.tl = x->at<uint2>(ly.tl);
+    p.ql = x->at<uint2>(ly.ql), p.kl = x->at<uint2>(ly.kl), p.vl = x->at<uint2>(ly.vl);
+    p.pl_acc = x->at<uint2>(ly.pl_acc), p.pl_ml = x->at<uint2>(ly.pl_ml);
     p.pass_tag = x->pass_tag;
     p.part_acc = x->at<float>(ly.part_acc);
     p.part_ml = x->at<float>(ly.part_ml);
@@ -617,7 +624,7 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.xs_bytes = pl.xs_bytes;
     // tagged handoff: one-row passes whose activation window holds whole rows (always so on the benchmark shapes). Measured
     // against the barrier variant of the same kernel: 1 % faster at one row, 2 % slower at two rows (twice the words to poll).
-    p.use_ll = (!x->no_tagged_handoff && !head_only && M == 1 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 &&
+    p.use_ll = (!x->no_tagged_handoff && !head_only && M == 1 && d <= kPassConsumers * 12 && d % 8 == 0 && f % 8 == 0 && c.head_dim <= 256 &&
                 (long long)pass_wseg(M, pl.xs_bytes) * kSegK >= std::max(d, f)) ? 1 : 0;
     const int grid = x->dev->num_sms;
     ASD_CUDA(x, launch_pass(M, p, grid, pl.smem, s));

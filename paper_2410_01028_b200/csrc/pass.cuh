@@ -78,6 +78,8 @@ struct PassParams {
     float* x;
     __nv_bfloat16 *q, *a, *t;
     uint2 *xl, *al, *tl;  // tagged handoff (one-row passes): hidden state [d], attention output [d/2], SwiGLU output [f/2] as (value, tag) words
+    uint2 *ql, *kl, *vl;  // tagged handoff: this pass's query [d], key and value [kv_dim], one bf16 per word
+    uint2 *pl_acc, *pl_ml;  // tagged handoff: attention partial results per (head, chunk): [head_dim] sums and (maximum, sum of weights)
     uint32_t pass_tag;     // tag of stage 0 of this pass; stage s writes pass_tag + s
     int use_ll;            // 1: launch the kernel variant that hands activations over through the tagged buffers (host: one row, d_model <= 5760)
     float *part_acc, *part_ml;
@@ -1289,9 +1291,17 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     vb = r1;
                 }
                 const __nv_bfloat16 ha = __float2bfloat16_rn(va), hb = __float2bfloat16_rn(vb);
+                if (ll) {  // the attention stage of this pass takes q, k, v from tagged words (k, v also go to the cache)
+                    uint2* dst = ra < p.d_model ? p.ql : (ra < p.d_model + p.kv_dim ? p.kl : p.vl);
+                    const int off = ra < p.d_model ? 0 : (ra < p.d_model + p.kv_dim ? p.d_model : p.d_model + p.kv_dim);
+                    ll_store(dst + (ra - off), (uint32_t)__bfloat16_as_ushort(ha), tag_out);
+                    ll_store(dst + (rb - off), (uint32_t)__bfloat16_as_ushort(hb), tag_out);
+                }
                 if (ra < p.d_model) {
-                    p.q[(size_t)m * p.d_model + ra] = ha;
-                    p.q[(size_t)m * p.d_model + rb] = hb;
+                    if (!ll) {
+                        p.q[(size_t)m * p.d_model + ra] = ha;
+                        p.q[(size_t)m * p.d_model + rb] = hb;
+                    }
                 } else if (ra < p.d_model + p.kv_dim) {
                     st.k_cache[(size_t)pos * p.kv_dim + (ra - p.d_model)] = ha;
                     st.k_cache[(size_t)pos * p.kv_dim + (rb - p.d_model)] = hb;
@@ -1490,7 +1500,11 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
     const int n_local = attn_local_items(p, M, n_chunks, first);
     const uint32_t gi0 = gi;
     gi += (uint32_t)(n_local * 2 * tile_slots);
-    stage_begin(p, stage);  // all consumer warps, also those without attention work
+    if (LL) trace_mark(p, stage, 1);  // tagged handoff: every item waits for exactly the words it needs
+    else stage_begin(p, stage);      // all consumer warps, also those without attention work
+    const uint32_t tag_in = p.pass_tag + (uint32_t)(stage - 1), tag_out = p.pass_tag + (uint32_t)stage;  // W_qkv's stage precedes this one
+    unsigned ll_spins = 0;
+    long long ll_t0 = 0;
     const int grp = warp >> 2;
     if (grp >= p.attn_groups) return;
 
@@ -1533,7 +1547,21 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         for (int u = 0; u < kQPerThread; ++u) {  // the first head's queries are requested before waiting for the tile
             const int i = gt + u * 128;
             const int m = i / hd, e = i - m * hd;
-            qreg[u] = (i < M * hd && q_head != kvh * group) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
+            qreg[u] = (!LL && i < M * hd && q_head != kvh * group) ? __ldcg(reinterpret_cast<const unsigned short*>(p.q) + (size_t)m * p.d_model + (size_t)(kvh * group) * hd + e) : 0;
+        }
+        // tagged handoff (one row): first look at this thread's words of q and of the fresh k and v; stale ones are asked for again where they are used
+        constexpr int kLLPer = LL ? 2 : 1;  // head_dim <= 256: at most two elements per thread
+        unsigned long long qraw[kLLPer] = {}, kraw[kLLPer] = {}, vraw[kLLPer] = {};
+        const bool has_fresh = LL && key0 <= p.pos0 && p.pos0 < key0 + kAttnChunk;
+        if (LL) {
+#pragma unroll
+            for (int u = 0; u < kLLPer; ++u) {
+                const int e = gt + u * 128;
+                if (e < hd) {
+                    if (q_head != kvh * group) qraw[u] = ll_load1(p.ql + (size_t)(kvh * group) * hd + e);
+                    if (has_fresh) kraw[u] = ll_load1(p.kl + (size_t)kvh * hd + e), vraw[u] = ll_load1(p.vl + (size_t)kvh * hd + e);
+                }
+            }
         }
         const int fresh0 = max(p.pos0, key0), fresh1 = min(last_pos, key0 + kAttnChunk - 1);
         const int n_fresh = fresh1 - fresh0 + 1;
@@ -1541,7 +1569,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         constexpr bool kVEarly = (M <= 2);
         constexpr int kVPre = kVEarly ? (M * 32 + 127) / 128 : 1;  // head_dim <= 256: at most 32 vectors per row
         uint4 vpre[kVPre];
-        if (kVEarly) {
+        if (kVEarly && !LL) {
 #pragma unroll
             for (int u = 0; u < kVPre; ++u) {
                 const int i = gt + u * 128;
@@ -1553,7 +1581,20 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
         }
         for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gk + t, stage, M * 1000 + j);
-        if (n_fresh > 0) {
+        if (LL) {
+            if (has_fresh) {  // this pass's key (element by element from the tagged words) over whatever the producer copied
+#pragma unroll
+                for (int u = 0; u < kLLPer; ++u) {
+                    const int e = gt + u * 128;
+                    if (e < hd) {
+                        while (!ll_ready(kraw[u], tag_in) && ll_keep_waiting(p, ll_spins, ll_t0, stage)) kraw[u] = ll_load1(p.kl + (size_t)kvh * hd + e);
+                        int sit, off;
+                        ta.locate(p.pos0 - key0, e >> 3, sit, off);
+                        *reinterpret_cast<unsigned short*>(slot_ptr(gk + sit) + off + (e & 7) * 2) = (unsigned short)kraw[u];
+                    }
+                }
+            }
+        } else if (n_fresh > 0) {
             for (int i = gt; i < n_fresh * vec_per_row; i += 128) {
                 const int fr = i / vec_per_row, c = i - fr * vec_per_row;
                 const int r = fresh0 + fr - key0;
@@ -1566,7 +1607,19 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         for (int g = 0; g < group; ++g) {
             const int head = kvh * group + g;
             bar_sync(bar_id, 128);  // patched tile visible; previous head's Ps / qs consumed
-            if (g == 0) {
+            if (LL) {
+                if (q_head != head) {
+#pragma unroll
+                    for (int u = 0; u < kLLPer; ++u) {
+                        const int e = gt + u * 128;
+                        if (e < hd) {
+                            if (g > 0) qraw[u] = ll_load1(p.ql + (size_t)head * hd + e);
+                            while (!ll_ready(qraw[u], tag_in) && ll_keep_waiting(p, ll_spins, ll_t0, stage)) qraw[u] = ll_load1(p.ql + (size_t)head * hd + e);
+                            qs[e] = __uint_as_float((uint32_t)qraw[u] << 16);
+                        }
+                    }
+                }
+            } else if (g == 0) {
                 if (q_head != head) {
 #pragma unroll
                     for (int u = 0; u < kQPerThread; ++u)
@@ -1652,7 +1705,20 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
             if (g == 0) {  // V tile: wait and patch once per item
                 for (int t = 0; t < tile_slots; ++t) ring_wait_full(p, sm, gv + t, stage, M * 1000 + 500 + j);
-                if (kVEarly) {
+                if (LL) {
+                    if (has_fresh) {
+#pragma unroll
+                        for (int u = 0; u < kLLPer; ++u) {
+                            const int e = gt + u * 128;
+                            if (e < hd) {
+                                while (!ll_ready(vraw[u], tag_in) && ll_keep_waiting(p, ll_spins, ll_t0, stage)) vraw[u] = ll_load1(p.vl + (size_t)kvh * hd + e);
+                                int sit, off;
+                                ta.locate(p.pos0 - key0, e >> 3, sit, off);
+                                *reinterpret_cast<unsigned short*>(slot_ptr(gv + sit) + off + (e & 7) * 2) = (unsigned short)vraw[u];
+                            }
+                        }
+                    }
+                } else if (kVEarly) {
 #pragma unroll
                     for (int u = 0; u < kVPre; ++u) {
                         const int i = gt + u * 128;
@@ -1677,12 +1743,15 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             bar_sync(bar_id, 128);
             if (gt < M) {
                 const float l = ((red[0 * kPassMaxRows + gt] + red[1 * kPassMaxRows + gt]) + red[2 * kPassMaxRows + gt]) + red[3 * kPassMaxRows + gt];
-                p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + gt) * 2 + 1] = l;
+                if (LL) ll_store(p.pl_ml + ((size_t)head * p.chunk_stride + chunk) * 2 + 1, __float_as_uint(l), tag_out);
+                else p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + gt) * 2 + 1] = l;
             }
             if (gt == 0) {
 #pragma unroll
-                for (int m = 0; m < M; ++m)
-                    p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * 2 + 0] = cmax[m];
+                for (int m = 0; m < M; ++m) {
+                    if (LL) ll_store(p.pl_ml + ((size_t)head * p.chunk_stride + chunk) * 2 + 0, __float_as_uint(cmax[m]), tag_out);
+                    else p.part_ml[(((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m) * 2 + 0] = cmax[m];
+                }
             }
             if (j == 0 && g == 0) trace_mark(p, stage, 4);
             // ---- P V: thread (c, kg) owns the 8 output dimensions of 16-byte chunk c for the keys kg, kg + 8, ... (one
@@ -1730,9 +1799,15 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                                     acc[u][d8] = v;
                                 }
                                 if (kg == 0 && active) {
-                                    float* dst = p.part_acc + (((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m0 + u) * hd + c * 8;
-                                    reinterpret_cast<float4*>(dst)[0] = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
-                                    reinterpret_cast<float4*>(dst)[1] = make_float4(acc[u][4], acc[u][5], acc[u][6], acc[u][7]);
+                                    if (LL) {
+                                        uint2* dst = p.pl_acc + ((size_t)head * p.chunk_stride + chunk) * hd + c * 8;
+#pragma unroll
+                                        for (int d8 = 0; d8 < 8; ++d8) ll_store(dst + d8, __float_as_uint(acc[u][d8]), tag_out);
+                                    } else {
+                                        float* dst = p.part_acc + (((size_t)head * p.chunk_stride + chunk) * kPassMaxRows + m0 + u) * hd + c * 8;
+                                        reinterpret_cast<float4*>(dst)[0] = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
+                                        reinterpret_cast<float4*>(dst)[1] = make_float4(acc[u][4], acc[u][5], acc[u][6], acc[u][7]);
+                                    }
                                 }
                             }
                     }
@@ -1746,6 +1821,63 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         const int jn = j + p.attn_groups;
         const bool report = (jn >= n_local) || ((first + jn) / n_chunks != kvh);
         bar_sync(bar_id, 128);
+        if (LL) {
+            // Tagged handoff: no ticket. The group that took the head's last chunk (the one with this pass's key) merges:
+            // it asks for the other chunks' partial results until their tags are this stage's (they come from items with
+            // lower numbers: other CTAs, or other groups and earlier rounds of this CTA, none of which waits for this one).
+            if (gt == 0) {
+                fence_proxy_async_smem();
+                for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
+            }
+            if (j == 0) trace_mark(p, stage, 6);
+            if (chunk == n_chunks - 1) {
+                for (int g = 0; g < group; ++g) {
+                    const int head = kvh * group + g;
+                    for (int e0 = 0; e0 < hd; e0 += 128) {  // one output dimension per thread (every lane runs the loop: shuffle below)
+                        const int e = e0 + gt;
+                        const bool act = e < hd;
+                        float mx = -INFINITY, l = 0.f, acc = 0.f;
+                        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+                            unsigned long long ra[8] = {}, rm[8] = {}, rl[8] = {};
+                            unsigned stale = 0u;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (act && c0 + i < n_chunks) stale |= 1u << i;
+                            for (;;) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    if (stale & (1u << i)) {
+                                        const size_t b = (size_t)head * p.chunk_stride + c0 + i;
+                                        ra[i] = ll_load1(p.pl_acc + b * hd + e);
+                                        ll_load2(p.pl_ml + b * 2, rm[i], rl[i]);
+                                    }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    if ((stale & (1u << i)) && ll_ready(ra[i], tag_out) && ll_ready(rm[i], tag_out) && ll_ready(rl[i], tag_out)) stale &= ~(1u << i);
+                                if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
+                                __nanosleep(100u);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (c0 + i < n_chunks) {  // same arithmetic as the merge of the other instantiations
+                                    const float cm = __uint_as_float((uint32_t)rm[i]);
+                                    const float mn = fmaxf(mx, cm);
+                                    const float s_old = expf(mx - mn), s_new = expf(cm - mn);
+                                    acc = __fmaf_rn(acc, s_old, __fmul_rn(__uint_as_float((uint32_t)ra[i]), s_new));
+                                    l = __fmaf_rn(l, s_old, __fmul_rn(__uint_as_float((uint32_t)rl[i]), s_new));
+                                    mx = mn;
+                                }
+                            }
+                        }
+                        const uint32_t ob = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__fdiv_rn(acc, l)));
+                        const uint32_t up = __shfl_down_sync(0xffffffffu, ob, 1);
+                        if (act && (gt & 1) == 0) ll_store(p.al + (((size_t)head * hd + e) >> 1), ob | (up << 16), tag_out);
+                    }
+                }
+            }
+            if (j == 0) trace_mark(p, stage, 7);
+            continue;
+        }
         if (gt == 0) {
             fence_proxy_async_smem();
             for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
@@ -1879,12 +2011,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
             gemv_stage<M, LL>(p, st, sm, gi, s);
         }
         trace_mark(p, s, 3);
-        // With the tagged handoff only the attention and the finish stage still wait at the grid barrier: the arrival in
-        // front of one of them publishes everything this CTA has written so far, the others just count.
+        // With the tagged handoff only the finish stage still waits at the grid barrier: the arrival in front of it
+        // publishes everything this CTA has written so far, the others just count.
         bool release = true;
         if (LL && s + 1 < p.n_stages) {
             const int next = p.stages[s + 1].type;
-            release = (next == kStAttn || next == kStFinish);
+            release = (next == kStFinish);
         }
         grid_arrive(p, release);
     }

@@ -131,10 +131,11 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     const int kvd = c.n_kv_heads * c.head_dim;
     const long long max_rows = std::max<long long>(std::max(c.vocab, 2 * c.d_ffn), std::max(c.d_model + 2 * kvd, c.d_model));
     const long long np_max = ((max_rows + 1) / 2 + dv.num_sms - 1) / dv.num_sms + 2;
+    if ((max_rows + 1) / 2 * dv.num_sms >= (1LL << 31)) return false;  // the kernel splits a matrix's pairs over the CTAs in 32-bit arithmetic
     // per-pair partial sums; when a CTA has fewer than 8 groups of 8 pairs up to 15 warps keep copies (at most 15 / groups
     // copies of at most 8 * groups pairs: 120 pairs in all)
     const size_t psum = ((size_t)std::max<long long>(np_max, 120) * 2 * M * 4 + 15) & ~(size_t)15;
-    const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 15) & ~(size_t)15;
+    const size_t misc = ((size_t)16 * kPassMaxRows * 4 * 4 + 32 + 64 * 4 + 8 * 4 * 4 + 15) & ~(size_t)15;  // reduction scratch, flags, slot generations, split table
     const size_t attn_scratch = ((size_t)M * c.head_dim * 4 + (size_t)M * kAttnChunk * 4 + 4 * kPassMaxRows * 4 + 16 + 15) & ~(size_t)15;
     // Activation window: the longest reduction dimension (in segments of 256 inputs) cut into as few windows as leave
     // the ring 20 slots. Every further window costs a stage of a multi-row pass a block-wide refill, every slot less
@@ -581,6 +582,9 @@ static int run_pass(asd_ctx* x, int M, int pos0, const int* dev_tokens, bool use
     p.embed = x->at<__nv_bfloat16>(ly.embed);
     p.d_model = d, p.vocab = c.vocab, p.kv_dim = kvd, p.head_dim = c.head_dim, p.n_heads = c.n_heads;
     p.n_kv_heads = c.n_kv_heads, p.d_ffn = f;
+    p.hd_shift = 0;
+    if ((c.head_dim & (c.head_dim - 1)) == 0)
+        while ((1 << p.hd_shift) < c.head_dim) ++p.hd_shift;
     p.eps = c.rms_eps;
     p.attn_scale = 1.0f / sqrtf((float)c.head_dim);
     p.rope_cos = x->at<float>(ly.rope_cos);

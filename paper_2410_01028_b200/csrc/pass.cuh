@@ -73,6 +73,7 @@ struct PassParams {
     const int* tokens;
     const __nv_bfloat16* embed;
     int d_model, vocab, kv_dim, head_dim, n_heads, n_kv_heads, d_ffn;
+    int hd_shift;  // log2(head_dim) when head_dim is a power of two, else 0 (divisions instead of shifts)
     float eps, attn_scale;
     const float *rope_cos, *rope_sin;
     float* x;
@@ -111,7 +112,7 @@ struct PassParams {
     int xs_bytes;      // bytes of the activation window (as few windows per stage as leave the ring 20 slots)
 };
 
-constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles)
+constexpr int kTraceEntries = 12;  // per stage and CTA: 0-7 consumer side, 8-10 producer side (first / last copy issued, stall cycles), 11 descriptor read
 constexpr int kSegK = 256;     // inputs per ring item (8 column blocks of 32; the last item of a row may hold fewer)
 constexpr int kBoxKeys = 64;   // keys per K/V box (one ring slot)
 constexpr int kGrpPairs = 8;   // pairs of weight rows per ring item: 16 rows, the M of one m16n8k16 tensor-core step
@@ -139,6 +140,7 @@ struct PassSmem {
     float* red;   // [16][kPassMaxRows*4]
     int* flag;    // [8]
     volatile unsigned* consumed;  // [64] generations of each ring slot that consumers have finished with
+    const int* split;             // [8][4] per stage type: this CTA's first pair, pair count, groups of 16 rows, warp sets per group
     float* psum;
     unsigned char* reg_a;
 };
@@ -158,7 +160,7 @@ __device__ __forceinline__ void stage_pair_rows(int type, const PassParams& p, i
             base = p.d_model + p.kv_dim;
             pp = pair - nq - nk;
         }
-        const int head = pp / half, j = pp - head * half;
+        const int head = p.hd_shift ? (pp >> (p.hd_shift - 1)) : pp / half, j = pp - head * half;
         ra = base + head * p.head_dim + j;
         rb = ra + half;
     } else {
@@ -172,9 +174,9 @@ __device__ __forceinline__ void stage_pair_rows(int type, const PassParams& p, i
 __device__ __forceinline__ void cta_pairs(int n_rows, int type, int& pair0, int& np) {
     const int n_pairs = (n_rows + 1) >> 1;
     const int align = (type == kStGateUp) ? 2 : 1;
-    const int units = n_pairs / align;
-    pair0 = (int)((long long)blockIdx.x * units / gridDim.x) * align;
-    const int pair1 = (blockIdx.x + 1 == gridDim.x) ? n_pairs : (int)((long long)(blockIdx.x + 1) * units / gridDim.x) * align;
+    const unsigned units = (unsigned)(n_pairs / align);  // units * gridDim.x < 2^32 (the host refuses larger matrices): 32-bit divisions
+    pair0 = (int)(blockIdx.x * units / gridDim.x) * align;
+    const int pair1 = (blockIdx.x + 1 == gridDim.x) ? n_pairs : (int)((blockIdx.x + 1) * units / gridDim.x) * align;
     np = pair1 - pair0;
 }
 
@@ -182,9 +184,9 @@ __device__ __forceinline__ void cta_pairs(int n_rows, int type, int& pair0, int&
 // [b*T/G, (b+1)*T/G): mostly chunks of one head, so queries, tickets and DRAM pages are reused.
 __device__ __forceinline__ int attn_local_items(const PassParams& p, int M, int& n_chunks, int& first) {
     n_chunks = (p.pos0 + M - 1) / kAttnChunk + 1;
-    const long long total = (long long)p.n_kv_heads * n_chunks;
-    first = (int)((long long)blockIdx.x * total / gridDim.x);
-    return (int)((long long)(blockIdx.x + 1) * total / gridDim.x) - first;
+    const unsigned total = (unsigned)(p.n_kv_heads * n_chunks);  // heads * chunks * CTAs stays far below 2^32
+    first = (int)(blockIdx.x * total / gridDim.x);
+    return (int)((blockIdx.x + 1) * total / gridDim.x) - first;
 }
 
 // ============================================================================================ ring protocol
@@ -282,7 +284,7 @@ struct ProdState {
 
 // move to the next stage that streams anything for this lane; false when the pass has no more
 template <int M>
-__device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& c, int lane) {
+__device__ __forceinline__ bool prod_next_stage(const PassParams& p, const PassSmem& sm, ProdState& c, int lane) {
     for (;;) {
         c.gi += (uint32_t)c.n_items;
         c.n_items = 0;
@@ -296,9 +298,9 @@ __device__ __forceinline__ bool prod_next_stage(const PassParams& p, ProdState& 
             c.n_items = n_local * 2 * (kAttnChunk / kBoxKeys) * nhb;
             c.tm_k = st.tm_k, c.tm_v = st.tm_v;
         } else {
-            int pair0;
-            cta_pairs(st.n_rows, st.type, pair0, c.np);
-            c.n_oct = (c.np + kGrpPairs - 1) / kGrpPairs;
+            const int pair0 = sm.split[st.type * 4 + 0];
+            c.np = sm.split[st.type * 4 + 1];
+            c.n_oct = sm.split[st.type * 4 + 2];
             c.n_items = c.n_oct * ((st.n_in + kSegK - 1) / kSegK);
             c.row_blocks = (st.n_in + 31) >> 5;  // 32-input column blocks per row
             c.slab = st.W + (size_t)pair0 * c.row_blocks * 128;
@@ -352,7 +354,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
     const uint64_t pol_stream = make_policy_evict_first();  // weights are read once per pass: do not let them age in L2
     ProdState c{};
     c.s = -1;
-    bool active = prod_next_stage<M>(p, c, lane);
+    bool active = prod_next_stage<M>(p, sm, c, lane);
     long long t_progress = clock64();
     long long tp_first = (p.trace && lane == 0) ? global_ns() : 0, stall = 0, t_blocked = 0;
     bool blocked = false;
@@ -383,7 +385,7 @@ __device__ void pass_producer(const PassParams& p, const PassSmem& sm) {
                         producer_trace(p, c.s, tp_first, stall);
                         stall = 0;
                     }
-                    active = prod_next_stage<M>(p, c, lane);
+                    active = prod_next_stage<M>(p, sm, c, lane);
                     if (p.trace && lane == 0) tp_first = global_ns();
                 }
             } else {
@@ -780,10 +782,10 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     const int type = st.type;
     const bool norm = (type == kStQkv || type == kStGateUp || type == kStLmHead);
     const int n_in = st.n_in, n_rows = st.n_rows;
-    int pair0, np;
-    cta_pairs(n_rows, type, pair0, np);
+    // this CTA's share of the matrix (computed once per launch: the split costs three integer divisions)
+    const int pair0 = sm.split[type * 4 + 0], np = sm.split[type * 4 + 1];
     const int n_seg = (n_in + kSegK - 1) / kSegK;
-    const int n_oct = (np + kGrpPairs - 1) / kGrpPairs;  // groups of 16 rows (8 pairs; the last group may hold fewer)
+    const int n_oct = sm.split[type * 4 + 2];  // groups of 16 rows (8 pairs; the last group may hold fewer)
     const int wseg = pass_wseg(M, p.xs_bytes);
     const int xstride = wseg * kSegK + kXsPad;  // bf16 elements per activation row in the window
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(sm.reg_a);
@@ -802,9 +804,13 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     // Fewer groups than warps (the d x d matrices leave ~28 rows to a CTA): several warps share a group, warp set ks
     // taking the segments congruent to ks modulo S and summing into its own copy of the partial sums; the copies are
     // added in the epilogue in the order ks = 0, 1, ... (a fixed order that depends on the matrix shape only).
-    const int S = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
+    const int S = sm.split[type * 4 + 3];
     const int copy_stride = np * 2 * M;
-    for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
+    // A warp's first item of the stage stores its sums, later items add: the partial sums need no zeroing (only when a
+    // row has fewer segments than warp sets, i.e. some copies would never be written, they are zeroed and all items add)
+    const bool store_first = n_seg >= S;
+    if (!store_first)
+        for (int i = tid; i < S * copy_stride; i += kPassConsumers) psum[i] = 0.f;
     constexpr bool kKeepX = (M == 1);
     const bool keep = kKeepX && norm && n_in <= kPassConsumers * 12;
     uint2 gpre[3] = {make_uint2(0u, 0u), make_uint2(0u, 0u), make_uint2(0u, 0u)};  // this thread's RMSNorm gains
@@ -828,7 +834,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         int ra, rb;
         stage_pair_rows(type, p, pair0 + (tid - m * np), ra, rb);
         if (ra < p.d_model + p.kv_dim) {
-            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+            const int half = p.head_dim >> 1, jr = p.hd_shift ? (ra & (p.head_dim - 1)) : ra % p.head_dim;
             pre0 = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
             pre1 = p.rope_sin[(size_t)(p.pos0 + m) * half + jr];
         }
@@ -837,7 +843,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         int ra, rb;
         stage_pair_rows(type, p, pair0 + tid, ra, rb);
         if (ra < p.d_model + p.kv_dim) {
-            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+            const int half = p.head_dim >> 1, jr = p.hd_shift ? (ra & (p.head_dim - 1)) : ra % p.head_dim;
 #pragma unroll
             for (int m = 0; m < (kPre ? M : 0); ++m) {
                 pre[m] = p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
@@ -1165,12 +1171,18 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                     const int wr = g8 + 8 * hr;
                     if (wr < rows) {
                         float* dst = psum_w + (size_t)(kGrpRows * o + wr) * M;
+                        const bool first = store_first && seg == ((S > 1) ? ks : 0);
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int mm = 2 * q4 + e;
-                            if (mm < M) dst[mm] += (acc[0][2 * hr + e] + acc[2][2 * hr + e]) + (acc[1][2 * hr + e] + acc[3][2 * hr + e]);
-                            if (M > 8 && mm + 8 < M)
-                                dst[mm + 8] += (acc2[0][2 * hr + e] + acc2[2][2 * hr + e]) + (acc2[1][2 * hr + e] + acc2[3][2 * hr + e]);
+                            if (mm < M) {
+                                const float v = (acc[0][2 * hr + e] + acc[2][2 * hr + e]) + (acc[1][2 * hr + e] + acc[3][2 * hr + e]);
+                                dst[mm] = first ? v : dst[mm] + v;
+                            }
+                            if (M > 8 && mm + 8 < M) {
+                                const float v = (acc2[0][2 * hr + e] + acc2[2][2 * hr + e]) + (acc2[1][2 * hr + e] + acc2[3][2 * hr + e]);
+                                dst[mm + 8] = first ? v : dst[mm + 8] + v;
+                            }
                         }
                     }
                 }
@@ -1263,7 +1275,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         // memory round trip per row would add up
         float rc[M], rs[M];
         if (type == kStQkv && ra < p.d_model + p.kv_dim) {
-            const int half = p.head_dim >> 1, jr = ra % p.head_dim;
+            const int half = p.head_dim >> 1, jr = p.hd_shift ? (ra & (p.head_dim - 1)) : ra % p.head_dim;
 #pragma unroll
             for (int m = 0; m < M; ++m) {
                 rc[m] = (kPre && pl == tid) ? pre[kPre ? m : 0] : p.rope_cos[(size_t)(p.pos0 + m) * half + jr];
@@ -1961,6 +1973,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     sm.red = reinterpret_cast<float*>(base + p.off_misc);
     sm.flag = reinterpret_cast<int*>(sm.red + 16 * kPassMaxRows * 4);
     sm.consumed = reinterpret_cast<volatile unsigned*>(sm.flag + 8);
+    int* split = reinterpret_cast<int*>(const_cast<unsigned*>(sm.consumed) + 64);
+    sm.split = split;
     sm.psum = reinterpret_cast<float*>(base + p.off_psum);
     sm.reg_a = base + p.off_reg_a;
 
@@ -1971,6 +1985,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
             sm.consumed[i] = 0u;
         }
         mbar_fence_init();
+    }
+    if (threadIdx.x >= 32 && threadIdx.x < 40) {  // split table: rows of the matrix of every stage type
+        const int type = threadIdx.x - 32;
+        const int n_rows = type == kStQkv ? p.d_model + 2 * p.kv_dim
+                         : (type == kStOproj || type == kStDown) ? p.d_model
+                         : type == kStGateUp ? 2 * p.d_ffn
+                         : type == kStLmHead ? p.vocab : 0;
+        int pair0 = 0, np = 0;
+        if (n_rows > 0) cta_pairs(n_rows, type, pair0, np);
+        const int n_oct = (np + kGrpPairs - 1) / kGrpPairs;
+        // fewer groups than warps: several warp sets share a group (see gemv_stage)
+        split[type * 4 + 0] = pair0, split[type * 4 + 1] = np, split[type * 4 + 2] = n_oct;
+        split[type * 4 + 3] = (n_oct > 0 && n_oct < 8) ? kPassConsumerWarps / n_oct : 1;
     }
     __syncthreads();
 
@@ -1988,9 +2015,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
     for (int s = 0; s < p.n_stages; ++s) {
         trace_mark(p, s, 0);
         const StageDesc st = p.stages[s];  // static: read before waiting for the previous stage
+        const int next_type = (s + 1 < p.n_stages) ? p.stages[s + 1].type : -1;  // (read now: at the end of the stage it would be a round trip)
         // the next descriptor is requested now so that reading it at the next stage boundary hits L1
         if (threadIdx.x < 2 && s + 1 < p.n_stages)
             asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(p.stages + s + 1) + threadIdx.x * 64));
+        if (p.trace && threadIdx.x == 0) p.trace[((size_t)s * kTraceEntries + 11) * gridDim.x + blockIdx.x] = st.type >= 0 ? global_ns() : 0;  // descriptor read
         if (st.type == kStEmbed) {
             stage_begin(p, s);
             const int d = p.d_model;
@@ -2014,10 +2043,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(const __grid_cons
         // With the tagged handoff only the finish stage still waits at the grid barrier: the arrival in front of it
         // publishes everything this CTA has written so far, the others just count.
         bool release = true;
-        if (LL && s + 1 < p.n_stages) {
-            const int next = p.stages[s + 1].type;
-            release = (next == kStFinish);
-        }
+        if (LL && next_type >= 0) release = (next_type == kStFinish);
         grid_arrive(p, release);
     }
 }

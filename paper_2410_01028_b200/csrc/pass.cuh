@@ -1834,60 +1834,12 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
         const bool report = (jn >= n_local) || ((first + jn) / n_chunks != kvh);
         bar_sync(bar_id, 128);
         if (LL) {
-            // Tagged handoff: no ticket. The group that took the head's last chunk (the one with this pass's key) merges:
-            // it asks for the other chunks' partial results until their tags are this stage's (they come from items with
-            // lower numbers: other CTAs, or other groups and earlier rounds of this CTA, none of which waits for this one).
+            // Tagged handoff: no ticket (the heads are merged in a second sweep below)
             if (gt == 0) {
                 fence_proxy_async_smem();
                 for (int t = 0; t < tile_slots; ++t) ring_release(p, sm, gv + t);
             }
             if (j == 0) trace_mark(p, stage, 6);
-            if (chunk == n_chunks - 1) {
-                for (int g = 0; g < group; ++g) {
-                    const int head = kvh * group + g;
-                    for (int e0 = 0; e0 < hd; e0 += 128) {  // one output dimension per thread (every lane runs the loop: shuffle below)
-                        const int e = e0 + gt;
-                        const bool act = e < hd;
-                        float mx = -INFINITY, l = 0.f, acc = 0.f;
-                        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
-                            unsigned long long ra[8] = {}, rm[8] = {}, rl[8] = {};
-                            unsigned stale = 0u;
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                if (act && c0 + i < n_chunks) stale |= 1u << i;
-                            for (;;) {
-#pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    if (stale & (1u << i)) {
-                                        const size_t b = (size_t)head * p.chunk_stride + c0 + i;
-                                        ra[i] = ll_load1(p.pl_acc + b * hd + e);
-                                        ll_load2(p.pl_ml + b * 2, rm[i], rl[i]);
-                                    }
-#pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    if ((stale & (1u << i)) && ll_ready(ra[i], tag_out) && ll_ready(rm[i], tag_out) && ll_ready(rl[i], tag_out)) stale &= ~(1u << i);
-                                if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
-                                __nanosleep(100u);
-                            }
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                if (c0 + i < n_chunks) {  // same arithmetic as the merge of the other instantiations
-                                    const float cm = __uint_as_float((uint32_t)rm[i]);
-                                    const float mn = fmaxf(mx, cm);
-                                    const float s_old = expf(mx - mn), s_new = expf(cm - mn);
-                                    acc = __fmaf_rn(acc, s_old, __fmul_rn(__uint_as_float((uint32_t)ra[i]), s_new));
-                                    l = __fmaf_rn(l, s_old, __fmul_rn(__uint_as_float((uint32_t)rl[i]), s_new));
-                                    mx = mn;
-                                }
-                            }
-                        }
-                        const uint32_t ob = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__fdiv_rn(acc, l)));
-                        const uint32_t up = __shfl_down_sync(0xffffffffu, ob, 1);
-                        if (act && (gt & 1) == 0) ll_store(p.al + (((size_t)head * hd + e) >> 1), ob | (up << 16), tag_out);
-                    }
-                }
-            }
-            if (j == 0) trace_mark(p, stage, 7);
             continue;
         }
         if (gt == 0) {
@@ -1958,6 +1910,61 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             }
         }
         if (j == 0) trace_mark(p, stage, 7);
+    }
+    if (LL) {
+        // Tagged handoff, second sweep: the group that took a head's last chunk (the one with this pass's key) merges the
+        // head, after ALL its items: it asks for the chunks' partial results until their tags are this stage's. Nobody who
+        // produces a partial result ever waits for a merge, so the wait ends; merging inside the first sweep would hold
+        // this CTA's later items (and through the ring its other groups) behind chunks that other CTAs reach last.
+        for (int j = grp; j < n_local; j += p.attn_groups) {
+            const int idx = first + j;
+            const int kvh = idx / n_chunks, chunk = idx - kvh * n_chunks;
+            if (chunk != n_chunks - 1) continue;
+            for (int g = 0; g < group; ++g) {
+                const int head = kvh * group + g;
+                for (int e0 = 0; e0 < hd; e0 += 128) {  // one output dimension per thread (every lane runs the loop: shuffle below)
+                    const int e = e0 + gt;
+                    const bool act = e < hd;
+                    float mx = -INFINITY, l = 0.f, acc = 0.f;
+                    for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+                        unsigned long long ra[8] = {}, rm[8] = {}, rl[8] = {};
+                        unsigned stale = 0u;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (act && c0 + i < n_chunks) stale |= 1u << i;
+                        for (;;) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (stale & (1u << i)) {
+                                    const size_t b = (size_t)head * p.chunk_stride + c0 + i;
+                                    ra[i] = ll_load1(p.pl_acc + b * hd + e);
+                                    ll_load2(p.pl_ml + b * 2, rm[i], rl[i]);
+                                }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if ((stale & (1u << i)) && ll_ready(ra[i], tag_out) && ll_ready(rm[i], tag_out) && ll_ready(rl[i], tag_out)) stale &= ~(1u << i);
+                            if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
+                            __nanosleep(100u);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (c0 + i < n_chunks) {  // same arithmetic as the merge of the other instantiations
+                                const float cm = __uint_as_float((uint32_t)rm[i]);
+                                const float mn = fmaxf(mx, cm);
+                                const float s_old = expf(mx - mn), s_new = expf(cm - mn);
+                                acc = __fmaf_rn(acc, s_old, __fmul_rn(__uint_as_float((uint32_t)ra[i]), s_new));
+                                l = __fmaf_rn(l, s_old, __fmul_rn(__uint_as_float((uint32_t)rl[i]), s_new));
+                                mx = mn;
+                            }
+                        }
+                    }
+                    const uint32_t ob = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__fdiv_rn(acc, l)));
+                    const uint32_t up = __shfl_down_sync(0xffffffffu, ob, 1);
+                    if (act && (gt & 1) == 0) ll_store(p.al + (((size_t)head * hd + e) >> 1), ob | (up << 16), tag_out);
+                }
+            }
+        }
+        if (grp == 0) trace_mark(p, stage, 7);
     }
 }
 

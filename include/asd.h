@@ -204,14 +204,14 @@ int asd_generate_device(asd_ctx* ctx, const int32_t* dev_prompt, int32_t n_promp
  * sums behind C_l and returns t_1.
  *   ASD_PREFILL_ROWS  passes of up to 16 rows through the decode kernel: row r of the prompt is bit-identical to
  *                     a one-row pass at the same position.
- *   ASD_PREFILL_GEMM  all rows but the last as dense bf16 products on the tensor cores (fp32 accumulation, the
- *                     same rounding points; the accumulation order differs, so results agree with
- *                     ASD_PREFILL_ROWS to rounding, not bit for bit), then the last row as a one-row pass.
+ *   ASD_PREFILL_GEMM  all rows as dense bf16 products on the tensor cores (fp32 accumulation, the same rounding
+ *                     points; the accumulation order differs, so results agree with ASD_PREFILL_ROWS to
+ *                     rounding, not bit for bit), then the LM head alone on the last row's hidden state.
  *                     Needs head_dim 64 or 128, else ASD_ERR_ARG.
  *   ASD_PREFILL_AUTO  (default) ASD_PREFILL_GEMM for prompts of more than 32 tokens where the shape allows it,
  *                     otherwise ASD_PREFILL_ROWS.
- * After a prompt that took the dense path, asd_get_last_cosines / asd_get_last_logits describe the one-row
- * pass of the last prompt token. */
+ * After a prompt that took the dense path, asd_get_last_cosines / asd_get_last_logits describe the last prompt
+ * token (one row). */
 #define ASD_PREFILL_AUTO 0
 #define ASD_PREFILL_ROWS 1
 #define ASD_PREFILL_GEMM 2

@@ -327,7 +327,7 @@ struct asd_ctx {
     int last_M = 0;
     bool debug_logits = false, last_has_logits = false, last_had_lm_head = false, trace = false;
     bool short_waits = false, inject_missing_arrival = false;  // test hooks of the bounded device waits (asd_set_debug)
-    bool no_tagged_handoff = false;  // asd_set_debug: one- and two-row passes use the grid barrier like the others
+    bool no_tagged_handoff = false;  // asd_set_debug: one-row passes use the grid barrier like the others
     // sampling (temperature > 0): every token is drawn; the draft steps of a round keep their distributions for the verify
     double temperature = 0.0;
     uint64_t seed = 0;

@@ -502,6 +502,11 @@ __device__ __forceinline__ void top2_merge(float& v, int& i, float& s, float ov,
 // until every tag is the one it expects: one round trip after the slowest producer's store, no fence, no barrier.
 // A buffer is only overwritten by a stage that itself needed ALL outputs of a later stage than every reader's, so no
 // reader can still be waiting for the old contents (same ordering a barrier would give, carried by the data).
+// The attention stage takes part: W_qkv's epilogue leaves q and this pass's k and v as tagged words (one bf16 each), a
+// (head, chunk) item leaves its partial result as tagged words, and the group that took a head's last chunk merges the
+// head once all items of its CTA are done. q, k, v and the partial results of a layer are overwritten by the next
+// layer's stages, which a CTA only reaches through W_o's stage, i.e. after every head's merged output (and with it
+// every read of q, k, v and of the partial results) exists.
 __device__ __forceinline__ void ll_store(uint2* dst, uint32_t data, uint32_t tag) {
     const unsigned long long v = ((unsigned long long)tag << 32) | (unsigned long long)data;
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(dst), "l"(v) : "memory");
@@ -1646,7 +1651,7 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
             q_head = head;
             bar_sync(bar_id, 128);
 
-            if (j == 0 && g == 0) trace_mark(p, stage, 2);  // attention timeline: 2 = inputs staged, 4 = softmax done, 5 = P V done, 6 = ticket taken, 7 = merged
+            if (j == 0 && g == 0) trace_mark(p, stage, 2);  // attention timeline: 2 = inputs staged, 4 = softmax done, 5 = P V done, 6 = ticket taken / value tile released, 7 = merged
             // ---- scores: thread t owns key key0 + t. Four independent partial sums per row (16-byte chunk parity x half
             //      of the chunk) keep the chains of dependent FMAs short; they are added in a fixed order.
             float sc[M];

@@ -1121,9 +1121,14 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
         const int o_first = (S > 1) ? ((ks < S) ? warp - ks * n_oct : n_oct) : warp;
         const int o_step = (S > 1) ? n_oct : kPassConsumerWarps;  // S > 1: exactly one group per warp
         float* psum_w = psum + (size_t)ks * copy_stride;
-        for (int sg = 0; sg < ws; ++sg) {
-            const int seg = w0 + sg;
-            if (S > 1 && seg % S != ks) continue;
+        // this warp set's segments of the window: ks, ks + S, ... (one remainder per window instead of one per segment)
+        int seg_first = w0;
+        if (S > 1) {
+            const int r = w0 % S;
+            seg_first = w0 + (ks >= r ? ks - r : ks + S - r);
+        }
+        for (int seg = seg_first; seg < w0 + ws; seg += S) {
+            const int sg = seg - w0;
             for (int o = o_first; o < n_oct; o += o_step) {
                 const uint32_t g = gi + (uint32_t)(seg * n_oct + o);
                 const int rows = 2 * min(kGrpPairs, np - kGrpPairs * o);

@@ -82,3 +82,37 @@ def test_sixteen_row_prompt_passes_are_bit_identical_to_one_row_passes():
     np.testing.assert_array_equal(dec.get_last_logits()[0], l_rows)
     assert t1 == t2
     assert n_r == len(prompt)
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=["d512_hd128", "d1024_gqa"])
+def test_tagged_handoff_and_grid_barrier_variants_of_the_one_row_pass_agree_bit_for_bit(shape):
+    """The one-row pass hands activations over as tagged words (no grid barrier); the debug flag makes it use the grid
+    barrier like the multi-row passes. Same arithmetic, so logits, cosines and K/V must be identical."""
+    import paper_2410_01028_b200 as asd
+    model = synth.make_model(shape, seed=31, std=0.05)
+    dec = asd.Decoder(shape, max_seq=300, max_draft=8)
+    dec.load_weights_host(model)
+    dec.set_prefill_mode(asd.PREFILL_ROWS)
+    prompt = synth.make_prompt(shape.vocab, 250, seed=32)           # decode steps cross the chunk border at 256
+    cont = synth.make_prompt(shape.vocab, 10, seed=33)
+    runs = []
+    for barrier in (False, True):
+        dec.reset()
+        dec.set_debug(True, no_tagged_handoff=barrier)
+        t = dec.prefill(prompt)
+        logits, cos = [], []
+        for r in [int(t)] + [int(v) for v in cont]:
+            dec.decode_step(r)
+            logits.append(dec.get_last_logits()[0].copy())
+            ca, cm = dec.get_last_cosines()
+            cos.append(np.concatenate([ca[:, 0], cm[:, 0]]))
+        kv = [dec.get_kv(l, p) for l in range(shape.n_layers) for p in range(len(prompt), len(prompt) + 11)]
+        runs.append((logits, cos, kv))
+    dec.set_debug(True, no_tagged_handoff=False)
+    for a, b in zip(runs[0][0], runs[1][0]):
+        np.testing.assert_array_equal(a, b)
+    for a, b in zip(runs[0][1], runs[1][1]):
+        np.testing.assert_array_equal(a, b)
+    for (ka, va), (kb, vb) in zip(runs[0][2], runs[1][2]):
+        np.testing.assert_array_equal(ka, kb)
+        np.testing.assert_array_equal(va, vb)

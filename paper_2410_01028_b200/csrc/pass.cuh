@@ -1145,20 +1145,43 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
                 for (int a = 0; a < 4; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
 #pragma unroll
                 for (int a = 0; a < (M > 8 ? 4 : 1); ++a) acc2[a][0] = acc2[a][1] = acc2[a][2] = acc2[a][3] = 0.f;
+                // Operands of four column blocks in registers, then 8 steps; twice per full item. Lanes whose weight row lies
+                // beyond the item's rows, or whose activation row beyond M, read whatever follows in the slot / the last
+                // activation row: every output element depends on its own weight row and activation row only, and the
+                // outputs of such rows are never stored. Only column blocks past the end of a ragged last segment must
+                // contribute nothing and are replaced by zeros.
+                if (nblk == kSegBlocks) {
 #pragma unroll
-                for (int h = 0; h < kSegBlocks / 4; ++h) {  // halves of 4 column blocks: operands in registers, then 8 steps
-                    if (h * 4 < nblk) {
+                    for (int h = 0; h < kSegBlocks / 4; ++h) {
+                        uint4 wlo[4], whi[4], xv[4], xv2[M > 8 ? 4 : 1];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            wlo[j] = *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk);
+                            whi[j] = *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk + 8 * 64);
+                            xv[j] = *reinterpret_cast<const uint4*>(xa + sg * kSegK + (h * 4 + j) * 32);
+                            if (M > 8) xv2[j] = *reinterpret_cast<const uint4*>(xb2 + sg * kSegK + (h * 4 + j) * 32);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            mma_bf16_16816(acc[(j & 1) * 2 + 0], wlo[j].x, whi[j].x, wlo[j].y, whi[j].y, xv[j].x, xv[j].y);
+                            mma_bf16_16816(acc[(j & 1) * 2 + 1], wlo[j].z, whi[j].z, wlo[j].w, whi[j].w, xv[j].z, xv[j].w);
+                            if (M > 8) {
+                                mma_bf16_16816(acc2[(j & 1) * 2 + 0], wlo[j].x, whi[j].x, wlo[j].y, whi[j].y, xv2[j].x, xv2[j].y);
+                                mma_bf16_16816(acc2[(j & 1) * 2 + 1], wlo[j].z, whi[j].z, wlo[j].w, whi[j].w, xv2[j].z, xv2[j].w);
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll 1
+                    for (int h = 0; h * 4 < nblk; ++h) {
                         uint4 wlo[4], whi[4], xv[4], xv2[M > 8 ? 4 : 1];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const bool inb = h * 4 + j < nblk;
-                            wlo[j] = (inb && g8 < rows) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk) : make_uint4(0u, 0u, 0u, 0u);
-                            whi[j] = (inb && g8 + 8 < rows) ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk + 8 * 64)
-                                                           : make_uint4(0u, 0u, 0u, 0u);
-                            xv[j] = (g8 < M) ? *reinterpret_cast<const uint4*>(xa + sg * kSegK + (h * 4 + j) * 32) : make_uint4(0u, 0u, 0u, 0u);
-                            if (M > 8)
-                                xv2[j] = (g8 + 8 < M) ? *reinterpret_cast<const uint4*>(xb2 + sg * kSegK + (h * 4 + j) * 32)
-                                                      : make_uint4(0u, 0u, 0u, 0u);
+                            wlo[j] = inb ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk) : make_uint4(0u, 0u, 0u, 0u);
+                            whi[j] = inb ? *reinterpret_cast<const uint4*>(sl + (h * 4 + j) * blk + 8 * 64) : make_uint4(0u, 0u, 0u, 0u);
+                            xv[j] = *reinterpret_cast<const uint4*>(xa + sg * kSegK + (h * 4 + j) * 32);
+                            if (M > 8) xv2[j] = *reinterpret_cast<const uint4*>(xb2 + sg * kSegK + (h * 4 + j) * 32);
                         }
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {

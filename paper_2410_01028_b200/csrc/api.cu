@@ -140,15 +140,23 @@ static bool plan_pass(const DeviceInfo& dv, const asd_config& c, int M, PassPlan
     // Activation window: the longest reduction dimension (in segments of 256 inputs) cut into as few windows as leave
     // the ring 20 slots. Every further window costs a stage of a multi-row pass a block-wide refill, every slot less
     // costs bandwidth (one row, 7B shape: 24 slots 0.402 ms per 4 layers, 21: 0.409, 16: 0.422, 12: 0.481); 20 was the
-    // best trade for three and four rows. One row always fits whole.
+    // best trade for three and four rows (measured again with 22 and 24 after the kernel had changed: four and five rows
+    // 0.7 % slower). Windows do not get shorter than a row of d_model while that leaves 16 slots: the RMSNorm stages want
+    // their rows whole (six to nine rows: 1-2.5 % faster than with W_d's row cut into equal parts). One row always fits whole.
     const size_t seg_max = ((size_t)std::max(c.d_model, c.d_ffn) + kSegK - 1) / kSegK;
+    const size_t seg_norm = ((size_t)c.d_model + kSegK - 1) / kSegK;  // the RMSNorm stages want their rows whole in the window
     const long long fixed = 1024 + (long long)(psum + misc) + 2 * 64 * 8;
     size_t wseg_plan = seg_max;
+    auto leaves_ring = [&](size_t wseg, long long slots) {
+        const size_t bytes = (size_t)M * (wseg * kSegK + kXsPad) * 2;
+        return (long long)dv.max_smem - fixed - (long long)((bytes + 15) & ~(size_t)15) >= slots * kSlotBytes;
+    };
     for (size_t nw = 1; nw <= seg_max; ++nw) {
         wseg_plan = (seg_max + nw - 1) / nw;
-        const size_t bytes = (size_t)M * (wseg_plan * kSegK + kXsPad) * 2;
-        if ((long long)dv.max_smem - fixed - (long long)((bytes + 15) & ~(size_t)15) >= 20LL * kSlotBytes) break;
+        if (leaves_ring(wseg_plan, 20)) break;
     }
+    // not shorter than a row of d_model while the ring keeps 16 slots: the RMSNorm stages want their rows whole
+    if (wseg_plan < seg_norm && leaves_ring(seg_norm, 16)) wseg_plan = seg_norm;
     const int xs_bytes = (int)((size_t)M * (wseg_plan * kSegK + kXsPad) * 2);
     const size_t xs = (size_t)M * ((size_t)pass_wseg(M, xs_bytes) * kSegK + kXsPad) * 2;
     // up to three groups of four warps work on attention items, as many as their scratch fits the window's bytes

@@ -625,7 +625,7 @@ __device__ __forceinline__ void norm_rows_into_window(const float* xf, const __n
     else norm_rows_call<M>(xf, gain, n_in, wlen, xstride, eps, xs, red);
 }
 
-// Epilogues of a GEMV stage with four or more activation rows, as functions of their own (their registers are their
+// Epilogues of a GEMV stage with three or more activation rows, as functions of their own (their registers are their
 // own; everything they need comes as scalar arguments, so nothing is re-read from the parameter block or the stage
 // table). The (weight row or pair, activation row) items of the CTA are spread over all consumer threads instead of
 // giving a thread all M rows of its pair. Every item is computed exactly as the one-row path computes it, and the
@@ -830,7 +830,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     // One or two rows: what the epilogue will need from global memory is requested ahead of the weight stream
     // (the rotary factors of this thread's pair before the barrier, the old hidden state of its row after it),
     // so the epilogue does not wait for a memory round trip.
-    constexpr bool kSpreadEpi = (M >= 4);  // measured: spreading the epilogue's items over the threads pays from four rows on
+    constexpr bool kSpreadEpi = (M >= 3);  // measured: spreading the epilogue's items over the threads pays from three rows on (two rows: no difference)
     constexpr bool kPre = (M <= 2);
     float pre[kPre ? 2 * M : 1];
     float pre0 = 0.f, pre1 = 0.f;  // spread epilogue: what the first item of this thread / warp needs (see the epi_*_rows functions)
@@ -1235,7 +1235,7 @@ __device__ void gemv_stage(const PassParams& p, const StageDesc& st, const PassS
     }
 
     if constexpr (!kSpreadEpi) {
-    // ---- epilogue of a pass of up to three rows: thread t owns pairs t, t+480, ... of this CTA and all M rows of them
+    // ---- epilogue of a pass of one or two rows: thread t owns pairs t, t+480, ... of this CTA and all M rows of them
     float s_loc[M][3];
     float best_v[M], sec_v[M];
     int best_i[M];

@@ -1959,35 +1959,42 @@ __device__ void attn_stage(const PassParams& p, const StageDesc& st, const PassS
                     const int e = e0 + gt;
                     const bool act = e < hd;
                     float mx = -INFINITY, l = 0.f, acc = 0.f;
-                    for (int c0 = 0; c0 < n_chunks; c0 += 8) {
-                        unsigned long long ra[8] = {}, rm[8] = {}, rl[8] = {};
-                        unsigned stale = 0u;
+                    // Lane i of every warp fetches (maximum, sum of weights) of chunk c0 + i, 32 chunks per memory round trip,
+                    // and hands them round by shuffle; every thread fetches its own dimension's sums 16 chunks at a time
+                    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+                        unsigned long long rm = 0, rl = 0;
+                        bool ml_stale = c0 + glane < n_chunks;
+#pragma unroll 1
+                        for (int c1 = c0; c1 < c0 + 32 && c1 < n_chunks; c1 += 16) {
+                            unsigned long long ra[16] = {};
+                            unsigned stale = 0u;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (act && c0 + i < n_chunks) stale |= 1u << i;
-                        for (;;) {
+                            for (int i = 0; i < 16; ++i)
+                                if (act && c1 + i < n_chunks) stale |= 1u << i;
+                            for (;;) {
+                                if (ml_stale) ll_load2(p.pl_ml + ((size_t)head * p.chunk_stride + c0 + glane) * 2, rm, rl);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                if (stale & (1u << i)) {
-                                    const size_t b = (size_t)head * p.chunk_stride + c0 + i;
-                                    ra[i] = ll_load1(p.pl_acc + b * hd + e);
-                                    ll_load2(p.pl_ml + b * 2, rm[i], rl[i]);
+                                for (int i = 0; i < 16; ++i)
+                                    if (stale & (1u << i)) ra[i] = ll_load1(p.pl_acc + ((size_t)head * p.chunk_stride + c1 + i) * hd + e);
+                                if (ml_stale && ll_ready(rm, tag_out) && ll_ready(rl, tag_out)) ml_stale = false;
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    if ((stale & (1u << i)) && ll_ready(ra[i], tag_out)) stale &= ~(1u << i);
+                                if ((stale == 0u && !ml_stale) || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
+                                __nanosleep(100u);
+                            }
+                            __syncwarp();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                if (c1 + i < n_chunks) {  // (uniform) same arithmetic as the merge of the other instantiations
+                                    const float cm = __uint_as_float(__shfl_sync(0xffffffffu, (uint32_t)rm, (c1 - c0) + i));
+                                    const float cl = __uint_as_float(__shfl_sync(0xffffffffu, (uint32_t)rl, (c1 - c0) + i));
+                                    const float mn = fmaxf(mx, cm);
+                                    const float s_old = expf(mx - mn), s_new = expf(cm - mn);
+                                    acc = __fmaf_rn(acc, s_old, __fmul_rn(__uint_as_float((uint32_t)ra[i]), s_new));
+                                    l = __fmaf_rn(l, s_old, __fmul_rn(cl, s_new));
+                                    mx = mn;
                                 }
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                if ((stale & (1u << i)) && ll_ready(ra[i], tag_out) && ll_ready(rm[i], tag_out) && ll_ready(rl[i], tag_out)) stale &= ~(1u << i);
-                            if (stale == 0u || !ll_keep_waiting(p, ll_spins, ll_t0, stage)) break;
-                            __nanosleep(100u);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            if (c0 + i < n_chunks) {  // same arithmetic as the merge of the other instantiations
-                                const float cm = __uint_as_float((uint32_t)rm[i]);
-                                const float mn = fmaxf(mx, cm);
-                                const float s_old = expf(mx - mn), s_new = expf(cm - mn);
-                                acc = __fmaf_rn(acc, s_old, __fmul_rn(__uint_as_float((uint32_t)ra[i]), s_new));
-                                l = __fmaf_rn(l, s_old, __fmul_rn(__uint_as_float((uint32_t)rl[i]), s_new));
-                                mx = mn;
                             }
                         }
                     }

@@ -49,3 +49,39 @@ def test_head_size_against_oracle_and_row_invariance(shape):
     lg = dec.get_last_logits()
     for m in range(5):
         np.testing.assert_array_equal(lg[m], one[m])
+
+
+WIDE = synth.DecoderShape(n_layers=1, d_model=6144, n_heads=48, head_dim=128, d_ffn=2048, vocab=509)
+
+
+def test_rows_longer_than_the_register_paths_hold(request):
+    """d_model above 5760: the RMSNorm stages take the general (strided) path and the one-row pass synchronises at the
+    grid barrier (the tagged handoff needs its three chunks per thread). Against the oracle, lossless, row-invariant."""
+    import paper_2410_01028_b200 as asd
+    model = synth.make_model(WIDE, seed=8, std=0.02)
+    dec = asd.Decoder(WIDE, max_seq=96, max_draft=8)
+    dec.load_weights_host(model)
+    orc = oracle.Oracle(model, max_seq=96)
+    prompt = synth.make_prompt(WIDE.vocab, 40, seed=9)
+    teacher_forced_compare(dec, orc, prompt, 8)
+    ar, _ = dec.generate(prompt, 16, mode=asd.MODE_AR)
+    for k in (2, 5):
+        dec.set_skip_mask(np.array([0]), np.array([0]))
+        sp, _ = dec.generate(prompt, 16, mode=asd.MODE_SPEC_MANUAL_MASK, draft_len=k)
+        assert sp.tolist() == ar.tolist(), k
+    dec.set_debug(True)
+    dec.set_prefill_mode(asd.PREFILL_ROWS)
+    cont = synth.make_prompt(WIDE.vocab, 2, seed=10)
+    dec.reset()
+    t = dec.prefill(prompt)
+    rows = [int(t)] + [int(v) for v in cont]
+    one = []
+    for r in rows:
+        dec.decode_step(r)
+        one.append(dec.get_last_logits()[0].copy())
+    dec.reset()
+    dec.prefill(prompt)
+    dec.verify(rows)
+    lg = dec.get_last_logits()
+    for m in range(3):
+        np.testing.assert_array_equal(lg[m], one[m])

@@ -190,7 +190,7 @@ struct Layout {
     int chunk_stride;
     // dense prompt path: row-major copies of the sublayer matrices (one block per layer) and activations of a chunk
     size_t rm_layers, rm_layer_stride, rm_wqkv, rm_wo, rm_wgu, rm_wd;
-    size_t pf_x, pf_xn, pf_q, pf_a, pf_t, pf_c, pf_cos;
+    size_t pf_x, pf_xn, pf_q, pf_a, pf_t, pf_c, pf_cos;  // pf_c: two buffers (the halves of a product cut along its reduction dimension)
     int pf_rows;  // prompt rows per chunk of the dense path (0: shape not supported by it)
 };
 
@@ -305,7 +305,7 @@ static Layout make_layout(const asd_config& c) {
         L.pf_q = take(R * d * 2);
         L.pf_a = take(R * d * 2);
         L.pf_t = take(R * f * 2);
-        L.pf_c = take(R * d * 4);
+        L.pf_c = take((size_t)2 * R * d * 4);
         L.pf_cos = take((size_t)2 * c.n_layers * R * 4);
     }
     L.total = o;
@@ -994,10 +994,18 @@ extern "C" int asd_reset(asd_ctx* x) {
 }
 
 // ---------------------------------------------------------------- prefill (Section 3.2)
-// One sublayer product of the dense prompt path: the 64 x 256 weight boxes when that still gives every SM a tile.
-static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which, int M, int N, int K, const GemmEpi& ep) {
+// One sublayer product of the dense prompt path: the 64 x 256 weight boxes when that still gives every SM a tile. A
+// product with fp32 output (W_o, W_d) that has fewer such tiles than SMs is cut in two along its reduction dimension
+// instead of taking the 128-column tiles, which run at half the rate per SM (bound by shared-memory bandwidth): the
+// two halves are work items of their own and the row kernel that follows adds them (half 0 + half 1). *split_out
+// tells the caller whether it was.
+static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which, int M, int N, int K, GemmEpi ep, bool* split_out = nullptr) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
-    const int bn = (((N + 255) / 256) * m_tiles >= x->dev->num_sms) ? 256 : 128;
+    const int tiles256 = ((N + 255) / 256) * m_tiles;
+    const bool split = ep.mode == kGemmF32 && split_out && tiles256 < x->dev->num_sms && K >= 2048;
+    const int bn = (tiles256 >= x->dev->num_sms || split) ? 256 : 128;
+    ep.k_split = split ? 2 : 1;
+    if (split_out) *split_out = split;
     const CUtensorMap& tm_w = x->tm_w[(size_t)layer * 8 + (bn == 256 ? 4 : 0) + which];
     ASD_CUDA(x, launch_gemm_tn(tm_a, tm_w, M, N, K, bn, ep, x->stream));
     x->stats.kernel_launches += 1;
@@ -1041,15 +1049,18 @@ static int prefill_dense(asd_ctx* x, const int32_t* dev_tokens, int n, int pos0)
             o.err = err;
             o.mode = kGemmF32;
             o.c = pc, o.ldc = d;
-            if ((rc = dense_gemm(x, x->tm_a, l, 1, rows, d, d, o))) return rc;
-            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, gain(l, ly.l_mlp_norm), c.rms_eps, pxn, pcos + (size_t)l * R, s));
+            o.c_split_stride = (size_t)R * d;
+            bool split = false;
+            if ((rc = dense_gemm(x, x->tm_a, l, 1, rows, d, d, o, &split))) return rc;
+            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, split ? pc + (size_t)R * d : nullptr, gain(l, ly.l_mlp_norm), c.rms_eps, pxn,
+                                          pcos + (size_t)l * R, s));
             GemmEpi g{};
             g.err = err;
             g.mode = kGemmSwiglu;
             g.t = pt, g.ldt = f;
             if ((rc = dense_gemm(x, x->tm_xn, l, 2, rows, 2 * f, d, g))) return rc;
-            if ((rc = dense_gemm(x, x->tm_t, l, 3, rows, d, f, o))) return rc;
-            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, l + 1 < L ? gain(l + 1, ly.l_attn_norm) : nullptr, c.rms_eps, pxn,
+            if ((rc = dense_gemm(x, x->tm_t, l, 3, rows, d, f, o, &split))) return rc;
+            ASD_CUDA(x, launch_resid_norm(rows, d, px, pc, split ? pc + (size_t)R * d : nullptr, l + 1 < L ? gain(l + 1, ly.l_attn_norm) : nullptr, c.rms_eps, pxn,
                                           pcos + (size_t)(L + l) * R, s));
             x->stats.kernel_launches += 3;
         }

@@ -71,8 +71,8 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
 
 // ============================================================================================ GEMM epilogues
 // One call per (row, 32 consecutive columns starting at col0) with the fp32 accumulators in v.
-__device__ __forceinline__ void epi_f32(const GemmEpi& ep, int row, int col0, int N, const float (&v)[32]) {
-    float* dst = ep.c + (size_t)row * ep.ldc + col0;
+__device__ __forceinline__ void epi_f32(const GemmEpi& ep, int row, int col0, int N, const float (&v)[32], int half) {
+    float* dst = ep.c + (size_t)half * ep.c_split_stride + (size_t)row * ep.ldc + col0;
     if (col0 + 32 <= N && (ep.ldc & 3) == 0) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
@@ -196,6 +196,11 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (K + kGemmBK - 1) / kGemmBK;
+    // Work item = (tile, half of the reduction dimension); without a split there is one half. Items of half 0 come
+    // first, so CTAs that run together still share their weight tile.
+    const int k_split = (ep.mode == kGemmF32 && ep.k_split == 2) ? 2 : 1;
+    const int kb_per = (num_kb + k_split - 1) / k_split;
+    const int n_items = n_tiles_total * k_split;
     volatile int* err = ep.err;
 
     if (threadIdx.x == 0) {
@@ -222,10 +227,11 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (lane == 0) {
             int issued = 0;  // k-blocks requested so far, over all tiles of this CTA
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 // row tiles vary fastest: CTAs that run together share their weight tile (read once from HBM, then from L2)
+                const int tile = item % n_tiles_total, half = item / n_tiles_total;
                 const int m0 = (tile % m_tiles) * kGemmBM, n0 = (tile / m_tiles) * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = half * kb_per; kb < min(num_kb, (half + 1) * kb_per); ++kb) {
                     const int s = issued % kStages;
                     if (issued >= kStages) ok = mbar_wait(&empty[s], (uint32_t)((issued / kStages - 1) & 1), err, kErrGemmWait, 0, issued, s, 1);
                     if (!ok) break;
@@ -250,14 +256,15 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, BN);
             int done = 0, local = 0;  // k-blocks consumed so far; tiles of this CTA started so far
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
                 const int buf = local & 1;
+                const int kb0 = (item / n_tiles_total) * kb_per, kb1 = min(num_kb, kb0 + kb_per);
                 // the epilogue must have read this buffer's previous tile (tile local - 2) before it is overwritten
                 if (local >= 2) ok = mbar_wait(&acc_empty[buf], (uint32_t)((local / 2 - 1) & 1), err, kErrGemmWait, 3, local, buf, 4);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t tmem_d = tmem + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     const int s = done % kStages;
                     ok = mbar_wait(&full[s], (uint32_t)((done / kStages) & 1), err, kErrGemmWait, 1, done, s, 2);
                     if (!ok) break;
@@ -266,7 +273,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const uint64_t a_desc = umma_desc_k128(a_addr), b_desc = umma_desc_k128(a_addr + Cfg::kABytes);
 #pragma unroll
                     for (int k = 0; k < kGemmBK / 16; ++k)  // 16 elements = 32 bytes further along the swizzled row: +2 in the address field
-                        tc_mma_bf16(tmem_d, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_mma_bf16(tmem_d, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
                     tc_commit(&empty[s]);  // the stage may be refilled once these MMAs have read it
                     ++done;
                 }
@@ -277,8 +284,9 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         const int quarter = warp & 3;
         bool ok = true;
         int local = 0;
-        for (int tile = blockIdx.x; tile < n_tiles_total && ok; tile += gridDim.x, ++local) {
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++local) {
             const int buf = local & 1;
+            const int tile = item % n_tiles_total, half = item / n_tiles_total;
             const int m0 = (tile % m_tiles) * kGemmBM, n0 = (tile / m_tiles) * BN;
             const int row = m0 + quarter * 32 + lane;
             ok = mbar_wait(&acc_full[buf], (uint32_t)((local / 2) & 1), err, kErrGemmWait, 2, local, buf, 3) && *err == kErrNone;
@@ -290,7 +298,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 float v[32];
                 tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cb * 32), v);
                 if (row < M) {
-                    if (ep.mode == kGemmF32) epi_f32(ep, row, col0, N, v);
+                    if (ep.mode == kGemmF32) epi_f32(ep, row, col0, N, v, half);
                     else if (ep.mode == kGemmSwiglu) epi_swiglu(ep, row, col0, N, v);
                     else epi_qkv(ep, row, col0, N, v);
                 }
@@ -311,7 +319,8 @@ template <int BN>
 static cudaError_t launch_gemm_bn(const CUtensorMap& tm_a, const CUtensorMap& tm_w, int M, int N, int K, const GemmEpi& ep, cudaStream_t s) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM, n_tiles = (N + BN - 1) / BN;
     const int total = m_tiles * n_tiles;
-    gemm_tn_kernel<BN><<<total < g_gemm_ctas ? total : g_gemm_ctas, kGemmThreads, GemmCfg<BN>::kSmem, s>>>(tm_a, tm_w, M, N, K, m_tiles, total, ep);
+    const int items = total * ((ep.mode == kGemmF32 && ep.k_split == 2) ? 2 : 1);
+    gemm_tn_kernel<BN><<<items < g_gemm_ctas ? items : g_gemm_ctas, kGemmThreads, GemmCfg<BN>::kSmem, s>>>(tm_a, tm_w, M, N, K, m_tiles, total, ep);
     return cudaGetLastError();
 }
 
@@ -367,16 +376,17 @@ __global__ void __launch_bounds__(kRowThreads) embed_norm_kernel(const int* toke
 
 // The residual add with the cosine similarity of the hidden state before and after the sublayer (Section 3.2), and
 // the RMSNorm that feeds the next sublayer (its statistic is the |y|^2 just computed).
-__global__ void __launch_bounds__(kRowThreads) resid_norm_kernel(int d, float* x, const float* c, const __nv_bfloat16* gain, float eps,
+__global__ void __launch_bounds__(kRowThreads) resid_norm_kernel(int d, float* x, const float* c, const float* c2, const __nv_bfloat16* gain, float eps,
                                                                 __nv_bfloat16* xn, float* cos_out) {
     __shared__ float red[24];
     const int r = blockIdx.x;
     float* xr = x + (size_t)r * d;
     const float* cr = c + (size_t)r * d;
+    const float* cr2 = c2 ? c2 + (size_t)r * d : nullptr;  // second half of a product whose reduction dimension was cut in two
     float s[3] = {0.f, 0.f, 0.f};
     for (int i = threadIdx.x; i < d; i += kRowThreads) {
         const float xv = xr[i];
-        const float y = xv + cr[i];
+        const float y = xv + (cr2 ? cr[i] + cr2[i] : cr[i]);
         xr[i] = y;
         s[0] = fmaf(xv, y, s[0]);
         s[1] = fmaf(xv, xv, s[1]);
@@ -398,7 +408,7 @@ __global__ void __launch_bounds__(kRowThreads) resid_norm_kernel(int d, float* x
 // sublayer output are read once, 16 bytes per load, and the sums, the new hidden state and the normalised row all
 // come from those registers.
 template <int NV>
-__global__ void __launch_bounds__(kRowThreads) resid_norm_vec_kernel(int d, float* x, const float* c, const __nv_bfloat16* gain, float eps,
+__global__ void __launch_bounds__(kRowThreads) resid_norm_vec_kernel(int d, float* x, const float* c, const float* c2, const __nv_bfloat16* gain, float eps,
                                                                     __nv_bfloat16* xn, float* cos_out) {
     __shared__ float red[24];
     const int r = blockIdx.x, nvec = d >> 2;
@@ -410,6 +420,17 @@ __global__ void __launch_bounds__(kRowThreads) resid_norm_vec_kernel(int d, floa
         const int i = threadIdx.x + v * kRowThreads;
         y[v] = cv[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (i < nvec) y[v] = xr[i], cv[v] = cr[i];
+    }
+    if (c2) {  // the product came in two halves of its reduction dimension: half 0 + half 1
+        const float4* cr2 = reinterpret_cast<const float4*>(c2 + (size_t)r * d);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int i = threadIdx.x + v * kRowThreads;
+            if (i < nvec) {
+                const float4 o = cr2[i];
+                cv[v].x += o.x, cv[v].y += o.y, cv[v].z += o.z, cv[v].w += o.w;
+            }
+        }
     }
     float s[3] = {0.f, 0.f, 0.f};
 #pragma unroll
@@ -464,15 +485,15 @@ cudaError_t launch_embed_norm(const int* tokens, int n_rows, int d, int vocab, c
     embed_norm_kernel<<<n_rows, kRowThreads, 0, s>>>(tokens, d, vocab, embed, gain, eps, x, xn);
     return cudaGetLastError();
 }
-cudaError_t launch_resid_norm(int n_rows, int d, float* x, const float* c, const __nv_bfloat16* gain, float eps, __nv_bfloat16* xn,
+cudaError_t launch_resid_norm(int n_rows, int d, float* x, const float* c, const float* c2, const __nv_bfloat16* gain, float eps, __nv_bfloat16* xn,
                               float* cos_out, cudaStream_t s) {
     const int nv = (d + kRowThreads * 4 - 1) / (kRowThreads * 4);
-    if (d % 4 != 0 || nv > 8) resid_norm_kernel<<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
-    else if (nv <= 1) resid_norm_vec_kernel<1><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
-    else if (nv <= 2) resid_norm_vec_kernel<2><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
-    else if (nv <= 4) resid_norm_vec_kernel<4><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
-    else if (nv <= 5) resid_norm_vec_kernel<5><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
-    else resid_norm_vec_kernel<8><<<n_rows, kRowThreads, 0, s>>>(d, x, c, gain, eps, xn, cos_out);
+    if (d % 4 != 0 || nv > 8) resid_norm_kernel<<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
+    else if (nv <= 1) resid_norm_vec_kernel<1><<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
+    else if (nv <= 2) resid_norm_vec_kernel<2><<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
+    else if (nv <= 4) resid_norm_vec_kernel<4><<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
+    else if (nv <= 5) resid_norm_vec_kernel<5><<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
+    else resid_norm_vec_kernel<8><<<n_rows, kRowThreads, 0, s>>>(d, x, c, c2, gain, eps, xn, cos_out);
     return cudaGetLastError();
 }
 cudaError_t launch_sumcos(const float* cos_rows, int stride, int n_rows, int n_sub, double* sumcos, cudaStream_t s) {

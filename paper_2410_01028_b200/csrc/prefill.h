@@ -31,6 +31,8 @@ struct GemmEpi {
     // kGemmF32
     float* c;
     int ldc;
+    int k_split;            // 1, or 2: the reduction dimension is cut in two halves, each a work item of its own
+    size_t c_split_stride;  // floats between the partial results of the halves (the caller adds them: half 0 + half 1)
     // kGemmQkv: columns are [q | k | v]; inside every q and k head the rotary partners (j, j + head_dim/2) are
     // neighbours (2j, 2j+1); v columns are in natural order. Row r sits at position pos0 + r.
     __nv_bfloat16 *q, *k_cache, *v_cache;
@@ -54,7 +56,7 @@ cudaError_t launch_embed_norm(const int* tokens, int n_rows, int d, int vocab, c
 
 // y = x + c (in place in x), cos_out[r] = <x, y> / (|x| |y|) (Section 3.2), and, when gain is given,
 // xn[r, :] = bf16(RMSNorm(y) * gain) for the next sublayer
-cudaError_t launch_resid_norm(int n_rows, int d, float* x, const float* c, const __nv_bfloat16* gain, float eps, __nv_bfloat16* xn,
+cudaError_t launch_resid_norm(int n_rows, int d, float* x, const float* c, const float* c2, const __nv_bfloat16* gain, float eps, __nv_bfloat16* xn,
                               float* cos_out, cudaStream_t s);
 
 // sumcos[b] += sum over rows of cos_rows[b * stride + r], rows in a fixed order, double precision

@@ -463,12 +463,12 @@ static int make_tensor_maps(asd_ctx* x) {
         bool ok = encode_operand_map(encode, &x->tm_xn, x->ws + ly.pf_xn, d, R, kGemmBM) &&
                   encode_operand_map(encode, &x->tm_a, x->ws + ly.pf_a, d, R, kGemmBM) &&
                   encode_operand_map(encode, &x->tm_t, x->ws + ly.pf_t, f, R, kGemmBM);
-        x->tm_w.assign((size_t)12 * L, CUtensorMap{});
+        x->tm_w.assign((size_t)8 * L, CUtensorMap{});
         for (int l = 0; l < L && ok; ++l) {
             unsigned char* rw = x->ws + ly.rm_layers + (size_t)l * ly.rm_layer_stride;
-            for (int v = 0; v < 3 && ok; ++v) {
-                const uint32_t bn = 128u + 64u * v;  // weight boxes of 128, 192 and 256 rows
-                CUtensorMap* m = &x->tm_w[(size_t)l * 12 + v * 4];
+            for (int v = 0; v < 2 && ok; ++v) {
+                const uint32_t bn = v ? 256u : 128u;
+                CUtensorMap* m = &x->tm_w[(size_t)l * 8 + v * 4];
                 ok = encode_operand_map(encode, m + 0, rw + ly.rm_wqkv, d, d + 2 * kvd, bn) &&
                      encode_operand_map(encode, m + 1, rw + ly.rm_wo, d, d, bn) &&
                      encode_operand_map(encode, m + 2, rw + ly.rm_wgu, d, 2 * f, bn) &&
@@ -994,27 +994,19 @@ extern "C" int asd_reset(asd_ctx* x) {
 }
 
 // ---------------------------------------------------------------- prefill (Section 3.2)
-// Columns of a GEMM tile (rows of a weight box): 256 when that still gives every SM a tile, else 128; 192 when the
-// tiles then take fewer rounds over the SMs by more than the 11 % more shared-memory bytes they move per product.
-static int gemm_tile_cols(int N, int m_tiles, int sms) {
-    const int tiles256 = ((N + 255) / 256) * m_tiles, tiles192 = ((N + 191) / 192) * m_tiles;
-    const long long cost256 = (long long)((tiles256 + sms - 1) / sms) * 256 * 100, cost192 = (long long)((tiles192 + sms - 1) / sms) * 192 * 111;
-    if (tiles192 >= sms && cost192 < cost256) return 192;
-    return tiles256 >= sms ? 256 : 128;
-}
-
 // One sublayer product of the dense prompt path: the 64 x 256 weight boxes when that still gives every SM a tile. A
 // product with fp32 output (W_o, W_d) that has fewer such tiles than SMs is cut in two along its reduction dimension
 // instead of taking the 128-column tiles, which run at half the rate per SM (bound by shared-memory bandwidth): the
 // two halves are work items of their own and the row kernel that follows adds them (half 0 + half 1). *split_out
 // tells the caller whether it was.
 static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which, int M, int N, int K, GemmEpi ep, bool* split_out = nullptr) {
-    const int m_tiles = (M + kGemmBM - 1) / kGemmBM, sms = x->dev->num_sms;
-    const bool split = ep.mode == kGemmF32 && split_out && ((N + 255) / 256) * m_tiles < sms && K >= 2048;
-    const int bn = split ? 256 : gemm_tile_cols(N, m_tiles, sms);
+    const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
+    const int tiles256 = ((N + 255) / 256) * m_tiles;
+    const bool split = ep.mode == kGemmF32 && split_out && tiles256 < x->dev->num_sms && K >= 2048;
+    const int bn = (tiles256 >= x->dev->num_sms || split) ? 256 : 128;
     ep.k_split = split ? 2 : 1;
     if (split_out) *split_out = split;
-    const CUtensorMap& tm_w = x->tm_w[(size_t)layer * 12 + (bn - 128) / 64 * 4 + which];
+    const CUtensorMap& tm_w = x->tm_w[(size_t)layer * 8 + (bn == 256 ? 4 : 0) + which];
     ASD_CUDA(x, launch_gemm_tn(tm_a, tm_w, M, N, K, bn, ep, x->stream));
     x->stats.kernel_launches += 1;
     return ASD_OK;
@@ -1585,7 +1577,7 @@ extern "C" int asd_gemm_bf16(void* cuda_stream, int32_t M, int32_t N, int32_t K,
     EncodeTiledFn encode = tensor_map_encoder();
     if (!encode) return ASD_ERR_CUDA;
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
-    const int bn = gemm_tile_cols(N, m_tiles, dv->num_sms);
+    const int bn = (((N + 255) / 256) * m_tiles >= dv->num_sms) ? 256 : 128;
     CUtensorMap tm_a, tm_w;
     if (!encode_operand_map(encode, &tm_a, const_cast<uint16_t*>(A), (size_t)K, (size_t)M, kGemmBM) ||
         !encode_operand_map(encode, &tm_w, const_cast<uint16_t*>(W), (size_t)K, (size_t)N, (uint32_t)bn))

@@ -173,8 +173,7 @@ static int g_gemm_ctas = 148;  // persistent CTAs per launch: the SM count of th
 
 template <int BN>
 struct GemmCfg {
-    static constexpr int kStages = (BN == 256) ? 4 : (BN == 192 ? 5 : 6);
-    static constexpr uint32_t kTmemCols = (BN == 128) ? 256u : 512u;  // two accumulators of BN columns in a power-of-two allocation
+    static constexpr int kStages = (BN == 256) ? 4 : 6;
     static constexpr uint32_t kABytes = kGemmBM * kGemmBK * 2;
     static constexpr uint32_t kBBytes = BN * kGemmBK * 2;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
@@ -216,7 +215,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         mbar_fence_init();
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, Cfg::kTmemCols);
+        tmem_alloc(tmem_slot, 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -312,7 +311,7 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, Cfg::kTmemCols);
+        tmem_dealloc(tmem, 2 * BN);
     }
 }
 
@@ -329,7 +328,6 @@ cudaError_t launch_gemm_tn(const CUtensorMap& tm_a, const CUtensorMap& tm_w, int
                            cudaStream_t s) {
     if (M <= 0 || N <= 0 || K <= 0) return cudaErrorInvalidValue;
     if (bn == 256) return launch_gemm_bn<256>(tm_a, tm_w, M, N, K, ep, s);
-    if (bn == 192) return launch_gemm_bn<192>(tm_a, tm_w, M, N, K, ep, s);
     if (bn == 128) return launch_gemm_bn<128>(tm_a, tm_w, M, N, K, ep, s);
     return cudaErrorInvalidValue;
 }
@@ -734,7 +732,6 @@ cudaError_t configure_prefill(int max_smem) {
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     if (sms > 0) g_gemm_ctas = sms;
     if ((e = cudaFuncSetAttribute(gemm_tn_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<256>::kSmem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(gemm_tn_kernel<192>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<192>::kSmem)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(gemm_tn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmCfg<128>::kSmem)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(flash_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fa_smem_bytes<128>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(flash_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fa_smem_bytes<64>())) != cudaSuccess) return e;

@@ -46,7 +46,7 @@ struct GemmEpi {
 cudaError_t configure_prefill(int max_smem);
 
 // C[M, N] = A[M, K] * W[N, K]^T, bf16 operands described by 2-D tensor maps (boxes of 64 x 128 for A, 64 x bn for W,
-// 128-byte swizzle), fp32 accumulation. bn is 128, 192 or 256.
+// 128-byte swizzle), fp32 accumulation. bn is 128 or 256.
 cudaError_t launch_gemm_tn(const CUtensorMap& tm_a, const CUtensorMap& tm_w, int M, int N, int K, int bn, const GemmEpi& ep,
                            cudaStream_t s);
 

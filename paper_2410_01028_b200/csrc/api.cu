@@ -1002,7 +1002,11 @@ extern "C" int asd_reset(asd_ctx* x) {
 static int dense_gemm(asd_ctx* x, const CUtensorMap& tm_a, int layer, int which, int M, int N, int K, GemmEpi ep, bool* split_out = nullptr) {
     const int m_tiles = (M + kGemmBM - 1) / kGemmBM;
     const int tiles256 = ((N + 255) / 256) * m_tiles;
-    const bool split = ep.mode == kGemmF32 && split_out && tiles256 < x->dev->num_sms && K >= 2048;
+    // cut in two when the 256-column tiles do not fill the SMs, or when twice as many half-length work items take fewer
+    // rounds' worth of time over the SMs (a half item costs a little more than half an item: 0.525)
+    const int sms = x->dev->num_sms;
+    const bool fewer_rounds = 525LL * ((2 * tiles256 + sms - 1) / sms) < 1000LL * ((tiles256 + sms - 1) / sms);
+    const bool split = ep.mode == kGemmF32 && split_out && K >= 2048 && (tiles256 < sms || fewer_rounds);
     const int bn = (tiles256 >= x->dev->num_sms || split) ? 256 : 128;
     ep.k_split = split ? 2 : 1;
     if (split_out) *split_out = split;
